@@ -1,0 +1,131 @@
+/*
+ * qgemm.h - C ABI of the B200 (sm_100a) block-quantised prefill GEMM library, dense and MoE.
+ *
+ * The operators are the ones the paper's Sec. 3.1 lists for the compute-bound prompt-processing
+ * phase: a dense GEMM over 4-bit / 8-bit block-quantised weights that reads the packed weight
+ * layout directly, the MoE expert GEMM over each expert's routed tokens, and the fused MoE
+ * gate/up projection that applies SiLU on the accumulators.  The paper does not describe routing,
+ * token permutation or the weighted combine that surround the expert GEMMs; they are defined here
+ * in the plainest way (see each call).
+ *
+ * Conventions for every compute call
+ *   - all data pointers are DEVICE pointers owned by the caller; the library never allocates,
+ *     frees or synchronises inside a compute call; the call is asynchronous on `stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream);
+ *   - return value: QG_OK (0) or a negative QG_ERR_* code; an error is detected before anything is
+ *     launched, so the outputs are untouched; nothing aborts, traps or throws;
+ *   - there is no fallback path: a shape the kernels do not accept is an error (the paper's
+ *     Sec. 3.2 "shape constraints" check, without its SIMD fallback);
+ *   - device-side waits are bounded; a wait that expires records QG_ERR_TIMEOUT in the context's
+ *     status word, the kernel exits cleanly and qg_poll_status() reports it.
+ *
+ * Data formats
+ *   activations / outputs  bf16, row-major, K (or N) contiguous
+ *   Q8 weights   int8  [N, K]      ("out x in", y = x * W^T), any value -128..127
+ *   Q4 weights   uint8 [N, K/2]    byte j of a row = weight 2j in the low nibble, 2j+1 in the high
+ *                                  nibble; nibble u in 0..15 encodes q = u - 8
+ *   scales       fp16  [N, K/32]   one per block of 32 consecutive k; w[n][k] = q[n][k]*scale[n][k/32];
+ *                                  any finite fp16 (negative, zero, subnormal) is legal
+ *   MoE weights  the same planes with a leading expert dimension E
+ *   accumulation fp32; results rounded to bf16 once (nearest even)
+ *
+ * Shape constraints (else QG_ERR_SHAPE): K % 256 == 0 (scale rows are fetched in 16-byte units),
+ * N % 8 == 0, 1 <= k <= E <= 1024, H % 8 == 0; M and R may be any value >= 0 (0 is a no-op).
+ * Pointers must be 16-byte aligned (else QG_ERR_ALIGN).
+ */
+#ifndef QGEMM_B200_H
+#define QGEMM_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qg_ctx qg_ctx; /* opaque: device id, SM count, tensor-map encoder, device status word */
+
+enum {
+    QG_OK = 0,
+    QG_ERR_NULL = -1,      /* a required pointer is NULL */
+    QG_ERR_SHAPE = -2,     /* a size violates the constraints above */
+    QG_ERR_ALIGN = -3,     /* a pointer is not 16-byte aligned */
+    QG_ERR_WORKSPACE = -4, /* workspace missing or too small */
+    QG_ERR_ARCH = -5,      /* the device is not compute capability 10.x */
+    QG_ERR_CUDA = -6,      /* a CUDA runtime / driver call failed */
+    QG_ERR_TIMEOUT = -7    /* a bounded device-side wait expired (reported by qg_poll_status) */
+};
+enum { QG_Q8 = 8, QG_Q4 = 4 };
+enum {
+    QG_MODE_PLAIN = 0,         /* Out[r, n]   = sum_k Ain[r, k] w_e[n, k]                      bf16 [R, N]   */
+    QG_MODE_GATE_UP_SILU = 1,  /* Out[r, f]   = silu(G[r, f]) * U[r, f], N = 2F               bf16 [R, N/2] */
+    QG_MODE_DOWN_WEIGHTED = 2, /* Out[r, n]   = topk_w[row_pair[r]] * (plain)                  bf16 [R, N]   */
+    QG_MODE_DOWN_ACCUM_F32 = 3 /* Out[row_pair[r] / k, n] += topk_w[row_pair[r]] * (plain)     f32  [M, N]   */
+};
+enum { QG_D_BF16 = 0, QG_D_F32_ACC = 1 };
+
+/* Create / destroy a context for `device` (these two may allocate a few bytes of device memory). */
+int qg_create(qg_ctx** out, int device);
+int qg_destroy(qg_ctx* ctx);
+const char* qg_strerror(int code);
+/* Synchronises `stream`, then returns and clears the device status word (QG_OK if no kernel gave up). */
+int qg_poll_status(qg_ctx* ctx, void* stream);
+/* Bytes of scratch moe_route needs for M tokens, E experts, top-k (per-block expert histograms). */
+size_t qg_route_workspace_bytes(int M, int E, int k);
+
+/*
+ * Dense quantised GEMM (Sec. 3.1, "Dense GEMM ... in 4-bit and 8-bit quantisation, reading the
+ * packed-quant weight layout"):  C[m, n] = sum_k A[m, k] * q[n, k] * scale[n, k/32].
+ *   qbits QG_Q8 or QG_Q4; A bf16 [M, K]; Wq / Wscale as above; C bf16 [M, N] (overwritten).
+ */
+int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq,
+                const void* Wscale, void* C, void* stream);
+
+/*
+ * Routing (the paper only says "routed tokens", Sec. 3.1; defined here): for every token the k
+ * experts that come first in the order (logit descending, expert index ascending), in that order;
+ * topk_w = softmax over those k logits (fp32).  Then the per-expert histogram, its exclusive
+ * prefix sum (expert_offsets[E] = M*k) and the stable counting sort of the pair ids p = t*k + s by
+ * expert: row_pair[r] = p of sorted row r, pair_row[p] = r.  All integer outputs are deterministic.
+ *   logits f32 [M, E]; topk_idx int32 [M, k]; topk_w f32 [M, k]; expert_counts int32 [E];
+ *   expert_offsets int32 [E+1]; row_pair, pair_row int32 [M*k].
+ *   If X (bf16 [M, H]) and Xperm (bf16 [M*k, H]) are both non-NULL the rows are also gathered:
+ *   Xperm[r, :] = X[row_pair[r] / k, :].
+ *   ws: scratch of at least qg_route_workspace_bytes(M, E, k) bytes (contents are clobbered).
+ */
+int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
+              int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row,
+              const void* X, void* Xperm, int H, void* ws, size_t ws_bytes, void* stream);
+
+/* Xperm[r, :] = X[row_pair[r] / k, :] for r in [0, M*k): bit copy of bf16 rows, H % 8 == 0. */
+int moe_permute(qg_ctx* ctx, int M, int k, int H, const void* X, const int32_t* row_pair, void* Xperm,
+                void* stream);
+
+/*
+ * Grouped quantised GEMM over expert segments (Sec. 3.1, "MoE expert GEMM" and "Fused MoE gate/up
+ * projection ... applies the SiLU activation on the tensor-core accumulators"): rows
+ * r in [expert_offsets[e], expert_offsets[e+1]) of Ain (bf16 [R, K], permuted order) are multiplied
+ * by expert e's weights (Wq [E, N, K or K/2], Wscale fp16 [E, N, K/32]).  `mode` selects the epilogue
+ * (see QG_MODE_*).  In mode 1 rows 0..F-1 of an expert's weights are the gate and F..2F-1 the up
+ * projection (N = 2F, F % 64 == 0).  Modes 2 and 3 need topk_w (f32 [M*k]) and row_pair; mode 3 also
+ * needs k and adds into a caller-zeroed f32 [M, N] with atomics (sum order not fixed).
+ * expert_offsets stays on the device; empty experts are legal.
+ */
+int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int K, const void* Ain,
+                      const int32_t* expert_offsets, const void* Wq, const void* Wscale,
+                      const float* topk_w, const int32_t* row_pair, int k, void* Out, void* stream);
+
+/*
+ * Combine (not described by the paper; plain definition): d_kind = QG_D_BF16:
+ *   Y[t, :] = sum_{s = 0..k-1, in that order, fp32} w(t, s) * D[pair_row[t*k+s], :], with
+ *   w = topk_w[t*k+s] if topk_w != NULL else 1 (rows already weighted).  D bf16 [M*k, H].
+ * d_kind = QG_D_F32_ACC: D is the f32 [M, H] accumulator of mode 3 and is only rounded to bf16.
+ * Y bf16 [M, H].
+ */
+int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
+                const float* topk_w, void* Y, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QGEMM_B200_H */

@@ -1,0 +1,171 @@
+"""Thin ctypes binding of the C-ABI library declared in include/qgemm.h.
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.  PyTorch is used
+for device memory and the current stream.  There is no fallback: if the shared library is missing or a
+call returns an error code, a QGemmError is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqgemm_b200.so")
+
+QG_Q8, QG_Q4 = 8, 4
+MODE_PLAIN, MODE_GATE_UP_SILU, MODE_DOWN_WEIGHTED, MODE_DOWN_ACCUM_F32 = 0, 1, 2, 3
+D_BF16, D_F32_ACC = 0, 1
+
+EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_route_workspace_bytes", "qgemm_dense",
+           "moe_route", "moe_permute", "moe_grouped_qgemm", "moe_combine"]
+
+
+class QGemmError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: error {code} ({strerror(code)})")
+        self.code = code
+
+
+_lib = None
+_ctx = {}
+
+
+def load():
+    """Loads libqgemm_b200.so (built by `python -m paper_2607_19438_b200.build` or __graft_entry__.build())."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise QGemmError(-6, f"CUDA library not built: {LIB_PATH} is missing (run __graft_entry__.build())")
+        lib = C.CDLL(LIB_PATH)
+        lib.qg_strerror.restype = C.c_char_p
+        lib.qg_strerror.argtypes = [C.c_int]
+        lib.qg_route_workspace_bytes.restype = C.c_size_t
+        lib.qg_route_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
+        lib.qg_create.argtypes = [C.POINTER(C.c_void_p), C.c_int]
+        lib.qg_destroy.argtypes = [C.c_void_p]
+        lib.qg_poll_status.argtypes = [C.c_void_p, C.c_void_p]
+        vp, ci = C.c_void_p, C.c_int
+        lib.qgemm_dense.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
+        lib.moe_route.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp, C.c_size_t, vp]
+        lib.moe_permute.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
+        lib.moe_grouped_qgemm.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp]
+        lib.moe_combine.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp, vp, vp]
+        _lib = lib
+    return _lib
+
+
+def strerror(code: int) -> str:
+    try:
+        return load().qg_strerror(code).decode()
+    except Exception:
+        return "?"
+
+
+def context(device: int | None = None):
+    """The per-device library context (created on first use)."""
+    if device is None:
+        device = torch.cuda.current_device()
+    if device not in _ctx:
+        h = C.c_void_p()
+        rc = load().qg_create(C.byref(h), int(device))
+        if rc != 0:
+            raise QGemmError(rc, "qg_create")
+        _ctx[device] = h
+    return _ctx[device]
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise QGemmError(rc, what)
+
+
+def poll_status():
+    """Synchronises the current stream and raises if a kernel recorded a device-side error."""
+    _check(load().qg_poll_status(context(), _stream()), "qg_poll_status")
+
+
+def route_workspace_bytes(M, E, k) -> int:
+    return int(load().qg_route_workspace_bytes(M, E, k))
+
+
+def qgemm_dense(qbits, A, Wq, Wscale, out=None):
+    """A bf16 [M,K]; Wq int8 [N,K] / uint8 [N,K/2]; Wscale fp16 [N,K/32] -> bf16 [M,N]."""
+    M, K = A.shape
+    N = Wq.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=A.device)
+    _check(load().qgemm_dense(context(), qbits, M, N, K, _ptr(A), _ptr(Wq), _ptr(Wscale), _ptr(out), _stream()),
+           "qgemm_dense")
+    return out
+
+
+def moe_route(logits, k, X=None, ws=None):
+    """logits f32 [M,E] -> dict(topk_idx, topk_w, counts, offsets, row_pair, pair_row[, Xperm])."""
+    M, E = logits.shape
+    dev = logits.device
+    i32 = dict(dtype=torch.int32, device=dev)
+    out = dict(topk_idx=torch.empty((M, k), **i32), topk_w=torch.empty((M, k), dtype=torch.float32, device=dev),
+               counts=torch.empty(E, **i32), offsets=torch.empty(E + 1, **i32),
+               row_pair=torch.empty(M * k, **i32), pair_row=torch.empty(M * k, **i32))
+    H = 0
+    Xp = None
+    if X is not None:
+        H = X.shape[1]
+        Xp = torch.empty((M * k, H), dtype=torch.bfloat16, device=dev)
+        out["Xperm"] = Xp
+    need = route_workspace_bytes(M, E, k)
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    _check(load().moe_route(context(), M, E, k, _ptr(logits), _ptr(out["topk_idx"]), _ptr(out["topk_w"]),
+                            _ptr(out["counts"]), _ptr(out["offsets"]), _ptr(out["row_pair"]), _ptr(out["pair_row"]),
+                            _ptr(X), _ptr(Xp), H, _ptr(ws), ws.numel(), _stream()), "moe_route")
+    return out
+
+
+def moe_permute(X, row_pair, k, out=None):
+    M, H = X.shape
+    if out is None:
+        out = torch.empty((M * k, H), dtype=torch.bfloat16, device=X.device)
+    _check(load().moe_permute(context(), M, k, H, _ptr(X), _ptr(row_pair), _ptr(out), _stream()), "moe_permute")
+    return out
+
+
+def moe_grouped_qgemm(mode, qbits, Ain, offsets, Wq, Wscale, topk_w=None, row_pair=None, k=1, out=None, M=None):
+    """Ain bf16 [R,K]; Wq [E,N,K(/2)]; Wscale fp16 [E,N,K/32]; see include/qgemm.h for the modes."""
+    R, K = Ain.shape
+    E, N = Wscale.shape[0], Wscale.shape[1]
+    dev = Ain.device
+    if out is None:
+        if mode == MODE_GATE_UP_SILU:
+            out = torch.empty((R, N // 2), dtype=torch.bfloat16, device=dev)
+        elif mode == MODE_DOWN_ACCUM_F32:
+            out = torch.zeros((M if M is not None else R // k, N), dtype=torch.float32, device=dev)
+        else:
+            out = torch.empty((R, N), dtype=torch.bfloat16, device=dev)
+    _check(load().moe_grouped_qgemm(context(), mode, qbits, R, E, N, K, _ptr(Ain), _ptr(offsets), _ptr(Wq),
+                                    _ptr(Wscale), _ptr(topk_w), _ptr(row_pair), k, _ptr(out), _stream()),
+           "moe_grouped_qgemm")
+    return out
+
+
+def moe_combine(D, pair_row, k, topk_w=None, d_kind=D_BF16, out=None):
+    if d_kind == D_F32_ACC:
+        M, H = D.shape
+    else:
+        H = D.shape[1]
+        M = D.shape[0] // k
+    if out is None:
+        out = torch.empty((M, H), dtype=torch.bfloat16, device=D.device)
+    _check(load().moe_combine(context(), M, k, H, _ptr(D), d_kind, _ptr(pair_row), _ptr(topk_w), _ptr(out), _stream()),
+           "moe_combine")
+    return out

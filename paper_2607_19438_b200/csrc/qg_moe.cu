@@ -1,0 +1,307 @@
+// MoE routing, segment bookkeeping, row permutation and combine kernels (HBM-bound, no tensor cores).
+//
+// The paper only speaks of each expert's "routed tokens" (Sec. 3.1); these kernels implement the
+// plain definitions stated in include/qgemm.h.  All integer outputs are deterministic: the
+// permutation is a stable counting sort built from per-block histograms, a scan and in-order ranks,
+// never from the completion order of atomics.
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "qg_internal.h"
+
+namespace qg {
+
+constexpr int ROUTE_TOKENS_PER_BLOCK = 32;  // tokens whose pairs form one histogram / scatter block
+constexpr int ROUTE_WARPS = 8;
+
+// Order of experts for one token: larger logit first, equal logits (IEEE ==, so -0 == +0) by lower
+// index; NaN after every number.
+__device__ __forceinline__ bool route_before(float a, int ia, float b, int ib) {
+    const bool na = (a != a), nb = (b != b);
+    if (na || nb) return (na == nb) ? (ia < ib) : nb;
+    if (a != b) return a > b;
+    return ia < ib;
+}
+
+// One warp per token (each warp walks ROUTE_TOKENS_PER_BLOCK / ROUTE_WARPS tokens).  Lane l owns the
+// logits e = l, l+32, ...; k rounds of (local best, warp arg-best by shuffles, mark taken).
+// Dynamic shared memory: per warp E floats (logits) + k floats (selected logits); then E ints (hist).
+__global__ void __launch_bounds__(ROUTE_WARPS * 32)
+route_topk_kernel(int M, int E, int k, const float* __restrict__ logits, int32_t* __restrict__ topk_idx,
+                  float* __restrict__ topk_w, int32_t* __restrict__ block_hist) {
+    extern __shared__ float sm[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* lg = sm + warp * (E + k);
+    float* sel = lg + E;
+    int* hist = reinterpret_cast<int*>(sm + ROUTE_WARPS * (E + k));
+    for (int e = threadIdx.x; e < E; e += blockDim.x) hist[e] = 0;
+    __syncthreads();
+
+    const int t0 = blockIdx.x * ROUTE_TOKENS_PER_BLOCK;
+    for (int tt = warp; tt < ROUTE_TOKENS_PER_BLOCK; tt += ROUTE_WARPS) {
+        const int t = t0 + tt;
+        if (t >= M) break;
+        const float* row = logits + static_cast<size_t>(t) * E;
+        for (int e = lane; e < E; e += 32) lg[e] = row[e];
+        __syncwarp();
+        uint32_t taken = 0;  // bit i: element lane + 32 i already selected
+        for (int s = 0; s < k; ++s) {
+            float bv = 0.f;
+            int bi = -1;
+            for (int e = lane, i = 0; e < E; e += 32, ++i) {
+                if ((taken >> i) & 1u) continue;
+                const float v = lg[e];
+                if (bi < 0 || route_before(v, e, bv, bi)) { bv = v; bi = e; }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, off);
+                const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, off);
+                if (oi >= 0 && (bi < 0 || route_before(ov, oi, bv, bi))) { bv = ov; bi = oi; }
+            }
+            if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
+            if (lane == 0) {
+                sel[s] = bv;
+                topk_idx[static_cast<size_t>(t) * k + s] = bi;
+                atomicAdd(&hist[bi], 1);
+            }
+        }
+        __syncwarp();
+        // softmax over the k selected logits; sel[0] is the maximum.
+        const float top = sel[0];
+        float part = 0.f;
+        for (int s = lane; s < k; s += 32) part += expf(sel[s] - top);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, off);
+        for (int s = lane; s < k; s += 32) topk_w[static_cast<size_t>(t) * k + s] = expf(sel[s] - top) / part;
+        __syncwarp();
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) block_hist[static_cast<size_t>(blockIdx.x) * E + e] = hist[e];
+}
+
+// One block.  block_hist [nb, E] -> exclusive prefix over blocks (in place), counts, offsets.
+// Thread (g, e): group g of G = blockDim / Epad walks a contiguous range of blocks.
+__global__ void __launch_bounds__(1024)
+route_scan_kernel(int nb, int E, int32_t* __restrict__ block_hist, int32_t* __restrict__ counts,
+                  int32_t* __restrict__ offsets) {
+    __shared__ int part[1024];
+    __shared__ int tot[1024];
+    const int G = 1024 / E > 0 ? 1024 / E : 1;
+    const int g = threadIdx.x / E, e = threadIdx.x % E;
+    const bool active = g < G;
+    const int per = (nb + G - 1) / G;
+    const int b0 = g * per, b1 = min(nb, b0 + per);
+    int sum = 0;
+    if (active)
+        for (int b = b0; b < b1; ++b) sum += block_hist[static_cast<size_t>(b) * E + e];
+    if (active) part[g * E + e] = sum;
+    __syncthreads();
+    int base = 0, total = 0;
+    if (active) {
+        for (int gg = 0; gg < G; ++gg) {
+            const int v = part[gg * E + e];
+            if (gg < g) base += v;
+            total += v;
+        }
+        int run = base;
+        for (int b = b0; b < b1; ++b) {
+            const size_t i = static_cast<size_t>(b) * E + e;
+            const int c = block_hist[i];
+            block_hist[i] = run;
+            run += c;
+        }
+        if (g == 0) { counts[e] = total; tot[e] = total; }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {  // E <= 1024: a serial prefix over shared memory is a few microseconds
+        int run = 0;
+        for (int i = 0; i < E; ++i) { offsets[i] = run; run += tot[i]; }
+        offsets[E] = run;
+    }
+}
+
+// Block b re-reads its pairs in ascending pair id and gives each the next free row of its expert:
+// row = offsets[e] + (pairs of e in earlier blocks) + (pairs of e earlier in this block).
+__global__ void __launch_bounds__(ROUTE_WARPS * 32)
+route_scatter_kernel(int M, int E, int k, const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ offsets,
+                     const int32_t* __restrict__ block_base, int32_t* __restrict__ row_pair,
+                     int32_t* __restrict__ pair_row) {
+    extern __shared__ int run[];  // E running row cursors
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int e = threadIdx.x; e < E; e += blockDim.x)
+        run[e] = offsets[e] + block_base[static_cast<size_t>(blockIdx.x) * E + e];
+    __syncthreads();
+    const long long p0 = static_cast<long long>(blockIdx.x) * ROUTE_TOKENS_PER_BLOCK * k;
+    const long long pend = min(static_cast<long long>(M) * k, p0 + static_cast<long long>(ROUTE_TOKENS_PER_BLOCK) * k);
+    for (long long base = p0; base < pend; base += blockDim.x) {
+        const long long p = base + threadIdx.x;
+        const bool valid = p < pend;
+        const int e = valid ? topk_idx[p] : (E + lane);
+        const uint32_t same = __match_any_sync(0xFFFFFFFFu, e);
+        const int rank = __popc(same & ((1u << lane) - 1u));
+        const int cnt = __popc(same);
+        for (int w = 0; w < ROUTE_WARPS; ++w) {
+            if (warp == w) {
+                int pos = 0;
+                if (valid) pos = run[e] + rank;
+                __syncwarp();
+                if (valid && rank == 0) run[e] += cnt;
+                if (valid) {
+                    row_pair[pos] = static_cast<int32_t>(p);
+                    pair_row[p] = pos;
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// Xperm[r, :] = X[row_pair[r] / k, :]; one warp per row, 16-byte vectors.
+__global__ void __launch_bounds__(256)
+permute_rows_kernel(int R, int k, int H8, const int4* __restrict__ X, const int32_t* __restrict__ row_pair,
+                    int4* __restrict__ Xp) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (int r = warp; r < R; r += nwarps) {
+        const int t = row_pair[r] / k;
+        const int4* src = X + static_cast<size_t>(t) * H8;
+        int4* dst = Xp + static_cast<size_t>(r) * H8;
+        for (int v = lane; v < H8; v += 32) dst[v] = __ldg(src + v);
+    }
+}
+
+__device__ __forceinline__ void add8(float (&acc)[8], const int4& v, float w) {
+    const uint32_t u[4] = {static_cast<uint32_t>(v.x), static_cast<uint32_t>(v.y), static_cast<uint32_t>(v.z),
+                           static_cast<uint32_t>(v.w)};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        acc[2 * i] = fmaf(w, __uint_as_float(u[i] << 16), acc[2 * i]);
+        acc[2 * i + 1] = fmaf(w, __uint_as_float(u[i] & 0xFFFF0000u), acc[2 * i + 1]);
+    }
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&b);
+}
+
+// Y[t, :] = sum_s w(t, s) * D[pair_row[t k + s], :] in slot order; one block per token.
+__global__ void __launch_bounds__(256)
+combine_kernel(int M, int k, int H8, const int4* __restrict__ D, const int32_t* __restrict__ pair_row,
+               const float* __restrict__ topk_w, int4* __restrict__ Y) {
+    const int t = blockIdx.x;
+    for (int v = threadIdx.x; v < H8; v += blockDim.x) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int s = 0; s < k; ++s) {
+            const int row = pair_row[static_cast<size_t>(t) * k + s];
+            const float w = topk_w ? topk_w[static_cast<size_t>(t) * k + s] : 1.0f;
+            add8(acc, __ldg(D + static_cast<size_t>(row) * H8 + v), w);
+        }
+        int4 o;
+        o.x = pack_bf16x2(acc[0], acc[1]); o.y = pack_bf16x2(acc[2], acc[3]);
+        o.z = pack_bf16x2(acc[4], acc[5]); o.w = pack_bf16x2(acc[6], acc[7]);
+        Y[static_cast<size_t>(t) * H8 + v] = o;
+    }
+}
+
+// Y = bf16(acc) for the f32 accumulator produced by the atomic-accumulate epilogue.
+__global__ void __launch_bounds__(256)
+round_f32_kernel(size_t n8, const float4* __restrict__ acc, int4* __restrict__ Y) {
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n8;
+         i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const float4 a = acc[2 * i], b = acc[2 * i + 1];
+        int4 o;
+        o.x = pack_bf16x2(a.x, a.y); o.y = pack_bf16x2(a.z, a.w);
+        o.z = pack_bf16x2(b.x, b.y); o.w = pack_bf16x2(b.z, b.w);
+        Y[i] = o;
+    }
+}
+
+static int launch_ok() { return cudaGetLastError() == cudaSuccess ? QG_OK : QG_ERR_CUDA; }
+
+}  // namespace qg
+
+extern "C" {
+
+size_t qg_route_workspace_bytes(int M, int E, int k) {
+    (void)k;
+    if (M <= 0 || E <= 0) return 16;
+    const size_t nb = (static_cast<size_t>(M) + qg::ROUTE_TOKENS_PER_BLOCK - 1) / qg::ROUTE_TOKENS_PER_BLOCK;
+    return nb * static_cast<size_t>(E) * sizeof(int32_t);
+}
+
+int moe_permute(qg_ctx* ctx, int M, int k, int H, const void* X, const int32_t* row_pair, void* Xperm, void* stream) {
+    if (!ctx || !X || !row_pair || !Xperm) return QG_ERR_NULL;
+    if (M < 0 || k < 1 || H < 8 || H % 8) return QG_ERR_SHAPE;
+    if (!qg::aligned16(X) || !qg::aligned16(Xperm)) return QG_ERR_ALIGN;
+    const long long R = static_cast<long long>(M) * k;
+    if (R == 0) return QG_OK;
+    if (R > 0x7FFFFFFF) return QG_ERR_SHAPE;
+    const int blocks = static_cast<int>(min(static_cast<long long>(ctx->sm_count) * 8, (R + 7) / 8));
+    qg::permute_rows_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<int>(R), k, H / 8, static_cast<const int4*>(X), row_pair, static_cast<int4*>(Xperm));
+    return qg::launch_ok();
+}
+
+int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
+              int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row, const void* X,
+              void* Xperm, int H, void* ws, size_t ws_bytes, void* stream) {
+    if (!ctx || !logits || !topk_idx || !topk_w || !expert_counts || !expert_offsets || !row_pair || !pair_row)
+        return QG_ERR_NULL;
+    if (M < 0 || E < 1 || E > 1024 || k < 1 || k > E) return QG_ERR_SHAPE;
+    if (static_cast<long long>(M) * k > 0x7FFFFFFF) return QG_ERR_SHAPE;
+    const bool gather = (X != nullptr) && (Xperm != nullptr);
+    if (gather && (H < 8 || H % 8)) return QG_ERR_SHAPE;
+    if (gather && (!qg::aligned16(X) || !qg::aligned16(Xperm))) return QG_ERR_ALIGN;
+    if (!ws || ws_bytes < qg_route_workspace_bytes(M, E, k)) return QG_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* hist = static_cast<int32_t*>(ws);
+    const int nb = (M + qg::ROUTE_TOKENS_PER_BLOCK - 1) / qg::ROUTE_TOKENS_PER_BLOCK;
+    if (M == 0) {  // no pairs: counts and offsets are all zero
+        if (cudaMemsetAsync(expert_counts, 0, sizeof(int32_t) * E, st) != cudaSuccess ||
+            cudaMemsetAsync(expert_offsets, 0, sizeof(int32_t) * (E + 1), st) != cudaSuccess) {
+            cudaGetLastError();
+            return QG_ERR_CUDA;
+        }
+        return QG_OK;
+    }
+    const size_t sm_topk = (static_cast<size_t>(qg::ROUTE_WARPS) * (E + k) + E) * sizeof(float);
+    if (sm_topk > 48 * 1024) {
+        if (cudaFuncSetAttribute(qg::route_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(sm_topk)) != cudaSuccess) {
+            cudaGetLastError();
+            return QG_ERR_CUDA;
+        }
+    }
+    qg::route_topk_kernel<<<nb, qg::ROUTE_WARPS * 32, sm_topk, st>>>(M, E, k, logits, topk_idx, topk_w, hist);
+    qg::route_scan_kernel<<<1, 1024, 0, st>>>(nb, E, hist, expert_counts, expert_offsets);
+    qg::route_scatter_kernel<<<nb, qg::ROUTE_WARPS * 32, E * sizeof(int), st>>>(M, E, k, topk_idx, expert_offsets, hist,
+                                                                               row_pair, pair_row);
+    int rc = qg::launch_ok();
+    if (rc != QG_OK) return rc;
+    if (gather) return moe_permute(ctx, M, k, H, X, row_pair, Xperm, stream);
+    return QG_OK;
+}
+
+int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
+                const float* topk_w, void* Y, void* stream) {
+    if (!ctx || !D || !Y) return QG_ERR_NULL;
+    if (M < 0 || k < 1 || H < 8 || H % 8) return QG_ERR_SHAPE;
+    if (d_kind != QG_D_BF16 && d_kind != QG_D_F32_ACC) return QG_ERR_SHAPE;
+    if (!qg::aligned16(D) || !qg::aligned16(Y)) return QG_ERR_ALIGN;
+    if (M == 0) return QG_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (d_kind == QG_D_F32_ACC) {
+        const size_t n8 = static_cast<size_t>(M) * H / 8;
+        const int blocks = static_cast<int>(min(static_cast<size_t>(ctx->sm_count) * 8, (n8 + 255) / 256));
+        qg::round_f32_kernel<<<blocks, 256, 0, st>>>(n8, static_cast<const float4*>(D), static_cast<int4*>(Y));
+        return qg::launch_ok();
+    }
+    if (!pair_row) return QG_ERR_NULL;
+    qg::combine_kernel<<<M, 256, 0, st>>>(M, k, H / 8, static_cast<const int4*>(D), pair_row, topk_w,
+                                         static_cast<int4*>(Y));
+    return qg::launch_ok();
+}
+
+}  // extern "C"

@@ -1,0 +1,97 @@
+"""GPU parity: qgemm_dense against the fp64 oracle (max|err| <= 2e-2 max|ref|, relative Frobenius <= 5e-3),
+plus integer-exact cases that must match bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2607_19438_b200 import binding as qg, synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def run_dense(qbits, A, Wq, Ws):
+    out = qg.qgemm_dense(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws))
+    qg.poll_status()
+    return out
+
+
+SHAPES = [
+    (8, 128, 2048, 2048),    # config 0
+    (4, 128, 2048, 2048),
+    (8, 300, 384, 512),      # ragged token tail, three weight tiles
+    (4, 300, 384, 512),
+    (8, 1, 128, 256), (4, 1, 128, 256),
+    (8, 17, 200, 256),       # N not a multiple of the weight tile
+    (4, 513, 136, 768),      # three token tiles of 256 with a tail of 1
+    (8, 257, 2560, 2048), (4, 1024, 3072, 1024),
+]
+
+
+@pytest.mark.parametrize("qbits,M,N,K", SHAPES, ids=[f"q{s[0]}-{s[1]}x{s[2]}x{s[3]}" for s in SHAPES])
+def test_dense_parity(qbits, M, N, K):
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=0)
+    out = run_dense(qbits, A, Wq, Ws)
+    ref = orc.qgemm_dense(qbits, A, Wq, Ws)
+    mx, rmax, fro = util.assert_close(util.host_bf16_f64(out), ref, f"dense q{qbits} {M}x{N}x{K}")
+    assert fro > 1e-4, "suspiciously exact: is the reference rounded?"
+
+
+@pytest.mark.parametrize("qbits", [8, 4])
+def test_dense_integer_exact_is_bit_exact(qbits):
+    """A in {-1,0,1}, power-of-two scales, K=256: every partial sum is an integer multiple of a power of two that
+    fp32 holds exactly, and the results fit bf16, so the GPU must reproduce the oracle bit for bit."""
+    M, N, K = 200, 256, 256
+    rng = np.random.default_rng(11)
+    A = synth.f32_to_bf16_bits(rng.integers(-1, 2, (M, K)).astype(np.float32))
+    if qbits == 8:
+        Wq = rng.integers(-3, 4, (N, K)).astype(np.int8)
+        Wq[0, :] = 0; Wq[0, 5] = -128; Wq[1, :] = 0; Wq[1, 255] = 127
+    else:
+        Wq = rng.integers(0, 256, (N, K // 2)).astype(np.uint8)
+        Wq[:, 8:] = 0x88                     # only the first 16 weights of each row are non-zero
+    Ws = (2.0 ** rng.integers(-3, 2, (N, K // 32))).astype(np.float16).view(np.uint16)
+    out = run_dense(qbits, A, Wq, Ws)
+    ref = orc.qgemm_dense(qbits, A, Wq, Ws)
+    assert np.array_equal(orc.bf16_to_f64(orc.f64_to_bf16(ref)), ref), "case is not exactly representable"
+    assert np.array_equal(util.host_bf16_f64(out), ref)
+
+
+@pytest.mark.parametrize("qbits", [8, 4])
+def test_dense_extreme_codes_and_scales(qbits):
+    """q = -128 / -8, negative, zero and subnormal fp16 scales (never flushed)."""
+    M, N, K = 64, 128, 512
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=2)
+    Ws = Ws.copy()
+    if qbits == 8:
+        Wq = Wq.copy(); Wq[::3, ::5] = -128
+    else:
+        Wq = Wq.copy(); Wq[::3, ::5] = 0x00      # both codes 0 -> q = -8
+    s = Ws.view(np.float16)
+    s[0::4, :] = -s[0::4, :]
+    s[1::4, 0] = 0.0
+    Ws[2::4, :] = np.arange(1, K // 32 + 1, dtype=np.uint16)      # subnormals 2^-24 .. 16 * 2^-24
+    out = run_dense(qbits, A, Wq, Ws)
+    ref = orc.qgemm_dense(qbits, A, Wq, Ws)
+    util.assert_close(util.host_bf16_f64(out), ref, "extreme")
+    sub = util.host_bf16_f64(out)[:, 2::4]
+    assert np.any(sub != 0.0), "subnormal scales were flushed to zero"
+    util.assert_close(sub, ref[:, 2::4], "subnormal rows")
+
+
+def test_dense_full_size_sampled_config1_gate_up():
+    """Config 1 gate/up projection at M = 2048 (the bench's launch configuration), checked on sampled outputs that
+    hit every 128-column and every 256-row tile."""
+    qbits, M, N, K = 8, 2048, 16384, 2048
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=0)
+    out = util.host_bf16_f64(run_dense(qbits, A, Wq, Ws))
+    rng = np.random.default_rng(0)
+    rows, cols = [], []
+    for rt in range(M // 128):
+        for ct in range(N // 128):
+            rows.append(rt * 128 + rng.integers(0, 128, 2)); cols.append(ct * 128 + rng.integers(0, 128, 2))
+    rows = np.concatenate(rows); cols = np.concatenate(cols)
+    ref = orc.qgemm_dense_sample(qbits, A, Wq, Ws, rows, cols)
+    util.assert_close(out[rows, cols], ref, "config 1 gate/up sampled")
+    assert np.all(np.isfinite(out))
