@@ -32,9 +32,10 @@ def gpu_layer(qbits, logits, X, W1q, W1s, W2q, W2s, k, fused_combine=False):
 
 
 CASES = [
-    ("small-q4", 4, 96, 256, 8, 128, 2, False), ("small-q8", 8, 96, 256, 8, 128, 2, False),
-    ("empty-experts-q4", 4, 5, 256, 16, 64, 2, False), ("k-eq-E-q8", 8, 40, 256, 4, 64, 4, False),
-    ("long-segments-q4", 4, 700, 256, 2, 128, 1, False), ("skewed-q4", 4, 512, 512, 32, 256, 8, True),
+    ("small-q4", 4, 96, 256, 8, 256, 2, False), ("small-q8", 8, 96, 256, 8, 256, 2, False),
+    ("empty-experts-q4", 4, 5, 256, 16, 256, 2, False), ("k-eq-E-q8", 8, 40, 512, 4, 256, 4, False),
+    ("long-segments-q4", 4, 700, 256, 2, 256, 1, False), ("long-segments-q8", 8, 650, 256, 3, 512, 2, False),
+    ("skewed-q4", 4, 512, 512, 32, 256, 8, True),
 ]
 
 
@@ -74,6 +75,6 @@ def test_moe_config3_shape_reduced_tokens():
     r, Hh, Dw, y, d = gpu_layer(qbits, logits, X, W1q, W1s, W2q, W2s, k)
     o = orc.moe_layer(qbits, logits, X, W1q, W1s, W2q, W2s, k)
     assert np.array_equal(r["row_pair"].cpu().numpy(), o["row_pair"])
-    assert (o["counts"] == 0).any()
+    assert o["counts"].min() <= 2 and o["counts"].max() >= 20      # short and long segments in one launch
     util.assert_close(util.host_bf16_f64(Hh), o["Hh"], "gate/up+silu cfg3")
     util.assert_close(util.host_bf16_f64(y), o["y"], "layer cfg3")
