@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the quantised prefill GEMM path on B200: one JSON line on stdout.
+
+A step is one pass of the whole hot path over one batch of synthetic input at M = 2048 tokens:
+  * the 2B-class dense Q8 layer set (QKV 2048->2560, O 2048->2048, gate/up 2048->16384, down 8192->2048):
+    four qgemm_dense calls;
+  * the 30B-A3B-shaped MoE Q4 layer (H=2048, E=128, top-8, F=768): moe_route (+ row gather),
+    moe_grouped_qgemm gate/up+SiLU, moe_grouped_qgemm down with routing weights, moe_combine.
+`value` is algorithmic TFLOP/s (2*M*N*K per dense GEMM, 2*R*3*F*H for the MoE layer, R = M*k) over the
+device-timed region with inputs resident in HBM; `e2e` repeats the step through the same C-ABI calls with the
+activations and logits in pinned host memory (copied in every step) and every output copied back.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+--impl reference times the CPU oracle (fp64, naive) on a bounded sample of the same workload.
+Under torchrun every rank runs its own replica of the step (the path shards by tokens with no exchange).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "Q4/Q8 prefill GEMM TFLOP/s & tok/s (dense+MoE), % of B200 bf16 tensor peak"
+M_TOKENS = 2048
+DENSE_SET = [("qkv", 2560, 2048), ("o", 2048, 2048), ("gate_up", 16384, 2048), ("down", 2048, 8192)]  # (name, N, K)
+MOE = dict(H=2048, E=128, k=8, F=768)
+# DRAM bytes per launch of the dominant kernel measured once with ncu (see profiles/); None until captured.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def dense_flops(M):
+    return sum(2.0 * M * N * K for _, N, K in DENSE_SET)
+
+
+def moe_flops(M):
+    return 2.0 * M * MOE["k"] * 3 * MOE["F"] * MOE["H"]
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["bf16_tflops"]), float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json, cuBLAS bf16 burst)"
+    return 1590.0, 6650.0, "fallback (earlier measurement on this pool)"
+
+
+# ------------------------------------------------------------------------------------------ synthetic inputs
+def host_inputs(M, seed):
+    from paper_2607_19438_b200 import synth
+    dense = []
+    for i, (name, N, K) in enumerate(DENSE_SET):
+        A, Wq, Ws = synth.dense_problem(8, M, N, K, seed=seed, tid_base=16 * (i + 1))
+        dense.append((name, A, Wq, Ws))
+    moe = synth.moe_problem(4, M, MOE["H"], MOE["E"], MOE["F"], seed=seed)
+    return dense, moe
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle arm
+def oracle_sample_step(dense, moe, m_dense, m_moe):
+    """Runs the oracle on the first m_dense rows of every dense GEMM and the first m_moe tokens of the MoE layer."""
+    from oracle import oracle as orc
+    for _, A, Wq, Ws in dense:
+        orc.qgemm_dense(8, A[:m_dense], Wq, Ws)
+    logits, X, W1q, W1s, W2q, W2s = moe
+    orc.moe_layer(4, logits[:m_moe], X[:m_moe], W1q, W1s, W2q, W2s, MOE["k"])
+    return dense_flops(m_dense) + moe_flops(m_moe)
+
+
+def cpu_baseline(dense, moe, m_dense=128, m_moe=64):
+    from oracle import oracle as orc
+    t = time.perf_counter()
+    fl = oracle_sample_step(dense, moe, m_dense, m_moe)
+    dt = time.perf_counter() - t
+    return {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"first {m_dense} of {M_TOKENS} rows of the 4 dense Q8 GEMMs + first {m_moe} tokens of the MoE Q4 "
+                      f"layer, fp64 naive, {dt:.1f} s",
+            "tok_per_s": 1.0 / (dense_flops(1) + moe_flops(1)) * fl / dt}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle as orc
+    dense, moe = host_inputs(M_TOKENS, seed=0)
+    # calibrate on a tiny sample, then size a step so that the whole run stays within a few minutes
+    t = time.perf_counter(); fl = oracle_sample_step(dense, moe, 2, 2); rate = fl / (time.perf_counter() - t)
+    budget = min(3.0, 150.0 / max(1, args.steps + args.warmup))
+    per_tok = dense_flops(1) + moe_flops(1)
+    m = int(max(1, min(128, rate * budget / per_tok)))
+    for _ in range(args.warmup):
+        oracle_sample_step(dense, moe, m, m)
+    t0 = time.perf_counter()
+    total = 0.0
+    for _ in range(args.steps):
+        total += oracle_sample_step(dense, moe, m, m)
+    dt = time.perf_counter() - t0
+    val = total / dt / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"cfg1 dense Q8 layer set + cfg3 MoE Q4 layer, M={M_TOKENS} (oracle on a sample)"},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "kind": "oracle", "cores": orc.num_threads(),
+                             "sample": f"each step: first {m} rows of the 4 dense GEMMs + first {m} tokens of the MoE layer"},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "20", "-i", str(index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill(); out = ""
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.strip().splitlines():
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "power_w_max": float(max(pw)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2607_19438_b200 import binding as qg
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    M = M_TOKENS
+    dense_h, moe_h = host_inputs(M, seed=rank)
+
+    def bf16(a): return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16)
+    def f16(a): return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.float16)
+    def raw(a): return torch.from_numpy(np.ascontiguousarray(a))
+
+    # weights live in HBM (model state); activations and logits have a pinned host copy for the e2e leg
+    dW = [(name, raw(Wq).to(dev), f16(Ws).to(dev)) for name, _, Wq, Ws in dense_h]
+    hA = [bf16(A).pin_memory() for _, A, _, _ in dense_h]
+    logits_h, X_h, W1q, W1s, W2q, W2s = moe_h
+    hL, hX = raw(logits_h).pin_memory(), bf16(X_h).pin_memory()
+    dW1q, dW1s, dW2q, dW2s = raw(W1q).to(dev), f16(W1s).to(dev), raw(W2q).to(dev), f16(W2s).to(dev)
+    dA = [a.to(dev) for a in hA]
+    dL, dX = hL.to(dev), hX.to(dev)
+    k, E, H, F = MOE["k"], MOE["E"], MOE["H"], MOE["F"]
+    R = M * k
+    i32 = dict(dtype=torch.int32, device=dev)
+    # all outputs and scratch preallocated: nothing is allocated inside a step
+    oC = [torch.empty((M, N), dtype=torch.bfloat16, device=dev) for _, N, _ in DENSE_SET]
+    ws = torch.empty(max(16, qg.route_workspace_bytes(M, E, k)), dtype=torch.uint8, device=dev)
+    o = dict(idx=torch.empty((M, k), **i32), w=torch.empty((M, k), dtype=torch.float32, device=dev),
+             counts=torch.empty(E, **i32), offsets=torch.empty(E + 1, **i32), row_pair=torch.empty(R, **i32),
+             pair_row=torch.empty(R, **i32), Xp=torch.empty((R, H), dtype=torch.bfloat16, device=dev),
+             Hh=torch.empty((R, F), dtype=torch.bfloat16, device=dev),
+             Dw=torch.empty((R, H), dtype=torch.bfloat16, device=dev), y=torch.empty((M, H), dtype=torch.bfloat16, device=dev))
+    hC = [torch.empty((M, N), dtype=torch.bfloat16).pin_memory() for _, N, _ in DENSE_SET]
+    hY = torch.empty((M, H), dtype=torch.bfloat16).pin_memory()
+
+    lib, ctx = qg.load(), qg.context(local)
+    import ctypes as C
+    P = lambda t: C.c_void_p(t.data_ptr())
+    stream = torch.cuda.current_stream()
+    S = C.c_void_p(stream.cuda_stream)
+    gemm_events = []   # (label, flops, start, end) recorded inside the timed region
+
+    def chk(rc, what):
+        if rc != 0:
+            raise qg.QGemmError(rc, what)
+
+    def step(A_list, L, X, record=False):
+        for i, (name, N, K) in enumerate(DENSE_SET):
+            if record:
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+            chk(lib.qgemm_dense(ctx, 8, M, N, K, P(A_list[i]), P(dW[i][1]), P(dW[i][2]), P(oC[i]), S), "qgemm_dense")
+            if record:
+                e1.record(stream); gemm_events.append(("dense_q8", 2.0 * M * N * K, e0, e1))
+        if record:
+            r0 = torch.cuda.Event(enable_timing=True); r1 = torch.cuda.Event(enable_timing=True); r0.record(stream)
+        chk(lib.moe_route(ctx, M, E, k, P(L), P(o["idx"]), P(o["w"]), P(o["counts"]), P(o["offsets"]), P(o["row_pair"]),
+                          P(o["pair_row"]), P(X), P(o["Xp"]), H, P(ws), ws.numel(), S), "moe_route")
+        if record:
+            r1.record(stream); gemm_events.append(("route_permute", 0.0, r0, r1))
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+        chk(lib.moe_grouped_qgemm(ctx, qg.MODE_GATE_UP_SILU, 4, R, E, 2 * F, H, P(o["Xp"]), P(o["offsets"]), P(dW1q),
+                                  P(dW1s), None, None, k, P(o["Hh"]), S), "moe_grouped_qgemm gate/up")
+        if record:
+            e1.record(stream); gemm_events.append(("moe_gate_up_q4", 2.0 * R * 2 * F * H, e0, e1))
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+        chk(lib.moe_grouped_qgemm(ctx, qg.MODE_DOWN_WEIGHTED, 4, R, E, H, F, P(o["Hh"]), P(o["offsets"]), P(dW2q),
+                                  P(dW2s), P(o["w"]), P(o["row_pair"]), k, P(o["Dw"]), S), "moe_grouped_qgemm down")
+        if record:
+            e1.record(stream); gemm_events.append(("moe_down_q4", 2.0 * R * F * H, e0, e1))
+            c0 = torch.cuda.Event(enable_timing=True); c1 = torch.cuda.Event(enable_timing=True); c0.record(stream)
+        chk(lib.moe_combine(ctx, M, k, H, P(o["Dw"]), qg.D_BF16, P(o["pair_row"]), None, P(o["y"]), S), "moe_combine")
+        if record:
+            c1.record(stream); gemm_events.append(("combine", 0.0, c0, c1))
+
+    LAUNCHES_PER_STEP = 4 + 3 + 1 + 2 + 1   # dense x4, route (topk, scan, scatter), permute, grouped x2, combine
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        sync_all()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+            dist.barrier()
+        return ms
+
+    # ---- device-resident leg
+    for _ in range(max(3, args.warmup)):
+        step(dA, dL, dX)
+    qg.poll_status()
+    sampler = ClockSampler(local) if rank == 0 else None
+    time.sleep(0.05)
+    ms = timed(lambda: step(dA, dL, dX, record=True), args.steps)
+    clocks = sampler.stop() if sampler else None
+    qg.poll_status()
+    flops_step = dense_flops(M) + moe_flops(M)
+    value = world * flops_step * args.steps / (ms * 1e-3) / 1e12
+
+    # per-kernel figures from the events recorded inside the timed region
+    agg = {}
+    for label, fl, a, b in gemm_events:
+        d = agg.setdefault(label, [0.0, 0.0, 0])
+        d[0] += fl; d[1] += a.elapsed_time(b); d[2] += 1
+    detail = {lab: {"launches": v[2], "avg_us": v[1] / v[2] * 1e3, "tflops": (v[0] / (v[1] * 1e-3) / 1e12) if v[0] else None}
+              for lab, v in agg.items()}
+    peak_tf, peak_hbm, peak_src = measured_peaks()
+    dq = agg["dense_q8"]
+    achieved = dq[0] / (dq[1] * 1e-3) / 1e12
+    roofline = {"kernel": "qgemm_kernel<Q8, 256 tokens> (qgemm_dense, 4 launches per step)", "bound": "tensor",
+                "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
+                "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "avg_launch_us": dq[1] / dq[2] * 1e3, "flops_per_launch": dq[0] / dq[2]}
+    gemm_ms = sum(v[1] for lab, v in agg.items() if v[0])
+    gemm_fl = sum(v[0] for lab, v in agg.items() if v[0])
+    dense_ms = agg["dense_q8"][1] / args.steps
+    moe_ms = sum(agg[lab][1] for lab in ("route_permute", "moe_gate_up_q4", "moe_down_q4", "combine")) / args.steps
+
+    # ---- end-to-end leg: host inputs in pinned memory, copies inside the timed region
+    def step_e2e():
+        for d, h in zip(dA, hA):
+            d.copy_(h, non_blocking=True)
+        dL.copy_(hL, non_blocking=True); dX.copy_(hX, non_blocking=True)
+        step(dA, dL, dX)
+        for h, d in zip(hC, oC):
+            h.copy_(d, non_blocking=True)
+        hY.copy_(o["y"], non_blocking=True)
+    e2e_steps = max(3, min(args.steps, 50))
+    for _ in range(3):
+        step_e2e()
+    ms_e2e = timed(step_e2e, e2e_steps)
+    h2d = sum(a.numel() * 2 for a in hA) + hL.numel() * 4 + hX.numel() * 2
+    d2h = sum(c.numel() * 2 for c in hC) + hY.numel() * 2
+    e2e_val = world * flops_step * e2e_steps / (ms_e2e * 1e-3) / 1e12
+
+    if rank == 0:
+        dense_h0, moe_h0 = dense_h, moe_h
+        cpu = cpu_baseline(dense_h0, moe_h0) if world == 1 else None
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"cfg1 dense Q8 layer set (QKV/O/gate-up/down, K=2048/8192) + cfg3 MoE Q4 layer "
+                                   f"(H=2048,E=128,top-8,F=768), M={M} tokens per GPU",
+                       "l2": "inputs exceed L2: 403 MB of weights stream per step", "parallelism": f"replicas x{world}"},
+            "tok_per_s": {"dense_q8_layer_set": world * M / (dense_ms * 1e-3), "moe_q4_layer": world * M / (moe_ms * 1e-3),
+                          "definition": "tokens / time of that layer's calls; not a whole-model figure"},
+            "gemm_only": {"tflops": gemm_fl / (gemm_ms * 1e-3) / 1e12, "frac_of_peak": gemm_fl / (gemm_ms * 1e-3) / 1e12 / peak_tf},
+            "frac_of_measured_bf16_peak": value / world / peak_tf, "frac_of_nominal_2250": value / world / 2250.0,
+            "roofline": roofline, "kernels": detail, "clocks": clocks,
+            "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps},
+            "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+        }
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
