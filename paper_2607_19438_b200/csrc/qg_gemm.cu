@@ -7,11 +7,11 @@
 // lanes) and the tokens the "N" side (up to BT = 128 or 256 per tile, TMEM columns): a weight is
 // dequantised once per tile and used by up to 256 tokens, and short expert segments only shrink N.
 //
-// Persistent CTA of 16 warps, one tile at a time, two TMEM accumulators (epilogue of tile j overlaps
+// Persistent CTA of 24 warps, one tile at a time, two TMEM accumulators (epilogue of tile j overlaps
 // the main loop of tile j+1):
 //   warp 0      TMA producer of activation tiles  X[BT, 64] (128-byte swizzle)      -> x ring
 //   warp 2      TMA producer of packed weights [128, 64] (+ scales every 4 k-blocks) -> raw ring
-//   warps 8-15  dequantise raw -> bf16 [128, 64] written in the swizzled K-major layout -> w ring
+//   warps 8-23  dequantise raw -> bf16 [128, 64] written in the swizzled K-major layout -> w ring
 //   warp 1      one thread issues tcgen05.mma (A = w ring, B = x ring, D in TMEM) and commits
 //   warps 4-7   epilogue: tcgen05.ld, fused activation / routing weight, bf16 stores
 //   warp 3      allocates and frees TMEM
@@ -26,10 +26,23 @@ namespace qg {
 
 constexpr int BW = 128;        // weight rows per tile (UMMA M)
 constexpr int BK = 64;         // k per pipeline stage (one 128-byte swizzle row of bf16)
-constexpr int NDW = 8;         // dequantising warps
-constexpr int NTHREADS = 512;
+constexpr int NDW = 16;        // dequantising warps
+constexpr int NTHREADS = 768;
 constexpr int MAX_E = 1024;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
+
+// Profiling builds (-DQG_PROFILE) accumulate, per CTA, the cycles each role spends in each wait.
+#ifdef QG_PROFILE
+#define QG_T0() long long qg_t0_ = clock64()
+#define QG_ACC(slot) do { if (p.stats) { long long now_ = clock64(); qg_stat_[slot] += now_ - qg_t0_; qg_t0_ = now_; } } while (0)
+#define QG_DECL() long long qg_stat_[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
+#define QG_FLUSH() do { if (p.stats) for (int i_ = 0; i_ < 12; ++i_) if (qg_stat_[i_]) atomicAdd(reinterpret_cast<unsigned long long*>(p.stats) + blockIdx.x * 12 + i_, static_cast<unsigned long long>(qg_stat_[i_])); } while (0)
+#else
+#define QG_T0() do {} while (0)
+#define QG_ACC(slot) do {} while (0)
+#define QG_DECL() do {} while (0)
+#define QG_FLUSH() do {} while (0)
+#endif
 
 struct GemmParams {
     int mode, R, N, K, E, k;
@@ -39,6 +52,7 @@ struct GemmParams {
     const float* topk_w;
     const int32_t* row_pair;
     int* status;
+    long long* stats;           // optional per-CTA cycle counters (profiling builds only), else nullptr
 };
 
 template <int QBITS, int BT>
@@ -52,7 +66,7 @@ struct Cfg {
     static constexpr int RAW_BYTES = BW * RAW_ROW;
     static constexpr int W_BYTES = BW * 128;
     static constexpr int SC_BYTES = BW * 16;                       // 8 fp16 scales per row
-    static constexpr int EXCH_BYTES = 64 * 33 * 4;                 // up -> gate exchange (gate/up mode)
+    static constexpr int EXCH_BYTES = 32 * 128 * 4;                // epilogue staging: [32 tokens][128 rows] fp32 or 2 x bf16
     static constexpr int OFF_X = 0;
     static constexpr int OFF_W = OFF_X + SX * X_BYTES;
     static constexpr int OFF_RAW = OFF_W + SB * W_BYTES;
@@ -144,6 +158,11 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
@@ -155,14 +174,16 @@ __device__ __forceinline__ float lds_scale(uint32_t addr) {
 
 template <int QBITS, int BT>
 __global__ void __launch_bounds__(NTHREADS, 1)
-qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_xh,
+             const __grid_constant__ CUtensorMap tm_w,
              const __grid_constant__ CUtensorMap tm_s, const GemmParams p) {
     using C = Cfg<QBITS, BT>;
     extern __shared__ uint8_t smem_dyn[];
     const uint32_t sbase = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     uint8_t* sgen = smem_dyn + (sbase - smem_u32(smem_dyn));
     int* prefix = reinterpret_cast<int*>(sgen + C::OFF_PREFIX);
-    float* exch = reinterpret_cast<float*>(sgen + C::OFF_EXCH);
+    float* stg32 = reinterpret_cast<float*>(sgen + C::OFF_EXCH);
+    __nv_bfloat16* stg16 = reinterpret_cast<__nv_bfloat16*>(sgen + C::OFF_EXCH);
     volatile int* misc = reinterpret_cast<volatile int*>(sgen + C::OFF_MISC);  // [0] tmem base, [1] abort, [2..3] epilogue go/stop
     const uint32_t bar0 = sbase + C::OFF_BAR;
     auto x_full = [&](int s) { return bar0 + 8u * s; };
@@ -186,7 +207,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         fence_mbar_init();
         fence_proxy_async_smem();
     }
-    if (warp == 0 && lane == 0) { prefetch_tmap(&tm_x); prefetch_tmap(&tm_w); prefetch_tmap(&tm_s); }
+    if (warp == 0 && lane == 0) { prefetch_tmap(&tm_x); prefetch_tmap(&tm_xh); prefetch_tmap(&tm_w); prefetch_tmap(&tm_s); }
     if (warp == 3) {
         tmem_alloc(sbase + C::OFF_MISC, C::TMEM_COLS);
         tmem_relinquish();
@@ -224,22 +245,33 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
+            QG_DECL();
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 const Tile tl = decode_tile(t, prefix, p, BT);
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % C::SX;
                     const uint32_t ph = (it / C::SX) & 1u;
+                    QG_T0();
                     if (!wait_bar(x_empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    mbar_arrive_expect_tx(x_full(s), C::X_BYTES);
-                    tma_load_2d(sbase + C::OFF_X + s * C::X_BYTES, &tm_x, kb * BK, tl.tok0, x_full(s));
+                    QG_ACC(0);
+                    // short segments fetch only the first BT/2 token rows (same shared-memory layout)
+                    if (tl.tok_end - tl.tok0 <= BT / 2) {
+                        mbar_arrive_expect_tx(x_full(s), C::X_BYTES / 2);
+                        tma_load_2d(sbase + C::OFF_X + s * C::X_BYTES, &tm_xh, kb * BK, tl.tok0, x_full(s));
+                    } else {
+                        mbar_arrive_expect_tx(x_full(s), C::X_BYTES);
+                        tma_load_2d(sbase + C::OFF_X + s * C::X_BYTES, &tm_x, kb * BK, tl.tok0, x_full(s));
+                    }
                 }
             }
+            QG_FLUSH();
         }
     } else if (warp == 2) {
         // ------------------------------------------------ packed weight + scale producer
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
+            QG_DECL();
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 const Tile tl = decode_tile(t, prefix, p, BT);
                 const int row_a = tl.e * p.N + tl.wt * ((p.mode == QG_MODE_GATE_UP_SILU) ? 64 : 128);
@@ -247,7 +279,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % C::SR;
                     const uint32_t ph = (it / C::SR) & 1u;
+                    QG_T0();
                     if (!wait_bar(r_empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    QG_ACC(1);
                     const bool with_scales = (kb & 3) == 0;
                     mbar_arrive_expect_tx(r_full(s), C::RAW_BYTES + (with_scales ? C::SC_BYTES : 0));
                     const uint32_t dst = sbase + C::OFF_RAW + s * C::RAW_BYTES;
@@ -260,24 +294,31 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     }
                 }
             }
+            QG_FLUSH();
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
             uint32_t it = 0, j = 0;
             bool ok = true;
+            QG_DECL();
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
                 const Tile tl = decode_tile(t, prefix, p, BT);
                 const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
                 const uint32_t idesc = umma_idesc_bf16(BW, n_mma);
                 const uint32_t a = j & 1u, aph = (j >> 1) & 1u;
+                QG_T0();
                 if (!wait_bar(acc_empty(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                QG_ACC(2);
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + a * BT;
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int sx = it % C::SX, sb = it % C::SB;
-                    if (!wait_bar(x_full(sx), (it / C::SX) & 1u, abort_flag, p.status) ||
-                        !wait_bar(w_full(sb), (it / C::SB) & 1u, abort_flag, p.status)) { ok = false; break; }
+                    QG_T0();
+                    if (!wait_bar(x_full(sx), (it / C::SX) & 1u, abort_flag, p.status)) { ok = false; break; }
+                    QG_ACC(3);
+                    if (!wait_bar(w_full(sb), (it / C::SB) & 1u, abort_flag, p.status)) { ok = false; break; }
+                    QG_ACC(4);
                     tc_fence_after_sync();
                     const uint64_t da = umma_desc_k_sw128(sbase + C::OFF_W + sb * C::W_BYTES);
                     const uint64_t db = umma_desc_k_sw128(sbase + C::OFF_X + sx * C::X_BYTES);
@@ -289,140 +330,193 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 }
                 if (ok) umma_commit(acc_full(a));
             }
+            QG_FLUSH();
         }
     } else if (warp >= 8) {
         // ------------------------------------------------ dequantise: raw ring -> w ring
+        // Thread (row = td / 4, part = td % 4) converts the 16 weights k = 16 part .. 16 part + 15 of its row per
+        // k-block.  The packed codes and the scale of k-block i+1 are fetched into registers before k-block i is
+        // converted, so shared-memory and barrier latency overlap the arithmetic.
         const int td = threadIdx.x - 256;
+        const int row = td >> 2, part = td & 3;
+        const uint32_t raw_off = (QBITS == 8) ? td * 16 : td * 8;
+        const uint32_t sc_off = row * 16 + ((part >> 1) << 1);
+        const uint32_t w_off0 = row * 128 + (((part * 2) ^ (row & 7)) << 4);
+        const uint32_t w_off1 = row * 128 + (((part * 2 + 1) ^ (row & 7)) << 4);
         uint32_t it = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            for (int kb = 0; kb < nkb; ++kb, ++it) {
-                const int sr = it % C::SR, sb = it % C::SB;
-                ok = wait_bar(r_full(sr), (it / C::SR) & 1u, abort_flag, p.status);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) break;
-                const uint32_t raw = sbase + C::OFF_RAW + sr * C::RAW_BYTES;
-                const uint32_t sc = sbase + C::OFF_SC + ((it >> 2) % C::NSB) * C::SC_BYTES;
-                const uint32_t wst = sbase + C::OFF_W + sb * C::W_BYTES;
-                if constexpr (QBITS == 8) {
-                    uint4 v[2];
-                    float s[2];
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const int piece = j * 256 + td;
-                        v[j] = lds128(raw + piece * 16);
-                        s[j] = lds_scale(sc + (piece >> 2) * 16 + (((it & 3) * 2 + ((piece & 3) >> 1)) << 1));
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(r_empty(sr));
-                    ok = wait_bar(w_empty(sb), ((it / C::SB) & 1u) ^ 1u, abort_flag, p.status);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) break;
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const int piece = j * 256 + td;
-                        const int row = piece >> 2, part = piece & 3;
-                        const float s256 = 256.f * s[j], c = -32896.f * s[j];
-                        uint32_t o[8];
-                        dq8_word(v[j].x, s256, c, o[0], o[1]);
-                        dq8_word(v[j].y, s256, c, o[2], o[3]);
-                        dq8_word(v[j].z, s256, c, o[4], o[5]);
-                        dq8_word(v[j].w, s256, c, o[6], o[7]);
-                        const uint32_t rbase = wst + row * 128;
-                        sts128(rbase + ((((part * 2) ^ (row & 7))) << 4), o[0], o[1], o[2], o[3]);
-                        sts128(rbase + ((((part * 2 + 1) ^ (row & 7))) << 4), o[4], o[5], o[6], o[7]);
-                    }
-                } else {
-                    const int row = td >> 1, half = td & 1;
-                    const uint4 v = lds128(raw + td * 16);
-                    const float s = lds_scale(sc + row * 16 + (((it & 3) * 2 + half) << 1));
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(r_empty(sr));
-                    ok = wait_bar(w_empty(sb), ((it / C::SB) & 1u) ^ 1u, abort_flag, p.status);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) break;
-                    const uint32_t rbase = wst + row * 128;
-                    uint32_t o[4];
-                    dq4_word(v.x, s, o);
-                    sts128(rbase + (((half * 4 + 0) ^ (row & 7)) << 4), o[0], o[1], o[2], o[3]);
-                    dq4_word(v.y, s, o);
-                    sts128(rbase + (((half * 4 + 1) ^ (row & 7)) << 4), o[0], o[1], o[2], o[3]);
-                    dq4_word(v.z, s, o);
-                    sts128(rbase + (((half * 4 + 2) ^ (row & 7)) << 4), o[0], o[1], o[2], o[3]);
-                    dq4_word(v.w, s, o);
-                    sts128(rbase + (((half * 4 + 3) ^ (row & 7)) << 4), o[0], o[1], o[2], o[3]);
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(w_full(sb));
+        QG_DECL();
+        uint4 nxt = make_uint4(0, 0, 0, 0);
+        float nxt_s = 0.f;
+        auto fetch = [&](uint32_t i) -> bool {
+            const int sr = i % C::SR;
+            bool good = wait_bar(r_full(sr), (i / C::SR) & 1u, abort_flag, p.status);
+            good = __all_sync(0xFFFFFFFFu, good);
+            if (!good) return false;
+            const uint32_t raw = sbase + C::OFF_RAW + sr * C::RAW_BYTES + raw_off;
+            if constexpr (QBITS == 8) {
+                nxt = lds128(raw);
+            } else {
+                const uint2 h = lds64(raw);
+                nxt.x = h.x; nxt.y = h.y;
             }
+            nxt_s = lds_scale(sbase + C::OFF_SC + ((i >> 2) % C::NSB) * C::SC_BYTES + sc_off + ((i & 3) << 2));
+            return true;
+        };
+        const int my_tiles = (total_tiles > static_cast<int>(blockIdx.x))
+                                 ? (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x)
+                                 : 0;
+        const uint32_t total_kb = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(nkb);
+        if (total_kb > 0) {
+            QG_T0();
+            ok = fetch(0);
+            QG_ACC(5);
         }
+        for (; ok && it < total_kb; ++it) {
+            const uint4 cur = nxt;
+            const float s = nxt_s;
+            QG_T0();
+            if (it + 1 < total_kb) {
+                ok = fetch(it + 1);
+                if (!ok) break;
+            }
+            QG_ACC(5);
+            const int sr = it % C::SR, sb = it % C::SB;
+            ok = wait_bar(w_empty(sb), ((it / C::SB) & 1u) ^ 1u, abort_flag, p.status);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            QG_ACC(6);
+            const uint32_t wst = sbase + C::OFF_W + sb * C::W_BYTES;
+            uint32_t o[8];
+            if constexpr (QBITS == 8) {
+                const float s256 = 256.f * s, c = -32896.f * s;
+                dq8_word(cur.x, s256, c, o[0], o[1]);
+                dq8_word(cur.y, s256, c, o[2], o[3]);
+                dq8_word(cur.z, s256, c, o[4], o[5]);
+                dq8_word(cur.w, s256, c, o[6], o[7]);
+            } else {
+                uint32_t q[4];
+                dq4_word(cur.x, s, q);
+                o[0] = q[0]; o[1] = q[1]; o[2] = q[2]; o[3] = q[3];
+                dq4_word(cur.y, s, q);
+                o[4] = q[0]; o[5] = q[1]; o[6] = q[2]; o[7] = q[3];
+            }
+            sts128(wst + w_off0, o[0], o[1], o[2], o[3]);
+            sts128(wst + w_off1, o[4], o[5], o[6], o[7]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(w_full(sb));
+                mbar_arrive(r_empty(sr));
+            }
+            QG_ACC(7);
+        }
+        if (td == 0) QG_FLUSH();
     } else if (warp >= 4) {
         // ------------------------------------------------ epilogue (warps 4..7 <-> TMEM lanes 32 (warp-4) ..)
         const int qd = warp - 4;
         const int et = threadIdx.x - 128;
         __nv_bfloat16* outb = static_cast<__nv_bfloat16*>(p.out);
         float* outf = static_cast<float*>(p.out);
-        uint32_t j = 0;
+        uint32_t j = 0, cc = 0;
+        QG_DECL();
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++j) {
             const Tile tl = decode_tile(t, prefix, p, BT);
             const uint32_t a = j & 1u, aph = (j >> 1) & 1u;
+            QG_T0();
             if (et == 0) misc[2 + a] = wait_bar(acc_full(a), aph, abort_flag, p.status) ? 1 : 0;
             tc_fence_before_sync();
             named_bar_sync(1, 128);
             if (!misc[2 + a]) break;
             tc_fence_after_sync();
+            QG_ACC(8);
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + a * BT;
-            for (int c = 0; c < n_mma; c += 32) {
+            for (int c = 0; c < n_mma; c += 32, ++cc) {
                 uint32_t v[32];
                 tmem_ld_32x32(taddr + c, v);
                 tmem_ld_wait();
-                if (p.mode == QG_MODE_GATE_UP_SILU) {
-                    const int F = p.N / 2;
-                    if (qd >= 2) {
-#pragma unroll
-                        for (int jj = 0; jj < 32; ++jj) exch[((qd - 2) * 32 + lane) * 33 + jj] = __uint_as_float(v[jj]);
+                const int row = qd * 32 + lane;          // weight row of this thread inside the tile
+                if (p.mode == QG_MODE_DOWN_ACCUM_F32) {
+                    // y[token, n] += w * acc: lanes are consecutive n, so each warp-wide red covers 128 bytes
+                    const int n = tl.wt * BW + row;
+                    const int tokl = tl.tok0 + c + lane;
+                    int trow = 0;
+                    float wv = 0.f;
+                    if (tokl < tl.tok_end) {
+                        const int pr = p.row_pair[tokl];
+                        wv = p.topk_w[pr];
+                        trow = pr / p.k;
                     }
-                    named_bar_sync(2, 128);
-                    if (qd < 2) {
-                        const int f = tl.wt * 64 + qd * 32 + lane;
 #pragma unroll
-                        for (int jj = 0; jj < 32; ++jj) {
-                            const int tok = tl.tok0 + c + jj;
-                            const float g = __uint_as_float(v[jj]);
-                            const float u = exch[(qd * 32 + lane) * 33 + jj];
-                            const float h = g / (1.0f + expf(-g)) * u;
-                            if (tok < tl.tok_end && f < F) outb[static_cast<size_t>(tok) * F + f] = __float2bfloat16_rn(h);
-                        }
+                    for (int jj = 0; jj < 32; ++jj) {
+                        const float w = __shfl_sync(0xFFFFFFFFu, wv, jj);
+                        const int tr = __shfl_sync(0xFFFFFFFFu, trow, jj);
+                        if (tl.tok0 + c + jj < tl.tok_end && n < p.N)
+                            atomicAdd(outf + static_cast<size_t>(tr) * p.N + n, w * __uint_as_float(v[jj]));
+                    }
+                } else if (p.mode == QG_MODE_GATE_UP_SILU) {
+                    // lanes 0..63 hold gate rows, 64..127 the matching up rows: transpose through shared memory
+                    // ([32 tokens][128 rows] fp32), then every thread finishes 16 outputs of one token.
+                    const int F = p.N / 2;
+#pragma unroll
+                    for (int jj = 0; jj < 32; ++jj) stg32[jj * 128 + row] = __uint_as_float(v[jj]);
+                    named_bar_sync(2, 128);
+                    const int tk = et >> 2, f0 = (et & 3) * 16;
+                    const int tok = tl.tok0 + c + tk;
+                    const float4* g4 = reinterpret_cast<const float4*>(stg32 + tk * 128 + f0);
+                    const float4* u4 = reinterpret_cast<const float4*>(stg32 + tk * 128 + 64 + f0);
+                    uint32_t o[8];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float4 g = g4[i], u = u4[i];
+                        const float h0 = __fdividef(g.x, 1.0f + __expf(-g.x)) * u.x;
+                        const float h1 = __fdividef(g.y, 1.0f + __expf(-g.y)) * u.y;
+                        const float h2 = __fdividef(g.z, 1.0f + __expf(-g.z)) * u.z;
+                        const float h3 = __fdividef(g.w, 1.0f + __expf(-g.w)) * u.w;
+                        o[2 * i] = bf16x2(h0, h1);
+                        o[2 * i + 1] = bf16x2(h2, h3);
+                    }
+                    if (tok < tl.tok_end) {
+                        uint4* dst = reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * F + tl.wt * 64 + f0);
+                        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
                     }
                     named_bar_sync(2, 128);
                 } else {
-                    const int n = tl.wt * BW + qd * 32 + lane;
-                    if (n < p.N) {
+                    // bf16 [32 tokens][128 rows] staging (two buffers, one barrier per chunk), then 16-byte stores
+                    // that cover 256 contiguous bytes per token.
+                    float wv = 1.0f;
+                    if (p.mode == QG_MODE_DOWN_WEIGHTED) {
+                        const int tokl = tl.tok0 + c + lane;
+                        wv = (tokl < tl.tok_end) ? p.topk_w[p.row_pair[tokl]] : 0.f;
+                    }
+                    __nv_bfloat16* st = stg16 + (cc & 1u) * 4096;
 #pragma unroll
-                        for (int jj = 0; jj < 32; ++jj) {
-                            const int tok = tl.tok0 + c + jj;
-                            if (tok >= tl.tok_end) break;
-                            float val = __uint_as_float(v[jj]);
-                            if (p.mode == QG_MODE_PLAIN) {
-                                outb[static_cast<size_t>(tok) * p.N + n] = __float2bfloat16_rn(val);
-                            } else {
-                                const int pr = p.row_pair[tok];
-                                val *= p.topk_w[pr];
-                                if (p.mode == QG_MODE_DOWN_WEIGHTED)
-                                    outb[static_cast<size_t>(tok) * p.N + n] = __float2bfloat16_rn(val);
-                                else
-                                    atomicAdd(outf + static_cast<size_t>(pr / p.k) * p.N + n, val);
-                            }
-                        }
+                    for (int jj = 0; jj < 32; ++jj) {
+                        float val = __uint_as_float(v[jj]);
+                        if (p.mode == QG_MODE_DOWN_WEIGHTED) val *= __shfl_sync(0xFFFFFFFFu, wv, jj);
+                        st[jj * 128 + row] = __float2bfloat16_rn(val);
+                    }
+                    named_bar_sync(2, 128);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int piece = i * 128 + et;
+                        const int tk = piece >> 4, c16 = piece & 15;
+                        const int tok = tl.tok0 + c + tk;
+                        const int n = tl.wt * BW + c16 * 8;
+                        if (tok < tl.tok_end && n < p.N)
+                            *reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * p.N + n) =
+                                *reinterpret_cast<const uint4*>(st + tk * 128 + c16 * 8);
                     }
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty(a));
+            QG_ACC(9);
         }
+        if (et == 0) QG_FLUSH();
     }
 
     // ---------------------------------------------------- teardown
@@ -440,9 +534,12 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const vo
                        cudaStream_t st) {
     using C = Cfg<QBITS, BT>;
     static_assert(C::SMEM_BYTES <= 232448, "shared memory budget");
-    CUtensorMap tm_x, tm_w, tm_s;
+    CUtensorMap tm_x, tm_xh, tm_w, tm_s;
     const uint64_t wrows = static_cast<uint64_t>(p.E) * p.N;
     int rc = make_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, p.R, BK, BT,
+                          CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc == QG_OK)
+        rc = make_tmap_2d(ctx, &tm_xh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, p.R, BK, BT / 2,
                           CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc == QG_OK)
         rc = make_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (QBITS == 8) ? p.K : p.K / 2, wrows,
@@ -463,12 +560,20 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const vo
     // Upper bound on the number of tiles (the exact count lives on the device for grouped calls).
     const long long max_tiles = (static_cast<long long>((p.R + BT - 1) / BT) + (p.offsets ? p.E : 0)) * p.n_wt;
     const int grid = static_cast<int>(max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count);
-    kern<<<grid, NTHREADS, C::SMEM_BYTES, st>>>(tm_x, tm_w, tm_s, p);
+    kern<<<grid, NTHREADS, C::SMEM_BYTES, st>>>(tm_x, tm_xh, tm_w, tm_s, p);
     return cudaGetLastError() == cudaSuccess ? QG_OK : QG_ERR_CUDA;
 }
 
-static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p, const void* X, const void* Wq,
+#ifdef QG_PROFILE
+static long long* g_stats = nullptr;   // device buffer [grid, 12] supplied by the profiling harness
+#endif
+
+static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in, const void* X, const void* Wq,
                          const void* Ws, cudaStream_t st) {
+    GemmParams p = p_in;
+#ifdef QG_PROFILE
+    p.stats = g_stats;
+#endif
     if (qbits == QG_Q8) return bt == 256 ? launch_gemm<8, 256>(ctx, p, X, Wq, Ws, st) : launch_gemm<8, 128>(ctx, p, X, Wq, Ws, st);
     return bt == 256 ? launch_gemm<4, 256>(ctx, p, X, Wq, Ws, st) : launch_gemm<4, 128>(ctx, p, X, Wq, Ws, st);
 }
@@ -476,6 +581,10 @@ static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p, co
 }  // namespace qg
 
 extern "C" {
+
+#ifdef QG_PROFILE
+void qg_debug_set_stats(long long* dev_buf) { qg::g_stats = dev_buf; }
+#endif
 
 int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq, const void* Wscale,
                 void* Cout, void* stream) {
@@ -509,7 +618,7 @@ int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int
     p.mode = mode; p.R = R; p.N = N; p.K = K; p.E = E; p.k = (k < 1) ? 1 : k;
     p.n_wt = (mode == QG_MODE_GATE_UP_SILU) ? (N / 128) : (N + qg::BW - 1) / qg::BW;
     p.offsets = expert_offsets; p.out = Out; p.topk_w = topk_w; p.row_pair = row_pair; p.status = ctx->d_status;
-    const int bt = (R / E > 160) ? 256 : 128;
+    const int bt = (R / E > 100) ? 256 : 128;   // expected rows per expert decide the token tile
     return qg::dispatch_gemm(ctx, qbits, bt, p, Ain, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 

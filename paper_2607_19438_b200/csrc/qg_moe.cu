@@ -247,14 +247,14 @@ int moe_permute(qg_ctx* ctx, int M, int k, int H, const void* X, const int32_t* 
 int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
               int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row, const void* X,
               void* Xperm, int H, void* ws, size_t ws_bytes, void* stream) {
-    if (!ctx || !logits || !topk_idx || !topk_w || !expert_counts || !expert_offsets || !row_pair || !pair_row)
-        return QG_ERR_NULL;
+    if (!ctx || !expert_counts || !expert_offsets) return QG_ERR_NULL;
     if (M < 0 || E < 1 || E > 1024 || k < 1 || k > E) return QG_ERR_SHAPE;
+    if (M > 0 && (!logits || !topk_idx || !topk_w || !row_pair || !pair_row)) return QG_ERR_NULL;
     if (static_cast<long long>(M) * k > 0x7FFFFFFF) return QG_ERR_SHAPE;
     const bool gather = (X != nullptr) && (Xperm != nullptr);
     if (gather && (H < 8 || H % 8)) return QG_ERR_SHAPE;
     if (gather && (!qg::aligned16(X) || !qg::aligned16(Xperm))) return QG_ERR_ALIGN;
-    if (!ws || ws_bytes < qg_route_workspace_bytes(M, E, k)) return QG_ERR_WORKSPACE;
+    if (M > 0 && (!ws || ws_bytes < qg_route_workspace_bytes(M, E, k))) return QG_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t* hist = static_cast<int32_t*>(ws);
     const int nb = (M + qg::ROUTE_TOKENS_PER_BLOCK - 1) / qg::ROUTE_TOKENS_PER_BLOCK;
