@@ -18,6 +18,7 @@
 // Every mbarrier wait is bounded; when one expires the CTA records QG_ERR_TIMEOUT and leaves.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <stdlib.h>
 
 #include "qg_internal.h"
 #include "qg_ptx.cuh"
@@ -37,7 +38,9 @@ constexpr uint32_t WAIT_LIMIT = 1u << 22;
 #define QG_ACC(slot) do { if (p.stats) { long long now_ = clock64(); qg_stat_[slot] += now_ - qg_t0_; qg_t0_ = now_; } } while (0)
 #define QG_DECL() long long qg_stat_[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
 #define QG_FLUSH() do { if (p.stats) for (int i_ = 0; i_ < 12; ++i_) if (qg_stat_[i_]) atomicAdd(reinterpret_cast<unsigned long long*>(p.stats) + blockIdx.x * 12 + i_, static_cast<unsigned long long>(qg_stat_[i_])); } while (0)
+#define QG_TRACE(ev, i) do { if (p.stats && blockIdx.x == 0 && (i) < 256) p.stats[148 * 12 + (ev) * 256 + (i)] = clock64(); } while (0)
 #else
+#define QG_TRACE(ev, i) do {} while (0)
 #define QG_T0() do {} while (0)
 #define QG_ACC(slot) do {} while (0)
 #define QG_DECL() do {} while (0)
@@ -53,23 +56,22 @@ struct GemmParams {
     const int32_t* row_pair;
     int* status;
     long long* stats;           // optional per-CTA cycle counters (profiling builds only), else nullptr
+    int dbg;                    // profiling builds only: bit 0 skip TMEM stores, bit 1 skip epilogue body
 };
 
 template <int QBITS, int BT>
 struct Cfg {
-    static constexpr int SX = (BT == 256) ? 4 : 5;                 // activation stages
-    static constexpr int SR = (QBITS == 8) ? ((BT == 256) ? 4 : 8) : 8;  // packed-weight stages
-    static constexpr int SB = (BT == 256) ? 2 : 3;                 // dequantised-weight stages
+    static constexpr int SX = (BT > 128) ? 5 : 6;                  // activation stages (shared memory)
+    static constexpr int SR = (QBITS == 8) ? 6 : 8;                // packed-weight stages (shared memory)
+    static constexpr int SB = 4;                                   // dequantised-weight stages (tensor memory)
     static constexpr int NSB = (SR + 3) / 4 + 1;                   // scale buffers (one per 4 k-blocks)
     static constexpr int X_BYTES = BT * 128;
     static constexpr int RAW_ROW = (QBITS == 8) ? 64 : 32;         // packed bytes per row per stage
     static constexpr int RAW_BYTES = BW * RAW_ROW;
-    static constexpr int W_BYTES = BW * 128;
     static constexpr int SC_BYTES = BW * 16;                       // 8 fp16 scales per row
     static constexpr int EXCH_BYTES = 32 * 128 * 4;                // epilogue staging: [32 tokens][128 rows] fp32 or 2 x bf16
     static constexpr int OFF_X = 0;
-    static constexpr int OFF_W = OFF_X + SX * X_BYTES;
-    static constexpr int OFF_RAW = OFF_W + SB * W_BYTES;
+    static constexpr int OFF_RAW = OFF_X + SX * X_BYTES;
     static constexpr int OFF_SC = OFF_RAW + SR * RAW_BYTES;
     static constexpr int OFF_EXCH = OFF_SC + NSB * SC_BYTES;
     static constexpr int OFF_PREFIX = OFF_EXCH + EXCH_BYTES;
@@ -77,7 +79,10 @@ struct Cfg {
     static constexpr int NBAR = 2 * SX + 2 * SR + 2 * SB + 4;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;        // + slack for 1024-byte alignment
-    static constexpr int TMEM_COLS = 2 * BT;
+    static constexpr int TMEM_COLS = 512;                          // two accumulators + SB weight stages
+    static constexpr int A_COL0 = 2 * BT;                          // first column of the weight stages
+    static constexpr int A_COLS = 32;                              // 64 bf16 per lane = 32 columns per stage
+    static_assert(2 * BT + SB * 32 <= 512, "tensor memory budget");
 };
 
 struct Tile {
@@ -254,6 +259,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     QG_T0();
                     if (!wait_bar(x_empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     QG_ACC(0);
+                    QG_TRACE(0, it);
                     // short segments fetch only the first BT/2 token rows (same shared-memory layout)
                     if (tl.tok_end - tl.tok0 <= BT / 2) {
                         mbar_arrive_expect_tx(x_full(s), C::X_BYTES / 2);
@@ -282,6 +288,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     QG_T0();
                     if (!wait_bar(r_empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     QG_ACC(1);
+                    QG_TRACE(1, it);
                     const bool with_scales = (kb & 3) == 0;
                     mbar_arrive_expect_tx(r_full(s), C::RAW_BYTES + (with_scales ? C::SC_BYTES : 0));
                     const uint32_t dst = sbase + C::OFF_RAW + s * C::RAW_BYTES;
@@ -317,16 +324,25 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     QG_T0();
                     if (!wait_bar(x_full(sx), (it / C::SX) & 1u, abort_flag, p.status)) { ok = false; break; }
                     QG_ACC(3);
+                    QG_TRACE(2, it);
                     if (!wait_bar(w_full(sb), (it / C::SB) & 1u, abort_flag, p.status)) { ok = false; break; }
                     QG_ACC(4);
+                    QG_TRACE(3, it);
                     tc_fence_after_sync();
-                    const uint64_t da = umma_desc_k_sw128(sbase + C::OFF_W + sb * C::W_BYTES);
+                    const uint32_t ta = tmem_base + C::A_COL0 + sb * C::A_COLS;
                     const uint64_t db = umma_desc_k_sw128(sbase + C::OFF_X + sx * C::X_BYTES);
+#ifdef QG_PROFILE
+                    const int nk4 = (p.dbg & 4) ? 1 : 4;
+#else
+                    const int nk4 = 4;
+#endif
 #pragma unroll
                     for (int k4 = 0; k4 < 4; ++k4)
-                        umma_f16_ss(d_tmem, da + 2u * k4, db + 2u * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
+                        if (k4 < nk4) umma_f16_ts(d_tmem, ta + 8u * k4, db + 2u * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
                     umma_commit(x_empty(sx));
                     umma_commit(w_empty(sb));
+                    QG_ACC(10);
+                    QG_TRACE(4, it);
                 }
                 if (ok) umma_commit(acc_full(a));
             }
@@ -334,15 +350,15 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         }
     } else if (warp >= 8) {
         // ------------------------------------------------ dequantise: raw ring -> w ring
-        // Thread (row = td / 4, part = td % 4) converts the 16 weights k = 16 part .. 16 part + 15 of its row per
-        // k-block.  The packed codes and the scale of k-block i+1 are fetched into registers before k-block i is
+        // Thread (row, part) converts the 16 weights k = 16 part .. 16 part + 15 of its weight row per k-block and
+        // writes them as 8 columns of its TMEM lane (the MMA reads its A operand from tensor memory).  The packed codes and the scale of k-block i+1 are fetched into registers before k-block i is
         // converted, so shared-memory and barrier latency overlap the arithmetic.
         const int td = threadIdx.x - 256;
-        const int row = td >> 2, part = td & 3;
-        const uint32_t raw_off = (QBITS == 8) ? td * 16 : td * 8;
+        const int row = (warp & 3) * 32 + lane;      // a warp may only touch the TMEM lanes of its quarter
+        const int part = (warp - 8) >> 2;
+        const uint32_t raw_off = (QBITS == 8) ? (row * 64 + part * 16) : (row * 32 + part * 8);
         const uint32_t sc_off = row * 16 + ((part >> 1) << 1);
-        const uint32_t w_off0 = row * 128 + (((part * 2) ^ (row & 7)) << 4);
-        const uint32_t w_off1 = row * 128 + (((part * 2 + 1) ^ (row & 7)) << 4);
+        const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + C::A_COL0 + part * 8;
         uint32_t it = 0;
         bool ok = true;
         QG_DECL();
@@ -381,12 +397,14 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 if (!ok) break;
             }
             QG_ACC(5);
+            if (td == 0) { QG_TRACE(5, it); }
             const int sr = it % C::SR, sb = it % C::SB;
             ok = wait_bar(w_empty(sb), ((it / C::SB) & 1u) ^ 1u, abort_flag, p.status);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             QG_ACC(6);
-            const uint32_t wst = sbase + C::OFF_W + sb * C::W_BYTES;
+            if (td == 0) { QG_TRACE(6, it); }
+            tc_fence_after_sync();
             uint32_t o[8];
             if constexpr (QBITS == 8) {
                 const float s256 = 256.f * s, c = -32896.f * s;
@@ -401,15 +419,21 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 dq4_word(cur.y, s, q);
                 o[4] = q[0]; o[5] = q[1]; o[6] = q[2]; o[7] = q[3];
             }
-            sts128(wst + w_off0, o[0], o[1], o[2], o[3]);
-            sts128(wst + w_off1, o[4], o[5], o[6], o[7]);
-            fence_proxy_async_smem();
+#ifdef QG_PROFILE
+            if (!(p.dbg & 1) || it < 4)
+#endif
+            {
+                tmem_st_32x32_x8(a_taddr + sb * C::A_COLS, o);
+                tmem_st_wait();
+            }
+            tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(w_full(sb));
                 mbar_arrive(r_empty(sr));
             }
             QG_ACC(7);
+            if (td == 0) { QG_TRACE(7, it); }
         }
         if (td == 0) QG_FLUSH();
     } else if (warp >= 4) {
@@ -432,7 +456,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             QG_ACC(8);
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + a * BT;
-            for (int c = 0; c < n_mma; c += 32, ++cc) {
+#ifdef QG_PROFILE
+            const int n_epi = (p.dbg & 2) ? 0 : n_mma;
+#else
+            const int n_epi = n_mma;
+#endif
+            for (int c = 0; c < n_epi; c += 32, ++cc) {
                 uint32_t v[32];
                 tmem_ld_32x32(taddr + c, v);
                 tmem_ld_wait();
@@ -571,11 +600,16 @@ static long long* g_stats = nullptr;   // device buffer [grid, 12] supplied by t
 static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in, const void* X, const void* Wq,
                          const void* Ws, cudaStream_t st) {
     GemmParams p = p_in;
+    if (const char* f = getenv("QG_FORCE_BT")) {   // tile-shape override for sweeps
+        const int v = atoi(f);
+        if (v == 128 || v == 192) bt = v;
+    }
 #ifdef QG_PROFILE
     p.stats = g_stats;
+    if (const char* d = getenv("QG_DBG")) p.dbg = atoi(d);
 #endif
-    if (qbits == QG_Q8) return bt == 256 ? launch_gemm<8, 256>(ctx, p, X, Wq, Ws, st) : launch_gemm<8, 128>(ctx, p, X, Wq, Ws, st);
-    return bt == 256 ? launch_gemm<4, 256>(ctx, p, X, Wq, Ws, st) : launch_gemm<4, 128>(ctx, p, X, Wq, Ws, st);
+    if (qbits == QG_Q8) return bt == 192 ? launch_gemm<8, 192>(ctx, p, X, Wq, Ws, st) : launch_gemm<8, 128>(ctx, p, X, Wq, Ws, st);
+    return bt == 192 ? launch_gemm<4, 192>(ctx, p, X, Wq, Ws, st) : launch_gemm<4, 128>(ctx, p, X, Wq, Ws, st);
 }
 
 }  // namespace qg
@@ -597,7 +631,7 @@ int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, cons
     p.mode = QG_MODE_PLAIN; p.R = M; p.N = N; p.K = K; p.E = 1; p.k = 1;
     p.n_wt = (N + qg::BW - 1) / qg::BW;
     p.offsets = nullptr; p.out = Cout; p.topk_w = nullptr; p.row_pair = nullptr; p.status = ctx->d_status;
-    const int bt = (M > 128) ? 256 : 128;
+    const int bt = (M > 128) ? 192 : 128;
     return qg::dispatch_gemm(ctx, qbits, bt, p, A, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 
@@ -618,7 +652,7 @@ int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int
     p.mode = mode; p.R = R; p.N = N; p.K = K; p.E = E; p.k = (k < 1) ? 1 : k;
     p.n_wt = (mode == QG_MODE_GATE_UP_SILU) ? (N / 128) : (N + qg::BW - 1) / qg::BW;
     p.offsets = expert_offsets; p.out = Out; p.topk_w = topk_w; p.row_pair = row_pair; p.status = ctx->d_status;
-    const int bt = (R / E > 100) ? 256 : 128;   // expected rows per expert decide the token tile
+    const int bt = (R / E > 100) ? 192 : 128;   // expected rows per expert decide the token tile
     return qg::dispatch_gemm(ctx, qbits, bt, p, Ain, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 
