@@ -3,18 +3,23 @@
 // Operation (paper Sec. 3.1: dense GEMM in 4-/8-bit quantisation, MoE expert GEMM, fused gate/up+SiLU):
 //   Out[t, n] = sum_k X[t, k] * q[n, k] * scale[n, k/32], per expert segment in the grouped case.
 //
-// Mapping onto the tensor cores.  The weight rows are the UMMA "M" side (128 rows per tile, TMEM
-// lanes) and the tokens the "N" side (up to BT = 128 or 256 per tile, TMEM columns): a weight is
-// dequantised once per tile and used by up to 256 tokens, and short expert segments only shrink N.
+// Mapping onto the tensor cores.  The weight rows are the UMMA "M" side and the tokens the "N" side.  Two CTAs
+// on neighbouring SMs form a pair (cluster of 2, tcgen05 cta_group::2): the pair's tile is 256 weight rows x BT
+// tokens (BT = 128 or 192).  Each CTA dequantises its own 128 weight rows straight into tensor memory, where the
+// MMA reads them as its A operand, and stages half of the token tile in shared memory as its half of the B
+// operand, so per SM only half of the activation bytes cross L2 -> SM and shared memory.
 //
-// Persistent CTA of 24 warps, one tile at a time, two TMEM accumulators (epilogue of tile j overlaps
-// the main loop of tile j+1):
-//   warp 0      TMA producer of activation tiles  X[BT, 64] (128-byte swizzle)      -> x ring
-//   warp 2      TMA producer of packed weights [128, 64] (+ scales every 4 k-blocks) -> raw ring
-//   warps 8-23  dequantise raw -> bf16 [128, 64] written in the swizzled K-major layout -> w ring
-//   warp 1      one thread issues tcgen05.mma (A = w ring, B = x ring, D in TMEM) and commits
-//   warps 4-7   epilogue: tcgen05.ld, fused activation / routing weight, bf16 stores
-//   warp 3      allocates and frees TMEM
+// Persistent CTA of 24 warps, one tile at a time, two TMEM accumulators (epilogue of tile j overlaps the main
+// loop of tile j+1):
+//   warp 0      TMA producer of this CTA's half activation tile X[BT/2, 64] (128-byte swizzle)    -> x ring
+//   warp 2      TMA producer of packed weights [128, 64] (+ scales every 4 k-blocks)              -> raw ring
+//   warps 8-23  dequantise raw -> bf16, written with tcgen05.st into TMEM weight stages (4 groups x 4 warps,
+//               group g converts every 4th k-block)
+//   warps 1, 3  (even CTA only) issue tcgen05.mma.cta_group::2 for the even / odd k-blocks and commit to both CTAs
+//   warps 4-7   epilogue: tcgen05.ld, fused activation / routing weight, staged 16-byte bf16 stores
+//   warp 3      also allocates and frees TMEM
+// Barriers the MMA waits on live in the even CTA and also collect the odd CTA's arrivals (remote mbarrier
+// arrive, TMA completion bytes); barriers that free a stage are signalled in both CTAs by the commit.
 // Every mbarrier wait is bounded; when one expires the CTA records QG_ERR_TIMEOUT and leaves.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -25,12 +30,11 @@
 
 namespace qg {
 
-constexpr int BW = 128;        // weight rows per tile (UMMA M)
+constexpr int BW = 128;        // weight rows per CTA tile (one UMMA M half)
 constexpr int BK = 64;         // k per pipeline stage (one 128-byte swizzle row of bf16)
-constexpr int NDW = 16;        // dequantising warps
 constexpr int NTHREADS = 768;
 constexpr int MAX_E = 1024;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint32_t WAIT_LIMIT = 1u << 18;   // polls; an unsatisfied try_wait poll lasts about 4 us, so about a second
 
 // Profiling builds (-DQG_PROFILE) accumulate, per CTA, the cycles each role spends in each wait.
 #ifdef QG_PROFILE
@@ -49,44 +53,49 @@ constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 struct GemmParams {
     int mode, R, N, K, E, k;
-    int n_wt;                   // weight tiles per expert
+    int n_wt;                   // 128-row weight tiles per expert (64 gate + 64 up rows each in gate/up mode)
     const int32_t* offsets;     // device expert offsets [E+1]; nullptr: one segment [0, R)
     void* out;
     const float* topk_w;
     const int32_t* row_pair;
     int* status;
     long long* stats;           // optional per-CTA cycle counters (profiling builds only), else nullptr
-    int dbg;                    // profiling builds only: bit 0 skip TMEM stores, bit 1 skip epilogue body
+    int dbg;                    // profiling builds only
 };
 
 template <int QBITS, int BT>
 struct Cfg {
-    static constexpr int SX = (BT > 128) ? 5 : 6;                  // activation stages (shared memory)
-    static constexpr int SR = (QBITS == 8) ? 6 : 8;                // packed-weight stages (shared memory)
-    static constexpr int SB = 4;                                   // dequantised-weight stages (tensor memory)
-    static constexpr int NSB = (SR + 3) / 4 + 1;                   // scale buffers (one per 4 k-blocks)
-    static constexpr int X_BYTES = BT * 128;
+    static constexpr int SX = 8;                                   // k-block stages: one ring index for the activation tile
+                                                                   // (smem), the packed weights (smem), the dequantised
+                                                                   // weights (TMEM) and the full/done barriers
+    static constexpr int SR = SX;
+    static constexpr int NACC = (BT > 128) ? 1 : 2;                // accumulators in tensor memory
+    static constexpr int NSB = 3;                                  // scale buffers (one per 4 k-blocks)
+    static constexpr int XH_ROWS = BT / 2;                         // token rows this CTA stages per k-block
+    static constexpr int X_BYTES = XH_ROWS * 128;
     static constexpr int RAW_ROW = (QBITS == 8) ? 64 : 32;         // packed bytes per row per stage
     static constexpr int RAW_BYTES = BW * RAW_ROW;
     static constexpr int SC_BYTES = BW * 16;                       // 8 fp16 scales per row
-    static constexpr int EXCH_BYTES = 32 * 128 * 4;                // epilogue staging: [32 tokens][128 rows] fp32 or 2 x bf16
+    static constexpr int STG_BYTES = 32 * 128 * 4;                 // epilogue staging: [32 tokens][128 rows] fp32 or 2 x bf16
     static constexpr int OFF_X = 0;
     static constexpr int OFF_RAW = OFF_X + SX * X_BYTES;
     static constexpr int OFF_SC = OFF_RAW + SR * RAW_BYTES;
-    static constexpr int OFF_EXCH = OFF_SC + NSB * SC_BYTES;
-    static constexpr int OFF_PREFIX = OFF_EXCH + EXCH_BYTES;
+    static constexpr int OFF_STG = OFF_SC + NSB * SC_BYTES;
+    static constexpr int OFF_PREFIX = OFF_STG + STG_BYTES;
     static constexpr int OFF_BAR = OFF_PREFIX + (MAX_E + 4) * 4;
-    static constexpr int NBAR = 2 * SX + 2 * SR + 2 * SB + 4;
+    static constexpr int NBAR = 2 * SX + 2 * SR + 4;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;        // + slack for 1024-byte alignment
-    static constexpr int TMEM_COLS = 512;                          // two accumulators + SB weight stages
-    static constexpr int A_COL0 = 2 * BT;                          // first column of the weight stages
+    static constexpr int TMEM_COLS = 512;                          // accumulator(s) + SX weight stages
+    static constexpr int A_COL0 = NACC * BT;                       // first column of the weight stages
     static constexpr int A_COLS = 32;                              // 64 bf16 per lane = 32 columns per stage
-    static_assert(2 * BT + SB * 32 <= 512, "tensor memory budget");
+    static_assert(NACC * BT + SX * 32 <= 512, "tensor memory budget");
+    static_assert(X_BYTES % 1024 == 0, "swizzled stages must stay 1024-byte aligned");
+    static_assert(SX == 8, "stage arithmetic below assumes a ring of eight");
 };
 
 struct Tile {
-    int e, wt, tok0, tok_end;
+    int e, pw, tok0, tok_end;   // expert, pair weight tile (weight tiles 2 pw and 2 pw + 1), token range
 };
 
 __device__ __forceinline__ Tile decode_tile(int t, const int* prefix, const GemmParams& p, int BT) {
@@ -101,16 +110,17 @@ __device__ __forceinline__ Tile decode_tile(int t, const int* prefix, const Gemm
     const int local = t - prefix[lo];
     Tile r;
     r.e = lo;
-    r.wt = local / n_tt;
+    r.pw = local / n_tt;
     r.tok0 = seg0 + (local % n_tt) * BT;
     r.tok_end = min(seg1, r.tok0 + BT);
     return r;
 }
 
 // Bounded wait on an mbarrier phase.  Returns false if the CTA is giving up.
+template <bool CLUSTER>
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1;
@@ -168,9 +178,6 @@ __device__ __forceinline__ uint2 lds64(uint32_t addr) {
     asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
 __device__ __forceinline__ float lds_scale(uint32_t addr) {
     unsigned short h;
     asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
@@ -178,53 +185,56 @@ __device__ __forceinline__ float lds_scale(uint32_t addr) {
 }
 
 template <int QBITS, int BT>
-__global__ void __launch_bounds__(NTHREADS, 1)
-qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_xh,
-             const __grid_constant__ CUtensorMap tm_w,
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
+qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const __grid_constant__ CUtensorMap tm_s, const GemmParams p) {
     using C = Cfg<QBITS, BT>;
     extern __shared__ uint8_t smem_dyn[];
     const uint32_t sbase = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     uint8_t* sgen = smem_dyn + (sbase - smem_u32(smem_dyn));
     int* prefix = reinterpret_cast<int*>(sgen + C::OFF_PREFIX);
-    float* stg32 = reinterpret_cast<float*>(sgen + C::OFF_EXCH);
-    __nv_bfloat16* stg16 = reinterpret_cast<__nv_bfloat16*>(sgen + C::OFF_EXCH);
+    float* stg32 = reinterpret_cast<float*>(sgen + C::OFF_STG);
+    __nv_bfloat16* stg16 = reinterpret_cast<__nv_bfloat16*>(sgen + C::OFF_STG);
     volatile int* misc = reinterpret_cast<volatile int*>(sgen + C::OFF_MISC);  // [0] tmem base, [1] abort, [2..3] epilogue go/stop
     const uint32_t bar0 = sbase + C::OFF_BAR;
-    auto x_full = [&](int s) { return bar0 + 8u * s; };
-    auto x_empty = [&](int s) { return bar0 + 8u * (C::SX + s); };
+    // full[s]   (even CTA): k-block in stage s is ready: both halves of the activation tile have landed (TMA bytes)
+    //           and all eight dequantising warps of the pair (4 per CTA) have written its weights to TMEM.
+    // done[s]   (both CTAs, by commit): the MMAs of the k-block in stage s have completed.
+    // r_full / r_empty: this CTA's packed-weight ring.   acc_full (both CTAs) / acc_empty (even CTA): accumulators.
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto done = [&](int s) { return bar0 + 8u * (C::SX + s); };
     auto r_full = [&](int s) { return bar0 + 8u * (2 * C::SX + s); };
     auto r_empty = [&](int s) { return bar0 + 8u * (2 * C::SX + C::SR + s); };
-    auto w_full = [&](int s) { return bar0 + 8u * (2 * C::SX + 2 * C::SR + s); };
-    auto w_empty = [&](int s) { return bar0 + 8u * (2 * C::SX + 2 * C::SR + C::SB + s); };
-    auto acc_full = [&](int s) { return bar0 + 8u * (2 * C::SX + 2 * C::SR + 2 * C::SB + s); };
-    auto acc_empty = [&](int s) { return bar0 + 8u * (2 * C::SX + 2 * C::SR + 2 * C::SB + 2 + s); };
+    auto acc_full = [&](int s) { return bar0 + 8u * (2 * C::SX + 2 * C::SR + s); };
+    auto acc_empty = [&](int s) { return bar0 + 8u * (2 * C::SX + 2 * C::SR + 2 + s); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();          // 0: issues the MMAs, 1: its peer
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     volatile int* abort_flag = misc + 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::SX; ++s) { mbar_init(x_full(s), 1); mbar_init(x_empty(s), 1); }
-        for (int s = 0; s < C::SR; ++s) { mbar_init(r_full(s), 1); mbar_init(r_empty(s), NDW); }
-        for (int s = 0; s < C::SB; ++s) { mbar_init(w_full(s), NDW); mbar_init(w_empty(s), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 4); }
+        for (int s = 0; s < C::SX; ++s) { mbar_init(full(s), 1 + 8); mbar_init(done(s), 1); }
+        for (int s = 0; s < C::SR; ++s) { mbar_init(r_full(s), 1); mbar_init(r_empty(s), 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 2); mbar_init(acc_empty(s), 8); }
         misc[1] = 0;
         fence_mbar_init();
         fence_proxy_async_smem();
     }
-    if (warp == 0 && lane == 0) { prefetch_tmap(&tm_x); prefetch_tmap(&tm_xh); prefetch_tmap(&tm_w); prefetch_tmap(&tm_s); }
+    if (warp == 0 && lane == 0) { prefetch_tmap(&tm_x); prefetch_tmap(&tm_w); prefetch_tmap(&tm_s); }
     if (warp == 3) {
-        tmem_alloc(sbase + C::OFF_MISC, C::TMEM_COLS);
-        tmem_relinquish();
+        tmem_alloc_pair(sbase + C::OFF_MISC, C::TMEM_COLS);
+        tmem_relinquish_pair();
     }
-    if (warp == 2) {  // prefix[e] = tiles before expert e; prefix[E] = total
+    const int n_pw = (p.n_wt + 1) >> 1;
+    if (warp == 2) {  // prefix[e] = pair tiles before expert e; prefix[E] = total
         int carry = 0;
         for (int e0 = 0; e0 < p.E; e0 += 32) {
             const int e = e0 + lane;
             int n = 0;
             if (e < p.E) {
                 const int cnt = p.offsets ? (p.offsets[e + 1] - p.offsets[e]) : p.R;
-                n = ((cnt + BT - 1) / BT) * p.n_wt;
+                n = ((cnt + BT - 1) / BT) * n_pw;
             }
             int inc = n;
 #pragma unroll
@@ -239,228 +249,245 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     }
     tc_fence_before_sync();
     __syncthreads();
+    cluster_sync_all();          // both CTAs' barriers are initialised and both halves of TMEM are allocated
     tc_fence_after_sync();
     const uint32_t tmem_base = static_cast<uint32_t>(misc[0]);
     const int total_tiles = prefix[p.E];
-    const int nkb = p.K / BK;
-    const int rows_half = (p.mode == QG_MODE_GATE_UP_SILU) ? (p.N / 2) : 64;  // row distance of the 2nd 64-row box
+    const int nkb = p.K / BK;     // a multiple of 4
+    const bool gate_up = (p.mode == QG_MODE_GATE_UP_SILU);
 
+    // Control warps walk their loops with all 32 lanes (converged) and keep the per-k-block instruction count small:
+    // a lone thread retires only one dependent instruction every few cycles and an mbarrier round trip costs a few
+    // hundred cycles, so the producers work in batches of four k-blocks and the MMA warp does one wait, one
+    // four-MMA statement and one commit per k-block.
     if (warp == 0) {
-        // ------------------------------------------------ activation producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            QG_DECL();
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const Tile tl = decode_tile(t, prefix, p, BT);
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % C::SX;
-                    const uint32_t ph = (it / C::SX) & 1u;
-                    QG_T0();
-                    if (!wait_bar(x_empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    QG_ACC(0);
-                    QG_TRACE(0, it);
-                    // short segments fetch only the first BT/2 token rows (same shared-memory layout)
-                    if (tl.tok_end - tl.tok0 <= BT / 2) {
-                        mbar_arrive_expect_tx(x_full(s), C::X_BYTES / 2);
-                        tma_load_2d(sbase + C::OFF_X + s * C::X_BYTES, &tm_xh, kb * BK, tl.tok0, x_full(s));
-                    } else {
-                        mbar_arrive_expect_tx(x_full(s), C::X_BYTES);
-                        tma_load_2d(sbase + C::OFF_X + s * C::X_BYTES, &tm_x, kb * BK, tl.tok0, x_full(s));
-                    }
-                }
-            }
-            QG_FLUSH();
-        }
-    } else if (warp == 2) {
-        // ------------------------------------------------ packed weight + scale producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            QG_DECL();
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const Tile tl = decode_tile(t, prefix, p, BT);
-                const int row_a = tl.e * p.N + tl.wt * ((p.mode == QG_MODE_GATE_UP_SILU) ? 64 : 128);
-                const int row_b = row_a + rows_half;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % C::SR;
-                    const uint32_t ph = (it / C::SR) & 1u;
-                    QG_T0();
-                    if (!wait_bar(r_empty(s), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    QG_ACC(1);
-                    QG_TRACE(1, it);
-                    const bool with_scales = (kb & 3) == 0;
-                    mbar_arrive_expect_tx(r_full(s), C::RAW_BYTES + (with_scales ? C::SC_BYTES : 0));
-                    const uint32_t dst = sbase + C::OFF_RAW + s * C::RAW_BYTES;
-                    tma_load_2d(dst, &tm_w, kb * C::RAW_ROW, row_a, r_full(s));
-                    tma_load_2d(dst + C::RAW_BYTES / 2, &tm_w, kb * C::RAW_ROW, row_b, r_full(s));
-                    if (with_scales) {
-                        const uint32_t sd = sbase + C::OFF_SC + ((it >> 2) % C::NSB) * C::SC_BYTES;
-                        tma_load_2d(sd, &tm_s, (kb >> 2) * 8, row_a, r_full(s));
-                        tma_load_2d(sd + C::SC_BYTES / 2, &tm_s, (kb >> 2) * 8, row_b, r_full(s));
-                    }
-                }
-            }
-            QG_FLUSH();
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            uint32_t it = 0, j = 0;
-            bool ok = true;
-            QG_DECL();
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++j) {
-                const Tile tl = decode_tile(t, prefix, p, BT);
-                const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
-                const uint32_t idesc = umma_idesc_bf16(BW, n_mma);
-                const uint32_t a = j & 1u, aph = (j >> 1) & 1u;
-                QG_T0();
-                if (!wait_bar(acc_empty(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                QG_ACC(2);
-                tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + a * BT;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int sx = it % C::SX, sb = it % C::SB;
-                    QG_T0();
-                    if (!wait_bar(x_full(sx), (it / C::SX) & 1u, abort_flag, p.status)) { ok = false; break; }
-                    QG_ACC(3);
-                    QG_TRACE(2, it);
-                    if (!wait_bar(w_full(sb), (it / C::SB) & 1u, abort_flag, p.status)) { ok = false; break; }
-                    QG_ACC(4);
-                    QG_TRACE(3, it);
-                    tc_fence_after_sync();
-                    const uint32_t ta = tmem_base + C::A_COL0 + sb * C::A_COLS;
-                    const uint64_t db = umma_desc_k_sw128(sbase + C::OFF_X + sx * C::X_BYTES);
-#ifdef QG_PROFILE
-                    const int nk4 = (p.dbg & 4) ? 1 : 4;
-#else
-                    const int nk4 = 4;
-#endif
-#pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4)
-                        if (k4 < nk4) umma_f16_ts(d_tmem, ta + 8u * k4, db + 2u * k4, idesc, (kb | k4) != 0 ? 1u : 0u);
-                    umma_commit(x_empty(sx));
-                    umma_commit(w_empty(sb));
-                    QG_ACC(10);
-                    QG_TRACE(4, it);
-                }
-                if (ok) umma_commit(acc_full(a));
-            }
-            QG_FLUSH();
-        }
-    } else if (warp >= 8) {
-        // ------------------------------------------------ dequantise: raw ring -> w ring
-        // Thread (row, part) converts the 16 weights k = 16 part .. 16 part + 15 of its weight row per k-block and
-        // writes them as 8 columns of its TMEM lane (the MMA reads its A operand from tensor memory).  The packed codes and the scale of k-block i+1 are fetched into registers before k-block i is
-        // converted, so shared-memory and barrier latency overlap the arithmetic.
-        const int td = threadIdx.x - 256;
-        const int row = (warp & 3) * 32 + lane;      // a warp may only touch the TMEM lanes of its quarter
-        const int part = (warp - 8) >> 2;
-        const uint32_t raw_off = (QBITS == 8) ? (row * 64 + part * 16) : (row * 32 + part * 8);
-        const uint32_t sc_off = row * 16 + ((part >> 1) << 1);
-        const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + C::A_COL0 + part * 8;
-        uint32_t it = 0;
+        // ------------------------------------------------ activation producer (this CTA's half of the token tile)
+        uint32_t s = 0, ph = 0;      // first stage of the next batch (0 or 4) and the parity of its next "done" phase
+        const uint32_t full_leader = map_to_cta(full(0), 0);
         bool ok = true;
         QG_DECL();
-        uint4 nxt = make_uint4(0, 0, 0, 0);
-        float nxt_s = 0.f;
-        auto fetch = [&](uint32_t i) -> bool {
-            const int sr = i % C::SR;
-            bool good = wait_bar(r_full(sr), (i / C::SR) & 1u, abort_flag, p.status);
-            good = __all_sync(0xFFFFFFFFu, good);
-            if (!good) return false;
-            const uint32_t raw = sbase + C::OFF_RAW + sr * C::RAW_BYTES + raw_off;
-            if constexpr (QBITS == 8) {
-                nxt = lds128(raw);
-            } else {
-                const uint2 h = lds64(raw);
-                nxt.x = h.x; nxt.y = h.y;
+        for (int t = pair; t < total_tiles && ok; t += n_pairs) {
+            const Tile tl = decode_tile(t, prefix, p, BT);
+            const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
+            const int row0 = tl.tok0 + static_cast<int>(rank) * (n_mma >> 1);   // B rows split at N / 2
+            for (int kb = 0; kb < nkb; kb += 4) {
+                QG_T0();
+                // stages s..s+3 are free once the MMAs that read them eight k-blocks ago are done; the even and the odd
+                // stages belong to different MMA warps, each of which completes its k-blocks in order
+                if (!wait_bar<false>(done(s + 2), ph ^ 1u, abort_flag, p.status) ||
+                    !wait_bar<false>(done(s + 3), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                QG_ACC(0);
+                if (lane == 0) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (rank == 0) mbar_arrive_expect_tx(full(s + j), 2 * C::X_BYTES);
+                        tma_load_2d_pair(sbase + C::OFF_X + (s + j) * C::X_BYTES, &tm_x, (kb + j) * BK, row0,
+                                         full_leader + 8u * (s + j));
+                    }
+                }
+                __syncwarp();
+                s ^= 4u;
+                if (s == 0) ph ^= 1u;
             }
-            nxt_s = lds_scale(sbase + C::OFF_SC + ((i >> 2) % C::NSB) * C::SC_BYTES + sc_off + ((i & 3) << 2));
-            return true;
-        };
-        const int my_tiles = (total_tiles > static_cast<int>(blockIdx.x))
-                                 ? (total_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x)
-                                 : 0;
-        const uint32_t total_kb = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(nkb);
-        if (total_kb > 0) {
-            QG_T0();
-            ok = fetch(0);
-            QG_ACC(5);
         }
-        for (; ok && it < total_kb; ++it) {
-            const uint4 cur = nxt;
-            const float s = nxt_s;
-            QG_T0();
-            if (it + 1 < total_kb) {
-                ok = fetch(it + 1);
+        __syncwarp();
+        if (lane == 0) QG_FLUSH();
+    } else if (warp == 2) {
+        // ------------------------------------------------ packed weight + scale producer (local ring)
+        uint32_t s = 0, ph = 0, sg = 0;     // first raw stage of the batch (0 or 4), parity, scale buffer
+        bool ok = true;
+        QG_DECL();
+        for (int t = pair; t < total_tiles && ok; t += n_pairs) {
+            const Tile tl = decode_tile(t, prefix, p, BT);
+            const int wt = 2 * tl.pw + static_cast<int>(rank);
+            const int row_a = tl.e * p.N + wt * (gate_up ? 64 : 128);
+            const int row_b = row_a + (gate_up ? (p.N / 2) : 64);
+            for (int kb = 0; kb < nkb; kb += 4) {
+                QG_T0();
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (ok && !wait_bar<false>(r_empty(s + j), ph ^ 1u, abort_flag, p.status)) ok = false;
                 if (!ok) break;
+                QG_ACC(1);
+                if (lane == 0) {
+                    const uint32_t sd = sbase + C::OFF_SC + sg * C::SC_BYTES;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        mbar_arrive_expect_tx(r_full(s + j), C::RAW_BYTES + (j == 0 ? C::SC_BYTES : 0));
+                        const uint32_t dst = sbase + C::OFF_RAW + (s + j) * C::RAW_BYTES;
+                        tma_load_2d(dst, &tm_w, (kb + j) * C::RAW_ROW, row_a, r_full(s + j));
+                        tma_load_2d(dst + C::RAW_BYTES / 2, &tm_w, (kb + j) * C::RAW_ROW, row_b, r_full(s + j));
+                        if (j == 0) {   // the 8 scales per row that cover these four k-blocks
+                            tma_load_2d(sd, &tm_s, (kb >> 2) * 8, row_a, r_full(s));
+                            tma_load_2d(sd + C::SC_BYTES / 2, &tm_s, (kb >> 2) * 8, row_b, r_full(s));
+                        }
+                    }
+                }
+                __syncwarp();
+                if (++sg == C::NSB) sg = 0;
+                s ^= 4u;
+                if (s == 0) ph ^= 1u;
             }
+        }
+        __syncwarp();
+        if (lane == 0) QG_FLUSH();
+    } else if (warp == 1 || warp == 3) {
+        // ------------------------------------------------ MMA issuers (even CTA of the pair only)
+        // One warp needs about 500-560 cycles to issue the four TMEM-operand MMAs, the commit and the wait of a
+        // k-block, more than the 256-512 cycles the tensor cores need for it, and two warps issue concurrently at
+        // full speed; so warps 1 and 3 take the even and the odd k-blocks.  MMAs of different threads are ordered
+        // only through completion, so the odd warp starts a tile after the "done" of the tile's first k-block (which
+        // overwrites the accumulator); within a tile the order of the accumulating k-blocks does not matter.
+        if (rank == 0) {
+            const uint32_t w = (warp == 3) ? 1u : 0u;
+            bool ok = true;
+            QG_DECL();
+            const uint32_t b_hi = (1024u >> 4) | (1u << 14) | (2u << 29);   // stride, version, 128-byte swizzle
+            const uint32_t b_lo0 = ((sbase + C::OFF_X) >> 4) | (1u << 16);
+            uint32_t j = 0;
+            for (int t = pair; t < total_tiles && ok; t += n_pairs, ++j) {
+                const Tile tl = decode_tile(t, prefix, p, BT);
+                const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
+                const uint32_t idesc = umma_idesc_bf16(2 * BW, n_mma);
+                const uint32_t a = (C::NACC == 2) ? (j & 1u) : 0u;
+                const uint32_t aph = (C::NACC == 2) ? ((j >> 1) & 1u) : (j & 1u);
+                const uint32_t i0 = j * static_cast<uint32_t>(nkb);          // first k-block of the tile (ring index)
+                QG_T0();
+                if (w == 0) {
+                    if (!wait_bar<true>(acc_empty(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                } else {
+                    if (!wait_bar<false>(done(i0 & 7u), (i0 >> 3) & 1u, abort_flag, p.status)) { ok = false; break; }
+                }
+                QG_ACC(2);
+                const uint32_t d_tmem = tmem_base + a * BT;
+                uint32_t i = i0 + w;
+                bool ready = mbar_try_wait_cluster(full(i & 7u), (i >> 3) & 1u);
+                for (int kb = static_cast<int>(w); kb < nkb; kb += 2, i += 2) {
+                    const uint32_t st = i & 7u;
+                    QG_T0();
+                    if (!ready && !wait_bar<true>(full(st), (i >> 3) & 1u, abort_flag, p.status)) { ok = false; break; }
+                    QG_ACC(3);
+                    tc_fence_after_sync();
+                    // start the wait for this warp's next k-block before issuing, so its latency is hidden
+                    ready = (kb + 2 < nkb) && mbar_try_wait_cluster(full((i + 2) & 7u), ((i + 2) >> 3) & 1u);
+                    if (lane == 0) {
+                        umma_kblock_ts_pair(d_tmem, tmem_base + C::A_COL0 + st * C::A_COLS,
+                                            b_lo0 + st * (C::X_BYTES >> 4), b_hi, idesc, kb != 0 ? 1u : 0u);
+                        umma_commit_pair(done(st));
+                    }
+                    __syncwarp();
+                    QG_ACC(10);
+                }
+                if (ok && lane == 0) umma_commit_pair(acc_full(a));
+                __syncwarp();
+            }
+            __syncwarp();
+            if (lane == 0 && w == 0) QG_FLUSH();
+        }
+    } else if (warp >= 8) {
+        // ------------------------------------------------ dequantise: raw ring -> TMEM weight stages
+        // Four groups of four warps; group g owns TMEM weight stage g and converts the k-blocks i = g (mod 4), so
+        // a warp has four k-block periods for one round of waits, loads, arithmetic and tensor-memory stores.
+        // Warp (g, q) covers weight rows 32 q .. 32 q + 31 (a warp may only touch the TMEM lanes of its quarter);
+        // thread = one row, all 64 k of the k-block: 64 bytes (Q8) or 32 bytes (Q4) of packed codes, read from the
+        // swizzled raw tile without bank conflicts, 2 scales, 32 TMEM columns out.
+        const int g = (warp - 8) >> 2, q = warp & 3;
+        const int row = q * 32 + lane;
+        const uint32_t swz = (QBITS == 8) ? ((row >> 1) & 3u) : ((row >> 2) & 1u);
+        const uint32_t raw_row = row * C::RAW_ROW;
+        const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + C::A_COL0;
+        const uint32_t full_leader = map_to_cta(full(0), 0);
+        const int my_tiles = (total_tiles > pair) ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
+        const uint32_t n_own = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(nkb >> 2);
+        QG_DECL();
+        for (uint32_t n = 0; n < n_own; ++n) {       // own k-block i = 4 n + g
+            const uint32_t sr = ((n & 1u) << 2) + g;               // ring stage i % 8
+            const uint32_t phr = (n >> 1) & 1u;                    // parity of (i / 8)
+            QG_T0();
+            // the scales of this group of four k-blocks arrive with the first of them (stage 0 or 4)
+            if (!wait_bar<false>(r_full((n & 1u) << 2), phr, abort_flag, p.status)) break;
+            if (!wait_bar<false>(r_full(sr), phr, abort_flag, p.status)) break;
             QG_ACC(5);
-            if (td == 0) { QG_TRACE(5, it); }
-            const int sr = it % C::SR, sb = it % C::SB;
-            ok = wait_bar(w_empty(sb), ((it / C::SB) & 1u) ^ 1u, abort_flag, p.status);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
+            if (warp == 8 && lane == 0) { QG_TRACE(5, 4 * n); }
+            const uint32_t raw = sbase + C::OFF_RAW + sr * C::RAW_BYTES + raw_row;
+            const uint32_t scw = *reinterpret_cast<const uint32_t*>(
+                sgen + C::OFF_SC + (n % C::NSB) * C::SC_BYTES + row * 16 + g * 4);
+            const float s0 = __half2float(__ushort_as_half(static_cast<unsigned short>(scw & 0xFFFFu)));
+            const float s1 = __half2float(__ushort_as_half(static_cast<unsigned short>(scw >> 16)));
+            uint32_t o[32];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {            // k = 32 h .. 32 h + 31 share one scale
+                const float sc = h ? s1 : s0;
+                uint32_t* oh = o + 16 * h;
+                if constexpr (QBITS == 8) {
+                    const uint4 v0 = lds128(raw + (((2 * h) ^ swz) << 4));
+                    const uint4 v1 = lds128(raw + (((2 * h + 1) ^ swz) << 4));
+                    const float s256 = 256.f * sc, c = -32896.f * sc;
+                    dq8_word(v0.x, s256, c, oh[0], oh[1]);
+                    dq8_word(v0.y, s256, c, oh[2], oh[3]);
+                    dq8_word(v0.z, s256, c, oh[4], oh[5]);
+                    dq8_word(v0.w, s256, c, oh[6], oh[7]);
+                    dq8_word(v1.x, s256, c, oh[8], oh[9]);
+                    dq8_word(v1.y, s256, c, oh[10], oh[11]);
+                    dq8_word(v1.z, s256, c, oh[12], oh[13]);
+                    dq8_word(v1.w, s256, c, oh[14], oh[15]);
+                } else {
+                    const uint4 v = lds128(raw + ((h ^ swz) << 4));
+                    uint32_t w4[4];
+                    dq4_word(v.x, sc, w4); oh[0] = w4[0]; oh[1] = w4[1]; oh[2] = w4[2]; oh[3] = w4[3];
+                    dq4_word(v.y, sc, w4); oh[4] = w4[0]; oh[5] = w4[1]; oh[6] = w4[2]; oh[7] = w4[3];
+                    dq4_word(v.z, sc, w4); oh[8] = w4[0]; oh[9] = w4[1]; oh[10] = w4[2]; oh[11] = w4[3];
+                    dq4_word(v.w, sc, w4); oh[12] = w4[0]; oh[13] = w4[1]; oh[14] = w4[2]; oh[15] = w4[3];
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(r_empty(sr));             // the packed codes are in registers now
+            QG_ACC(7);
+            // TMEM stage sr is free once the MMAs of k-block i - 8 (same stage) have completed
+            if (n >= 2 && !wait_bar<false>(done(sr), (phr ^ 1u), abort_flag, p.status)) break;
             QG_ACC(6);
-            if (td == 0) { QG_TRACE(6, it); }
+            if (warp == 8 && lane == 0) { QG_TRACE(6, 4 * n); }
             tc_fence_after_sync();
-            uint32_t o[8];
-            if constexpr (QBITS == 8) {
-                const float s256 = 256.f * s, c = -32896.f * s;
-                dq8_word(cur.x, s256, c, o[0], o[1]);
-                dq8_word(cur.y, s256, c, o[2], o[3]);
-                dq8_word(cur.z, s256, c, o[4], o[5]);
-                dq8_word(cur.w, s256, c, o[6], o[7]);
-            } else {
-                uint32_t q[4];
-                dq4_word(cur.x, s, q);
-                o[0] = q[0]; o[1] = q[1]; o[2] = q[2]; o[3] = q[3];
-                dq4_word(cur.y, s, q);
-                o[4] = q[0]; o[5] = q[1]; o[6] = q[2]; o[7] = q[3];
-            }
-#ifdef QG_PROFILE
-            if (!(p.dbg & 1) || it < 4)
-#endif
             {
-                tmem_st_32x32_x8(a_taddr + sb * C::A_COLS, o);
-                tmem_st_wait();
+                uint32_t (&o0)[16] = *reinterpret_cast<uint32_t (*)[16]>(o);
+                uint32_t (&o1)[16] = *reinterpret_cast<uint32_t (*)[16]>(o + 16);
+                tmem_st_32x32_x16(a_taddr + sr * C::A_COLS, o0);
+                tmem_st_32x32_x16(a_taddr + sr * C::A_COLS + 16, o1);
             }
+            tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(w_full(sb));
-                mbar_arrive(r_empty(sr));
-            }
+            if (lane == 0) mbar_arrive_cluster(full_leader + 8u * sr);
             QG_ACC(7);
-            if (td == 0) { QG_TRACE(7, it); }
+            if (warp == 8 && lane == 0) { QG_TRACE(7, 4 * n); }
         }
-        if (td == 0) QG_FLUSH();
+        __syncwarp();
+        if (warp == 8 && lane == 0) QG_FLUSH();
     } else if (warp >= 4) {
         // ------------------------------------------------ epilogue (warps 4..7 <-> TMEM lanes 32 (warp-4) ..)
         const int qd = warp - 4;
         const int et = threadIdx.x - 128;
         __nv_bfloat16* outb = static_cast<__nv_bfloat16*>(p.out);
         float* outf = static_cast<float*>(p.out);
+        const uint32_t acc_empty_base = map_to_cta(acc_empty(0), 0);
         uint32_t j = 0, cc = 0;
         QG_DECL();
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++j) {
+        for (int t = pair; t < total_tiles; t += n_pairs, ++j) {
             const Tile tl = decode_tile(t, prefix, p, BT);
-            const uint32_t a = j & 1u, aph = (j >> 1) & 1u;
+            const int wt = 2 * tl.pw + static_cast<int>(rank);     // may be one past the last tile: nothing is stored
+            const uint32_t a = (C::NACC == 2) ? (j & 1u) : 0u;
+            const uint32_t aph = (C::NACC == 2) ? ((j >> 1) & 1u) : (j & 1u);
+            const uint32_t fl = j & 1u;       // flag slot: alternates so a slow warp never reads a newer flag
             QG_T0();
-            if (et == 0) misc[2 + a] = wait_bar(acc_full(a), aph, abort_flag, p.status) ? 1 : 0;
+            if (et == 0) misc[2 + fl] = wait_bar<false>(acc_full(a), aph, abort_flag, p.status) ? 1 : 0;
             tc_fence_before_sync();
             named_bar_sync(1, 128);
-            if (!misc[2 + a]) break;
+            if (!misc[2 + fl]) break;
             tc_fence_after_sync();
             QG_ACC(8);
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + a * BT;
-#ifdef QG_PROFILE
-            const int n_epi = (p.dbg & 2) ? 0 : n_mma;
-#else
-            const int n_epi = n_mma;
-#endif
+            const int n_epi = (wt < p.n_wt) ? n_mma : 0;
             for (int c = 0; c < n_epi; c += 32, ++cc) {
                 uint32_t v[32];
                 tmem_ld_32x32(taddr + c, v);
@@ -468,7 +495,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 const int row = qd * 32 + lane;          // weight row of this thread inside the tile
                 if (p.mode == QG_MODE_DOWN_ACCUM_F32) {
                     // y[token, n] += w * acc: lanes are consecutive n, so each warp-wide red covers 128 bytes
-                    const int n = tl.wt * BW + row;
+                    const int n = wt * BW + row;
                     const int tokl = tl.tok0 + c + lane;
                     int trow = 0;
                     float wv = 0.f;
@@ -484,7 +511,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                         if (tl.tok0 + c + jj < tl.tok_end && n < p.N)
                             atomicAdd(outf + static_cast<size_t>(tr) * p.N + n, w * __uint_as_float(v[jj]));
                     }
-                } else if (p.mode == QG_MODE_GATE_UP_SILU) {
+                } else if (gate_up) {
                     // lanes 0..63 hold gate rows, 64..127 the matching up rows: transpose through shared memory
                     // ([32 tokens][128 rows] fp32), then every thread finishes 16 outputs of one token.
                     const int F = p.N / 2;
@@ -507,7 +534,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                         o[2 * i + 1] = bf16x2(h2, h3);
                     }
                     if (tok < tl.tok_end) {
-                        uint4* dst = reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * F + tl.wt * 64 + f0);
+                        uint4* dst = reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * F + wt * 64 + f0);
                         dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                         dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
                     }
@@ -533,7 +560,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                         const int piece = i * 128 + et;
                         const int tk = piece >> 4, c16 = piece & 15;
                         const int tok = tl.tok0 + c + tk;
-                        const int n = tl.wt * BW + c16 * 8;
+                        const int n = wt * BW + c16 * 8;
                         if (tok < tl.tok_end && n < p.N)
                             *reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * p.N + n) =
                                 *reinterpret_cast<const uint4*>(st + tk * 128 + c16 * 8);
@@ -542,7 +569,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty(a));
+            if (lane == 0) mbar_arrive_cluster(acc_empty_base + 8u * a);
             QG_ACC(9);
         }
         if (et == 0) QG_FLUSH();
@@ -554,8 +581,10 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         // copies may still be in flight towards this CTA's shared memory: give them time to land
         for (int i = 0; i < 64; ++i) __nanosleep(2000);
     }
+    tc_fence_before_sync();
+    cluster_sync_all();          // the peer no longer reads this CTA's shared memory or signals its barriers
     tc_fence_after_sync();
-    if (warp == 3) tmem_dealloc(tmem_base, C::TMEM_COLS);
+    if (warp == 3) tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
 }
 
 template <int QBITS, int BT>
@@ -563,16 +592,13 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const vo
                        cudaStream_t st) {
     using C = Cfg<QBITS, BT>;
     static_assert(C::SMEM_BYTES <= 232448, "shared memory budget");
-    CUtensorMap tm_x, tm_xh, tm_w, tm_s;
+    CUtensorMap tm_x, tm_w, tm_s;
     const uint64_t wrows = static_cast<uint64_t>(p.E) * p.N;
-    int rc = make_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, p.R, BK, BT,
-                          CU_TENSOR_MAP_SWIZZLE_128B);
-    if (rc == QG_OK)
-        rc = make_tmap_2d(ctx, &tm_xh, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, p.R, BK, BT / 2,
+    int rc = make_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, p.R, BK, C::XH_ROWS,
                           CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc == QG_OK)
         rc = make_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (QBITS == 8) ? p.K : p.K / 2, wrows,
-                          C::RAW_ROW, 64, CU_TENSOR_MAP_SWIZZLE_NONE);
+                          C::RAW_ROW, 64, (QBITS == 8) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
     if (rc == QG_OK)
         rc = make_tmap_2d(ctx, &tm_s, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, Ws, p.K / 32, wrows, 8, 64,
                           CU_TENSOR_MAP_SWIZZLE_NONE);
@@ -586,15 +612,17 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const vo
         }
         attr_set = true;
     }
-    // Upper bound on the number of tiles (the exact count lives on the device for grouped calls).
-    const long long max_tiles = (static_cast<long long>((p.R + BT - 1) / BT) + (p.offsets ? p.E : 0)) * p.n_wt;
-    const int grid = static_cast<int>(max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count);
-    kern<<<grid, NTHREADS, C::SMEM_BYTES, st>>>(tm_x, tm_xh, tm_w, tm_s, p);
+    // Upper bound on the number of pair tiles (the exact count lives on the device for grouped calls).
+    const long long max_tiles =
+        (static_cast<long long>((p.R + BT - 1) / BT) + (p.offsets ? p.E : 0)) * ((p.n_wt + 1) / 2);
+    const long long pairs_hw = ctx->sm_count / 2;
+    const int grid = 2 * static_cast<int>(max_tiles < pairs_hw ? max_tiles : pairs_hw);
+    kern<<<grid, NTHREADS, C::SMEM_BYTES, st>>>(tm_x, tm_w, tm_s, p);
     return cudaGetLastError() == cudaSuccess ? QG_OK : QG_ERR_CUDA;
 }
 
 #ifdef QG_PROFILE
-static long long* g_stats = nullptr;   // device buffer [grid, 12] supplied by the profiling harness
+static long long* g_stats = nullptr;   // device buffer supplied by the profiling harness
 #endif
 
 static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in, const void* X, const void* Wq,
@@ -602,14 +630,14 @@ static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in,
     GemmParams p = p_in;
     if (const char* f = getenv("QG_FORCE_BT")) {   // tile-shape override for sweeps
         const int v = atoi(f);
-        if (v == 128 || v == 192) bt = v;
+        if (v == 128 || v == 256) bt = v;
     }
 #ifdef QG_PROFILE
     p.stats = g_stats;
     if (const char* d = getenv("QG_DBG")) p.dbg = atoi(d);
 #endif
-    if (qbits == QG_Q8) return bt == 192 ? launch_gemm<8, 192>(ctx, p, X, Wq, Ws, st) : launch_gemm<8, 128>(ctx, p, X, Wq, Ws, st);
-    return bt == 192 ? launch_gemm<4, 192>(ctx, p, X, Wq, Ws, st) : launch_gemm<4, 128>(ctx, p, X, Wq, Ws, st);
+    if (qbits == QG_Q8) return bt == 256 ? launch_gemm<8, 256>(ctx, p, X, Wq, Ws, st) : launch_gemm<8, 128>(ctx, p, X, Wq, Ws, st);
+    return bt == 256 ? launch_gemm<4, 256>(ctx, p, X, Wq, Ws, st) : launch_gemm<4, 128>(ctx, p, X, Wq, Ws, st);
 }
 
 }  // namespace qg
@@ -622,23 +650,26 @@ void qg_debug_set_stats(long long* dev_buf) { qg::g_stats = dev_buf; }
 
 int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq, const void* Wscale,
                 void* Cout, void* stream) {
-    if (!ctx || !A || !Wq || !Wscale || !Cout) return QG_ERR_NULL;
+    if (!ctx) return QG_ERR_NULL;
     if (qbits != QG_Q8 && qbits != QG_Q4) return QG_ERR_SHAPE;
     if (M < 0 || N < 8 || N % 8 || K < 256 || K % 256) return QG_ERR_SHAPE;
+    if (M == 0) return QG_OK;     // nothing to do: empty tensors may carry null pointers
+    if (!A || !Wq || !Wscale || !Cout) return QG_ERR_NULL;
     if (!qg::aligned16(A) || !qg::aligned16(Wq) || !qg::aligned16(Wscale) || !qg::aligned16(Cout)) return QG_ERR_ALIGN;
-    if (M == 0) return QG_OK;
     qg::GemmParams p{};
     p.mode = QG_MODE_PLAIN; p.R = M; p.N = N; p.K = K; p.E = 1; p.k = 1;
     p.n_wt = (N + qg::BW - 1) / qg::BW;
     p.offsets = nullptr; p.out = Cout; p.topk_w = nullptr; p.row_pair = nullptr; p.status = ctx->d_status;
-    const int bt = (M > 128) ? 192 : 128;
+    const int bt = (M > 128) ? 256 : 128;
     return qg::dispatch_gemm(ctx, qbits, bt, p, A, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 
 int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int K, const void* Ain,
                       const int32_t* expert_offsets, const void* Wq, const void* Wscale, const float* topk_w,
                       const int32_t* row_pair, int k, void* Out, void* stream) {
-    if (!ctx || !Ain || !expert_offsets || !Wq || !Wscale || !Out) return QG_ERR_NULL;
+    if (!ctx) return QG_ERR_NULL;
+    if (R == 0) return QG_OK;     // nothing to do: empty tensors may carry null pointers
+    if (!Ain || !expert_offsets || !Wq || !Wscale || !Out) return QG_ERR_NULL;
     if (qbits != QG_Q8 && qbits != QG_Q4) return QG_ERR_SHAPE;
     if (mode < QG_MODE_PLAIN || mode > QG_MODE_DOWN_ACCUM_F32) return QG_ERR_SHAPE;
     if (R < 0 || E < 1 || E > qg::MAX_E || N < 8 || N % 8 || K < 256 || K % 256) return QG_ERR_SHAPE;
@@ -647,12 +678,11 @@ int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int
     if (mode == QG_MODE_DOWN_ACCUM_F32 && k < 1) return QG_ERR_SHAPE;
     if (static_cast<long long>(E) * N > 0x7FFFFFFF) return QG_ERR_SHAPE;
     if (!qg::aligned16(Ain) || !qg::aligned16(Wq) || !qg::aligned16(Wscale) || !qg::aligned16(Out)) return QG_ERR_ALIGN;
-    if (R == 0) return QG_OK;
     qg::GemmParams p{};
     p.mode = mode; p.R = R; p.N = N; p.K = K; p.E = E; p.k = (k < 1) ? 1 : k;
     p.n_wt = (mode == QG_MODE_GATE_UP_SILU) ? (N / 128) : (N + qg::BW - 1) / qg::BW;
     p.offsets = expert_offsets; p.out = Out; p.topk_w = topk_w; p.row_pair = row_pair; p.status = ctx->d_status;
-    const int bt = (R / E > 100) ? 192 : 128;   // expected rows per expert decide the token tile
+    const int bt = (R / E > 100) ? 256 : 128;   // expected rows per expert decide the token tile
     return qg::dispatch_gemm(ctx, qbits, bt, p, Ain, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 

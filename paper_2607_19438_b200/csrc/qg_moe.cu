@@ -232,8 +232,10 @@ size_t qg_route_workspace_bytes(int M, int E, int k) {
 }
 
 int moe_permute(qg_ctx* ctx, int M, int k, int H, const void* X, const int32_t* row_pair, void* Xperm, void* stream) {
-    if (!ctx || !X || !row_pair || !Xperm) return QG_ERR_NULL;
+    if (!ctx) return QG_ERR_NULL;
     if (M < 0 || k < 1 || H < 8 || H % 8) return QG_ERR_SHAPE;
+    if (M == 0) return QG_OK;
+    if (!X || !row_pair || !Xperm) return QG_ERR_NULL;
     if (!qg::aligned16(X) || !qg::aligned16(Xperm)) return QG_ERR_ALIGN;
     const long long R = static_cast<long long>(M) * k;
     if (R == 0) return QG_OK;
@@ -286,11 +288,12 @@ int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* to
 
 int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
                 const float* topk_w, void* Y, void* stream) {
-    if (!ctx || !D || !Y) return QG_ERR_NULL;
+    if (!ctx) return QG_ERR_NULL;
     if (M < 0 || k < 1 || H < 8 || H % 8) return QG_ERR_SHAPE;
     if (d_kind != QG_D_BF16 && d_kind != QG_D_F32_ACC) return QG_ERR_SHAPE;
-    if (!qg::aligned16(D) || !qg::aligned16(Y)) return QG_ERR_ALIGN;
     if (M == 0) return QG_OK;
+    if (!D || !Y) return QG_ERR_NULL;
+    if (!qg::aligned16(D) || !qg::aligned16(Y)) return QG_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (d_kind == QG_D_F32_ACC) {
         const size_t n8 = static_cast<size_t>(M) * H / 8;

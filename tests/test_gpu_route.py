@@ -104,8 +104,9 @@ def test_error_codes_are_returned_before_any_launch():
     A = torch.zeros((4, 256), dtype=torch.bfloat16, device="cuda")
     Wq = torch.zeros((8, 256), dtype=torch.int8, device="cuda")
     Ws = torch.zeros((8, 8), dtype=torch.float16, device="cuda")
+    big = torch.zeros(8 * 256 + 16, dtype=torch.int8, device="cuda")
     with pytest.raises(qg.QGemmError) as e:
-        qg.qgemm_dense(8, A, Wq.view(-1)[1:], Ws)     # misaligned weight pointer
+        qg.qgemm_dense(8, A, big[1:1 + 8 * 256].view(8, 256), Ws)     # misaligned weight pointer
     assert e.value.code == -3
     with pytest.raises(qg.QGemmError) as e:
         qg.qgemm_dense(5, A, Wq, Ws)
