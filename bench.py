@@ -218,7 +218,7 @@ def run_ours(args):
                 e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True); e0.record(stream)
             chk(lib.qgemm_dense(ctx, 8, M, N, K, P(A_list[i]), P(dW[i][1]), P(dW[i][2]), P(oC[i]), S), "qgemm_dense")
             if record:
-                e1.record(stream); gemm_events.append(("dense_q8", 2.0 * M * N * K, e0, e1))
+                e1.record(stream); gemm_events.append(("dense_q8_" + name, 2.0 * M * N * K, e0, e1))
         if record:
             r0 = torch.cuda.Event(enable_timing=True); r1 = torch.cuda.Event(enable_timing=True); r0.record(stream)
         chk(lib.moe_route(ctx, M, E, k, P(L), P(o["idx"]), P(o["w"]), P(o["counts"]), P(o["offsets"]), P(o["row_pair"]),
@@ -284,7 +284,10 @@ def run_ours(args):
     detail = {lab: {"launches": v[2], "avg_us": v[1] / v[2] * 1e3, "tflops": (v[0] / (v[1] * 1e-3) / 1e12) if v[0] else None}
               for lab, v in agg.items()}
     peak_tf, peak_hbm, peak_src = measured_peaks()
-    dq = agg["dense_q8"]
+    dq = [0.0, 0.0, 0]
+    for lab, v in agg.items():
+        if lab.startswith("dense_q8_"):
+            dq[0] += v[0]; dq[1] += v[1]; dq[2] += v[2]
     achieved = dq[0] / (dq[1] * 1e-3) / 1e12
     roofline = {"kernel": "qgemm_kernel<Q8, 256 tokens> (qgemm_dense, 4 launches per step)", "bound": "tensor",
                 "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
@@ -292,7 +295,7 @@ def run_ours(args):
                 "avg_launch_us": dq[1] / dq[2] * 1e3, "flops_per_launch": dq[0] / dq[2]}
     gemm_ms = sum(v[1] for lab, v in agg.items() if v[0])
     gemm_fl = sum(v[0] for lab, v in agg.items() if v[0])
-    dense_ms = agg["dense_q8"][1] / args.steps
+    dense_ms = dq[1] / args.steps
     moe_ms = sum(agg[lab][1] for lab in ("route_permute", "moe_gate_up_q4", "moe_down_q4", "combine")) / args.steps
 
     # ---- end-to-end leg: host inputs in pinned memory, copies inside the timed region

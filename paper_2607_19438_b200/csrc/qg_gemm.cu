@@ -69,7 +69,8 @@ struct Cfg {
                                                                    // (smem), the packed weights (smem), the dequantised
                                                                    // weights (TMEM) and the full/done barriers
     static constexpr int SR = SX;
-    static constexpr int NACC = (BT > 128) ? 1 : 2;                // accumulators in tensor memory
+    static constexpr int NACC = (BT > 192) ? 1 : 2;                // accumulators in tensor memory
+    static constexpr int SA = ((512 - NACC * BT) / 32 >= 8) ? 8 : 4;   // dequantised-weight stages in tensor memory
     static constexpr int NSB = 3;                                  // scale buffers (one per 4 k-blocks)
     static constexpr int XH_ROWS = BT / 2;                         // token rows this CTA stages per k-block
     static constexpr int X_BYTES = XH_ROWS * 128;
@@ -89,7 +90,7 @@ struct Cfg {
     static constexpr int TMEM_COLS = 512;                          // accumulator(s) + SX weight stages
     static constexpr int A_COL0 = NACC * BT;                       // first column of the weight stages
     static constexpr int A_COLS = 32;                              // 64 bf16 per lane = 32 columns per stage
-    static_assert(NACC * BT + SX * 32 <= 512, "tensor memory budget");
+    static_assert(NACC * BT + SA * 32 <= 512, "tensor memory budget");
     static_assert(X_BYTES % 1024 == 0, "swizzled stages must stay 1024-byte aligned");
     static_assert(SX == 8, "stage arithmetic below assumes a ring of eight");
 };
@@ -126,6 +127,14 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     *abort_flag = 1;
     atomicCAS(status, 0, QG_ERR_TIMEOUT);
     return false;
+}
+
+// Same for the MMA warps: a short non-blocking spin first (the barrier is usually complete or about to be), then
+// the bounded blocking wait.
+__device__ __forceinline__ bool spin_wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    for (int it = 0; it < 64; ++it)
+        if (mbar_test_wait_cluster(bar, parity)) return true;
+    return wait_bar<true>(bar, parity, abort_flag, status);
 }
 
 __device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
@@ -262,7 +271,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     // four-MMA statement and one commit per k-block.
     if (warp == 0) {
         // ------------------------------------------------ activation producer (this CTA's half of the token tile)
-        uint32_t s = 0, ph = 0;      // first stage of the next batch (0 or 4) and the parity of its next "done" phase
+        uint32_t s = 0, ph = 0;      // first stage of the next batch (0, 2, 4, 6) and the parity of its next "done" phase
         const uint32_t full_leader = map_to_cta(full(0), 0);
         bool ok = true;
         QG_DECL();
@@ -270,23 +279,28 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const Tile tl = decode_tile(t, prefix, p, BT);
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const int row0 = tl.tok0 + static_cast<int>(rank) * (n_mma >> 1);   // B rows split at N / 2
-            for (int kb = 0; kb < nkb; kb += 4) {
+            for (int kb = 0; kb < nkb; kb += 2) {
                 QG_T0();
-                // stages s..s+3 are free once the MMAs that read them eight k-blocks ago are done; the even and the odd
-                // stages belong to different MMA warps, each of which completes its k-blocks in order
-                if (!wait_bar<false>(done(s + 2), ph ^ 1u, abort_flag, p.status) ||
-                    !wait_bar<false>(done(s + 3), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                // a stage is free once the MMAs that read it eight k-blocks ago are done (even and odd stages
+                // belong to different MMA warps, so both are checked)
+                if (!wait_bar<false>(done(s), ph ^ 1u, abort_flag, p.status) ||
+                    !wait_bar<false>(done(s + 1), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                 QG_ACC(0);
+#ifdef QG_PROFILE
+                if (p.dbg & 8) {
+                    if (lane == 0 && rank == 0) { mbar_arrive(full(s)); mbar_arrive(full(s + 1)); }
+                } else
+#endif
                 if (lane == 0) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
+                    for (int j = 0; j < 2; ++j) {
                         if (rank == 0) mbar_arrive_expect_tx(full(s + j), 2 * C::X_BYTES);
                         tma_load_2d_pair(sbase + C::OFF_X + (s + j) * C::X_BYTES, &tm_x, (kb + j) * BK, row0,
                                          full_leader + 8u * (s + j));
                     }
                 }
                 __syncwarp();
-                s ^= 4u;
+                s = (s + 2u) & 7u;
                 if (s == 0) ph ^= 1u;
             }
         }
@@ -309,6 +323,11 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     if (ok && !wait_bar<false>(r_empty(s + j), ph ^ 1u, abort_flag, p.status)) ok = false;
                 if (!ok) break;
                 QG_ACC(1);
+#ifdef QG_PROFILE
+                if (p.dbg & 32) {
+                    if (lane == 0) { for (int j = 0; j < 4; ++j) mbar_arrive(r_full(s + j)); }
+                } else
+#endif
                 if (lane == 0) {
                     const uint32_t sd = sbase + C::OFF_SC + sg * C::SC_BYTES;
 #pragma unroll
@@ -354,24 +373,24 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 const uint32_t i0 = j * static_cast<uint32_t>(nkb);          // first k-block of the tile (ring index)
                 QG_T0();
                 if (w == 0) {
-                    if (!wait_bar<true>(acc_empty(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    if (!spin_wait_bar(acc_empty(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                 } else {
-                    if (!wait_bar<false>(done(i0 & 7u), (i0 >> 3) & 1u, abort_flag, p.status)) { ok = false; break; }
+                    if (!spin_wait_bar(done(i0 & 7u), (i0 >> 3) & 1u, abort_flag, p.status)) { ok = false; break; }
                 }
                 QG_ACC(2);
                 const uint32_t d_tmem = tmem_base + a * BT;
                 uint32_t i = i0 + w;
-                bool ready = mbar_try_wait_cluster(full(i & 7u), (i >> 3) & 1u);
+                bool ready = mbar_test_wait_cluster(full(i & 7u), (i >> 3) & 1u);
                 for (int kb = static_cast<int>(w); kb < nkb; kb += 2, i += 2) {
                     const uint32_t st = i & 7u;
                     QG_T0();
-                    if (!ready && !wait_bar<true>(full(st), (i >> 3) & 1u, abort_flag, p.status)) { ok = false; break; }
+                    if (!ready && !spin_wait_bar(full(st), (i >> 3) & 1u, abort_flag, p.status)) { ok = false; break; }
                     QG_ACC(3);
                     tc_fence_after_sync();
                     // start the wait for this warp's next k-block before issuing, so its latency is hidden
-                    ready = (kb + 2 < nkb) && mbar_try_wait_cluster(full((i + 2) & 7u), ((i + 2) >> 3) & 1u);
+                    ready = (kb + 2 < nkb) && mbar_test_wait_cluster(full((i + 2) & 7u), ((i + 2) >> 3) & 1u);
                     if (lane == 0) {
-                        umma_kblock_ts_pair(d_tmem, tmem_base + C::A_COL0 + st * C::A_COLS,
+                        umma_kblock_ts_pair(d_tmem, tmem_base + C::A_COL0 + (st & (C::SA - 1)) * C::A_COLS,
                                             b_lo0 + st * (C::X_BYTES >> 4), b_hi, idesc, kb != 0 ? 1u : 0u);
                         umma_commit_pair(done(st));
                     }
@@ -415,6 +434,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const float s0 = __half2float(__ushort_as_half(static_cast<unsigned short>(scw & 0xFFFFu)));
             const float s1 = __half2float(__ushort_as_half(static_cast<unsigned short>(scw >> 16)));
             uint32_t o[32];
+#ifdef QG_PROFILE
+            if (p.dbg & 16) {
+#pragma unroll
+                for (int z = 0; z < 32; ++z) o[z] = scw + z;
+            } else
+#endif
 #pragma unroll
             for (int h = 0; h < 2; ++h) {            // k = 32 h .. 32 h + 31 share one scale
                 const float sc = h ? s1 : s0;
@@ -443,16 +468,25 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             __syncwarp();
             if (lane == 0) mbar_arrive(r_empty(sr));             // the packed codes are in registers now
             QG_ACC(7);
-            // TMEM stage sr is free once the MMAs of k-block i - 8 (same stage) have completed
-            if (n >= 2 && !wait_bar<false>(done(sr), (phr ^ 1u), abort_flag, p.status)) break;
+            // its TMEM stage (i % SA) is free once the MMAs of k-block i - SA have completed
+            if constexpr (C::SA == 8) {
+                if (n >= 2 && !wait_bar<false>(done(sr), (phr ^ 1u), abort_flag, p.status)) break;
+            } else {
+                if (n >= 1 && !wait_bar<false>(done((((n - 1) & 1u) << 2) + g), ((n - 1) >> 1) & 1u, abort_flag, p.status)) break;
+            }
             QG_ACC(6);
             if (warp == 8 && lane == 0) { QG_TRACE(6, 4 * n); }
             tc_fence_after_sync();
             {
                 uint32_t (&o0)[16] = *reinterpret_cast<uint32_t (*)[16]>(o);
                 uint32_t (&o1)[16] = *reinterpret_cast<uint32_t (*)[16]>(o + 16);
-                tmem_st_32x32_x16(a_taddr + sr * C::A_COLS, o0);
-                tmem_st_32x32_x16(a_taddr + sr * C::A_COLS + 16, o1);
+#ifdef QG_PROFILE
+                if (!(p.dbg & 1) || n < 2)
+#endif
+                {
+                    tmem_st_32x32_x16(a_taddr + (sr & (C::SA - 1)) * C::A_COLS, o0);
+                    tmem_st_32x32_x16(a_taddr + (sr & (C::SA - 1)) * C::A_COLS + 16, o1);
+                }
             }
             tmem_st_wait();
             tc_fence_before_sync();
@@ -488,7 +522,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + a * BT;
             const int n_epi = (wt < p.n_wt) ? n_mma : 0;
-            for (int c = 0; c < n_epi; c += 32, ++cc) {
+#ifdef QG_PROFILE
+            const int n_epi2 = (p.dbg & 2) ? 0 : n_epi;
+#else
+            const int n_epi2 = n_epi;
+#endif
+            for (int c = 0; c < n_epi2; c += 32, ++cc) {
                 uint32_t v[32];
                 tmem_ld_32x32(taddr + c, v);
                 tmem_ld_wait();
@@ -625,19 +664,44 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const vo
 static long long* g_stats = nullptr;   // device buffer supplied by the profiling harness
 #endif
 
+// Token tile of a dense call: the candidate with the smallest modelled time.  A wave is one pair tile per SM pair;
+// a tile costs nkb k-blocks of about `period` cycles (measured: issue- and latency-bound, nearly independent of
+// the tile width) plus, for the single-accumulator 256-wide tile, an epilogue that is not overlapped.
+static int pick_token_tile(const qg_ctx* ctx, int M, int n_wt, int K) {
+    if (M <= 128) return 128;
+    const int cand[3] = {128, 192, 256};
+    const double period[3] = {670.0, 700.0, 720.0}, epilogue[3] = {0.0, 0.0, 8000.0};
+    const long long pairs = ctx->sm_count / 2, n_pw = (n_wt + 1) / 2;
+    int best = 256;
+    double best_cost = 1e300;
+    for (int c = 0; c < 3; ++c) {
+        const long long tiles = n_pw * ((M + cand[c] - 1) / cand[c]);
+        const long long waves = (tiles + pairs - 1) / pairs;
+        const double cost = static_cast<double>(waves) * ((K / BK) * period[c] + epilogue[c]);
+        if (cost < best_cost * 0.999) { best_cost = cost; best = cand[c]; }
+    }
+    return best;
+}
+
 static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in, const void* X, const void* Wq,
                          const void* Ws, cudaStream_t st) {
     GemmParams p = p_in;
     if (const char* f = getenv("QG_FORCE_BT")) {   // tile-shape override for sweeps
         const int v = atoi(f);
-        if (v == 128 || v == 256) bt = v;
+        if (v == 128 || v == 192 || v == 256) bt = v;
     }
 #ifdef QG_PROFILE
     p.stats = g_stats;
     if (const char* d = getenv("QG_DBG")) p.dbg = atoi(d);
 #endif
-    if (qbits == QG_Q8) return bt == 256 ? launch_gemm<8, 256>(ctx, p, X, Wq, Ws, st) : launch_gemm<8, 128>(ctx, p, X, Wq, Ws, st);
-    return bt == 256 ? launch_gemm<4, 256>(ctx, p, X, Wq, Ws, st) : launch_gemm<4, 128>(ctx, p, X, Wq, Ws, st);
+    if (qbits == QG_Q8) {
+        if (bt == 256) return launch_gemm<8, 256>(ctx, p, X, Wq, Ws, st);
+        if (bt == 192) return launch_gemm<8, 192>(ctx, p, X, Wq, Ws, st);
+        return launch_gemm<8, 128>(ctx, p, X, Wq, Ws, st);
+    }
+    if (bt == 256) return launch_gemm<4, 256>(ctx, p, X, Wq, Ws, st);
+    if (bt == 192) return launch_gemm<4, 192>(ctx, p, X, Wq, Ws, st);
+    return launch_gemm<4, 128>(ctx, p, X, Wq, Ws, st);
 }
 
 }  // namespace qg
@@ -660,7 +724,7 @@ int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, cons
     p.mode = QG_MODE_PLAIN; p.R = M; p.N = N; p.K = K; p.E = 1; p.k = 1;
     p.n_wt = (N + qg::BW - 1) / qg::BW;
     p.offsets = nullptr; p.out = Cout; p.topk_w = nullptr; p.row_pair = nullptr; p.status = ctx->d_status;
-    const int bt = (M > 128) ? 256 : 128;
+    const int bt = qg::pick_token_tile(ctx, M, p.n_wt, K);
     return qg::dispatch_gemm(ctx, qbits, bt, p, A, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 
@@ -682,7 +746,9 @@ int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int
     p.mode = mode; p.R = R; p.N = N; p.K = K; p.E = E; p.k = (k < 1) ? 1 : k;
     p.n_wt = (mode == QG_MODE_GATE_UP_SILU) ? (N / 128) : (N + qg::BW - 1) / qg::BW;
     p.offsets = expert_offsets; p.out = Out; p.topk_w = topk_w; p.row_pair = row_pair; p.status = ctx->d_status;
-    const int bt = (R / E > 100) ? 256 : 128;   // expected rows per expert decide the token tile
+    // expected rows per expert decide the token tile; 192 keeps two accumulators, so the short main loops of
+    // expert tiles overlap their epilogues
+    const int bt = (R / E > 100) ? 192 : 128;
     return qg::dispatch_gemm(ctx, qbits, bt, p, Ain, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 
