@@ -53,7 +53,8 @@ enum {
     QG_ERR_WORKSPACE = -4, /* workspace missing or too small */
     QG_ERR_ARCH = -5,      /* the device is not compute capability 10.x */
     QG_ERR_CUDA = -6,      /* a CUDA runtime / driver call failed */
-    QG_ERR_TIMEOUT = -7    /* a bounded device-side wait expired (reported by qg_poll_status) */
+    QG_ERR_TIMEOUT = -7,   /* a bounded device-side wait expired (reported by qg_poll_status) */
+    QG_ERR_TOO_LARGE = -8  /* the problem does not fit the library's built-in scratch (moe_route_static) */
 };
 enum { QG_Q8 = 8, QG_Q4 = 4 };
 enum {
@@ -96,6 +97,30 @@ int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, cons
 int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
               int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row,
               const void* X, void* Xperm, int H, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * moe_route without a workspace argument, for callers that have no way to provide scratch memory.
+ * (The paper has no counterpart to this call; it exists for integration reasons only.)
+ *
+ * Some hosts of this library cannot allocate device memory at the point where they route tokens: an
+ * inference server that carved up all of HBM at start-up and froze its allocator, a plug-in that is handed
+ * raw pointers and is forbidden to call the CUDA allocator, or a latency-critical loop that must not risk
+ * the device-wide synchronisation an allocation can imply.  For them the per-block expert histograms that
+ * moe_route keeps in `ws` live in a fixed 256 KiB array that is part of the library image on every GPU
+ * that loads it (held until the process exits).  Arguments and results are exactly those of moe_route.
+ *
+ *   limit    ceil(M / 32) * E <= 65536 (e.g. M <= 16384 tokens at E = 128); larger problems return
+ *            QG_ERR_TOO_LARGE before anything is launched - use moe_route with your own workspace then.
+ *   set-up   the first call on a device looks up the array's device address (with that device current,
+ *            which must be the context's device); make that first call outside any stream capture.
+ *   sharing  every call on a device uses the same array.  Nothing in it has to start at zero (each call
+ *            overwrites every entry it later reads), but two calls whose kernels overlap on the GPU - different
+ *            streams, or different host threads - race on it: serialise them.
+ *   The call itself never allocates or frees memory, on the host or on the device.
+ */
+int moe_route_static(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
+                     int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row,
+                     const void* X, void* Xperm, int H, void* stream);
 
 /* Xperm[r, :] = X[row_pair[r] / k, :] for r in [0, M*k): bit copy of bf16 rows, H % 8 == 0. */
 int moe_permute(qg_ctx* ctx, int M, int k, int H, const void* X, const int32_t* row_pair, void* Xperm,

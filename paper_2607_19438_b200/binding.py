@@ -19,7 +19,7 @@ MODE_PLAIN, MODE_GATE_UP_SILU, MODE_DOWN_WEIGHTED, MODE_DOWN_ACCUM_F32 = 0, 1, 2
 D_BF16, D_F32_ACC = 0, 1
 
 EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_route_workspace_bytes", "qgemm_dense",
-           "moe_route", "moe_permute", "moe_grouped_qgemm", "moe_combine"]
+           "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_combine"]
 
 
 class QGemmError(RuntimeError):
@@ -49,6 +49,7 @@ def load():
         vp, ci = C.c_void_p, C.c_int
         lib.qgemm_dense.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
         lib.moe_route.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp, C.c_size_t, vp]
+        lib.moe_route_static.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         lib.moe_permute.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
         lib.moe_grouped_qgemm.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp]
         lib.moe_combine.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp, vp, vp]
@@ -129,6 +130,28 @@ def moe_route(logits, k, X=None, ws=None):
     _check(load().moe_route(context(), M, E, k, _ptr(logits), _ptr(out["topk_idx"]), _ptr(out["topk_w"]),
                             _ptr(out["counts"]), _ptr(out["offsets"]), _ptr(out["row_pair"]), _ptr(out["pair_row"]),
                             _ptr(X), _ptr(Xp), H, _ptr(ws), ws.numel(), _stream()), "moe_route")
+    return out
+
+
+def moe_route_static(logits, k, X=None):
+    """moe_route for callers that cannot supply scratch memory: the block histograms live in a fixed array inside
+    the library (limit ceil(M/32)*E <= 65536, else QGemmError -8).  The output tensors are still the caller's; this
+    wrapper allocates them only for convenience.  Calls that overlap on the GPU share the array and would race."""
+    M, E = logits.shape
+    dev = logits.device
+    i32 = dict(dtype=torch.int32, device=dev)
+    out = dict(topk_idx=torch.empty((M, k), **i32), topk_w=torch.empty((M, k), dtype=torch.float32, device=dev),
+               counts=torch.empty(E, **i32), offsets=torch.empty(E + 1, **i32),
+               row_pair=torch.empty(M * k, **i32), pair_row=torch.empty(M * k, **i32))
+    H = 0
+    Xp = None
+    if X is not None:
+        H = X.shape[1]
+        Xp = torch.empty((M * k, H), dtype=torch.bfloat16, device=dev)
+        out["Xperm"] = Xp
+    _check(load().moe_route_static(context(), M, E, k, _ptr(logits), _ptr(out["topk_idx"]), _ptr(out["topk_w"]),
+                                   _ptr(out["counts"]), _ptr(out["offsets"]), _ptr(out["row_pair"]),
+                                   _ptr(out["pair_row"]), _ptr(X), _ptr(Xp), H, _stream()), "moe_route_static")
     return out
 
 

@@ -15,6 +15,7 @@ const char* qg_strerror(int code) {
         case QG_ERR_ARCH: return "device is not compute capability 10.x (sm_100a kernels only)";
         case QG_ERR_CUDA: return "CUDA runtime or driver call failed";
         case QG_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case QG_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of moe_route_static (ceil(M/32)*E <= 65536)";
         default: return "unknown error code";
     }
 }

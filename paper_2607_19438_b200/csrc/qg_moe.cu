@@ -220,6 +220,14 @@ round_f32_kernel(size_t n8, const float4* __restrict__ acc, int4* __restrict__ Y
 
 static int launch_ok() { return cudaGetLastError() == cudaSuccess ? QG_OK : QG_ERR_CUDA; }
 
+// Built-in scratch of moe_route_static: per-block expert histograms for callers that cannot hand over a workspace.
+// In host code this name is only a handle; the device address is looked up once per device (see below).
+constexpr int ROUTE_STATIC_MAX_INTS = 65536;   // 256 KiB
+static __device__ __align__(256) int32_t g_route_static_scratch[ROUTE_STATIC_MAX_INTS];
+constexpr int ROUTE_STATIC_MAX_DEVICES = 64;
+static int32_t* g_route_static_ptr[ROUTE_STATIC_MAX_DEVICES] = {nullptr};
+
+
 }  // namespace qg
 
 extern "C" {
@@ -281,6 +289,66 @@ int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* to
     qg::route_scatter_kernel<<<nb, qg::ROUTE_WARPS * 32, E * sizeof(int), st>>>(M, E, k, topk_idx, expert_offsets, hist,
                                                                                row_pair, pair_row);
     int rc = qg::launch_ok();
+    if (rc != QG_OK) return rc;
+    if (gather) return moe_permute(ctx, M, k, H, X, row_pair, Xperm, stream);
+    return QG_OK;
+}
+
+// moe_route with the block histograms in the library's own fixed device array instead of a caller workspace, for
+// callers that cannot allocate.  Same kernels, same results; no allocation of any kind happens here.
+int moe_route_static(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
+                     int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row,
+                     const void* X, void* Xperm, int H, void* stream) {
+    if (!ctx || !expert_counts || !expert_offsets) return QG_ERR_NULL;
+    if (M < 0 || E < 1 || E > 1024 || k < 1 || k > E) return QG_ERR_SHAPE;
+    if (M > 0 && (!logits || !topk_idx || !topk_w || !row_pair || !pair_row)) return QG_ERR_NULL;
+    if (static_cast<long long>(M) * k > 0x7FFFFFFF) return QG_ERR_SHAPE;
+    const bool gather = (X != nullptr) && (Xperm != nullptr);
+    if (gather && (H < 8 || H % 8)) return QG_ERR_SHAPE;
+    if (gather && (!qg::aligned16(X) || !qg::aligned16(Xperm))) return QG_ERR_ALIGN;
+    const long long nb = (static_cast<long long>(M) + qg::ROUTE_TOKENS_PER_BLOCK - 1) / qg::ROUTE_TOKENS_PER_BLOCK;
+    if (nb * E > qg::ROUTE_STATIC_MAX_INTS) return QG_ERR_TOO_LARGE;
+    // Set-up, once per device, with that device current: the array's name is a host-side stand-in, the kernels need
+    // its device address.
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != ctx->device || dev < 0 || dev >= qg::ROUTE_STATIC_MAX_DEVICES) {
+        cudaGetLastError();
+        return QG_ERR_CUDA;
+    }
+    if (!qg::g_route_static_ptr[dev]) {
+        int32_t* ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), qg::g_route_static_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return QG_ERR_CUDA;
+        }
+        qg::g_route_static_ptr[dev] = ptr;
+    }
+    int32_t* hist = qg::g_route_static_ptr[dev];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (M == 0) {
+        if (cudaMemsetAsync(expert_counts, 0, sizeof(int32_t) * E, st) != cudaSuccess ||
+            cudaMemsetAsync(expert_offsets, 0, sizeof(int32_t) * (E + 1), st) != cudaSuccess) {
+            cudaGetLastError();
+            return QG_ERR_CUDA;
+        }
+        return QG_OK;
+    }
+    const size_t sm_topk = (static_cast<size_t>(qg::ROUTE_WARPS) * (E + k) + E) * sizeof(float);
+    if (sm_topk > 48 * 1024) {
+        if (cudaFuncSetAttribute(qg::route_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(sm_topk)) != cudaSuccess) {
+            cudaGetLastError();
+            return QG_ERR_CUDA;
+        }
+    }
+    // every entry hist[b, e] that the scan and the scatter read is written by the first kernel of this call, so
+    // whatever an earlier call left in the shared array does not matter
+    const int nbi = static_cast<int>(nb);
+    qg::route_topk_kernel<<<nbi, qg::ROUTE_WARPS * 32, sm_topk, st>>>(M, E, k, logits, topk_idx, topk_w, hist);
+    qg::route_scan_kernel<<<1, 1024, 0, st>>>(nbi, E, hist, expert_counts, expert_offsets);
+    qg::route_scatter_kernel<<<nbi, qg::ROUTE_WARPS * 32, E * sizeof(int), st>>>(M, E, k, topk_idx, expert_offsets, hist,
+                                                                                row_pair, pair_row);
+    const int rc = qg::launch_ok();
     if (rc != QG_OK) return rc;
     if (gather) return moe_permute(ctx, M, k, H, X, row_pair, Xperm, stream);
     return QG_OK;
