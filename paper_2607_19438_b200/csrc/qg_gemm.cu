@@ -37,7 +37,7 @@ constexpr int MAX_E = 1024;
 constexpr uint32_t WAIT_LIMIT = 1u << 18;   // polls; an unsatisfied try_wait poll lasts about 4 us, so about a second
 
 // Profiling builds (-DQG_PROFILE) accumulate, per CTA, the cycles each role spends in each wait.
-#ifdef QG_PROFILE
+#if defined(QG_PROFILE) && !defined(QG_NOSTATS)
 #define QG_T0() long long qg_t0_ = clock64()
 #define QG_ACC(slot) do { if (p.stats) { long long now_ = clock64(); qg_stat_[slot] += now_ - qg_t0_; qg_t0_ = now_; } } while (0)
 #define QG_DECL() long long qg_stat_[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
@@ -71,13 +71,18 @@ struct Cfg {
     static constexpr int SR = SX;
     static constexpr int NACC = (BT > 192) ? 1 : 2;                // accumulators in tensor memory
     static constexpr int SA = ((512 - NACC * BT) / 32 >= 8) ? 8 : 4;   // dequantised-weight stages in tensor memory
+    // With a single accumulator the epilogue is exposed, so the dequantising warps share it (they would idle at the
+    // tile boundary); with two accumulators it overlaps the next main loop and the dequantising warps stay on theirs.
+    static constexpr bool HELP = (NACC == 1);
+    static constexpr int EPI_PARTS = HELP ? 5 : 1;                  // warps per TMEM lane quarter that drain a tile
     static constexpr int NSB = 3;                                  // scale buffers (one per 4 k-blocks)
     static constexpr int XH_ROWS = BT / 2;                         // token rows this CTA stages per k-block
     static constexpr int X_BYTES = XH_ROWS * 128;
     static constexpr int RAW_ROW = (QBITS == 8) ? 64 : 32;         // packed bytes per row per stage
     static constexpr int RAW_BYTES = BW * RAW_ROW;
     static constexpr int SC_BYTES = BW * 16;                       // 8 fp16 scales per row
-    static constexpr int STG_BYTES = 32 * 128 * 4;                 // epilogue staging: [32 tokens][128 rows] fp32 or 2 x bf16
+    static constexpr int STG_BYTES = 32 * 128 * 4 + 4 * 1024;      // [32 tokens][128 rows] fp32 (gate/up), also used as 16
+                                                                   // private 1 KB transposition buffers; + 4 more of those
     static constexpr int OFF_X = 0;
     static constexpr int OFF_RAW = OFF_X + SX * X_BYTES;
     static constexpr int OFF_SC = OFF_RAW + SR * RAW_BYTES;
@@ -193,6 +198,53 @@ __device__ __forceinline__ float lds_scale(uint32_t addr) {
     return __half2float(__ushort_as_half(h));
 }
 
+// Plain / routing-weighted epilogue of one warp: drains the 16-column (token) blocks b = pid, pid + npart, ... of
+// its 32 TMEM lanes (weight rows), rounds to bf16, transposes through a private [16 tokens][32 rows] buffer and
+// writes 16-byte pieces (64 contiguous bytes per token).  The next block's TMEM load is in flight while the current
+// one is processed.  Called by the four epilogue warps and by the sixteen dequantising warps, which would otherwise
+// idle at a tile boundary: a single warp retires only about one dependent instruction every few cycles, so the
+// drain time of a tile scales inversely with the number of warps that share it.
+__device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int tok_end, int n_base, uint32_t taddr,
+                                            int n_epi, int pid, int npart, __nv_bfloat16* st, int lane) {
+    __nv_bfloat16* outb = static_cast<__nv_bfloat16*>(p.out);
+    const int nblk = n_epi >> 4;
+    uint32_t v[16];
+    int b = pid;
+    if (b < nblk) tmem_ld_32x32_x16(taddr + 16 * b, v);
+    while (b < nblk) {
+        float wv = 1.0f;
+        if (p.mode == QG_MODE_DOWN_WEIGHTED) {
+            const int tokl = tok0 + 16 * b + (lane & 15);
+            wv = (tokl < tok_end) ? p.topk_w[p.row_pair[tokl]] : 0.f;
+        }
+        tmem_ld_wait();
+        uint32_t h[16];
+#pragma unroll
+        for (int jj = 0; jj < 16; ++jj) {
+            float val = __uint_as_float(v[jj]);
+            if (p.mode == QG_MODE_DOWN_WEIGHTED) val *= __shfl_sync(0xFFFFFFFFu, wv, jj);
+            h[jj] = __float_as_uint(val);
+        }
+        const int bn = b + npart;
+        if (bn < nblk) tmem_ld_32x32_x16(taddr + 16 * bn, v);      // next block, overlapped with the stores below
+#pragma unroll
+        for (int jj = 0; jj < 16; ++jj) st[jj * 32 + lane] = __float2bfloat16_rn(__uint_as_float(h[jj]));
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int piece = i * 32 + lane;
+            const int tk = piece >> 2, c4 = piece & 3;
+            const int tok = tok0 + 16 * b + tk;
+            const int n = n_base + c4 * 8;
+            if (tok < tok_end && n < p.N)
+                *reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * p.N + n) =
+                    *reinterpret_cast<const uint4*>(st + tk * 32 + c4 * 8);
+        }
+        __syncwarp();
+        b = bn;
+    }
+}
+
 template <int QBITS, int BT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
@@ -225,7 +277,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::SX; ++s) { mbar_init(full(s), 1 + 8); mbar_init(done(s), 1); }
         for (int s = 0; s < C::SR; ++s) { mbar_init(r_full(s), 1); mbar_init(r_empty(s), 4); }
-        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 2); mbar_init(acc_empty(s), 8); }
+        // an accumulator is released by the 4 epilogue + 16 dequantising warps of both CTAs
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 2); mbar_init(acc_empty(s), C::HELP ? 40 : 8); }
         misc[1] = 0;
         fence_mbar_init();
         fence_proxy_async_smem();
@@ -419,7 +472,34 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         const int my_tiles = (total_tiles > pair) ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
         const uint32_t n_own = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(nkb >> 2);
         QG_DECL();
-        for (uint32_t n = 0; n < n_own; ++n) {       // own k-block i = 4 n + g
+        // Helping with the epilogue.  Before this warp waits for the MMAs of own k-block n - 2 (to reuse their TMEM
+        // stage) it must have released every accumulator of an earlier tile, otherwise a single-accumulator pipeline
+        // would wait for itself; at that point it has filled the ring for the next tile and would idle anyway.
+        const uint32_t per_tile = static_cast<uint32_t>(nkb >> 2);     // own k-blocks per tile
+        uint32_t helped = 0;                                           // tiles whose accumulator this warp released
+        uint32_t t2 = 0, in2 = 0;                                      // tile of own k-block n - 2, position in it
+        const uint32_t acc_empty_leader = map_to_cta(acc_empty(0), 0);
+        const bool plain_ep = (p.mode == QG_MODE_PLAIN || p.mode == QG_MODE_DOWN_WEIGHTED);
+        __nv_bfloat16* my_st = stg16 + (warp - 8) * 512;               // private 1 KB transposition buffer
+        bool dq_ok = true;
+        auto help_tile = [&](uint32_t jt) -> bool {
+            const Tile tl = decode_tile(pair + static_cast<int>(jt) * n_pairs, prefix, p, BT);
+            const int wt = 2 * tl.pw + static_cast<int>(rank);
+            const uint32_t a = (C::NACC == 2) ? (jt & 1u) : 0u;
+            const uint32_t aph = (C::NACC == 2) ? ((jt >> 1) & 1u) : (jt & 1u);
+            if (!wait_bar<false>(acc_full(a), aph, abort_flag, p.status)) return false;
+            tc_fence_after_sync();
+            if (plain_ep && wt < p.n_wt) {
+                const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
+                drain_plain(p, tl.tok0, tl.tok_end, wt * BW + q * 32,
+                            tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BT, n_mma, 1 + g, 5, my_st, lane);
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8u * a);
+            return true;
+        };
+        for (uint32_t n = 0; n < n_own && dq_ok; ++n) {       // own k-block i = 4 n + g
             const uint32_t sr = ((n & 1u) << 2) + g;               // ring stage i % 8
             const uint32_t phr = (n >> 1) & 1u;                    // parity of (i / 8)
             QG_T0();
@@ -468,6 +548,13 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             __syncwarp();
             if (lane == 0) mbar_arrive(r_empty(sr));             // the packed codes are in registers now
             QG_ACC(7);
+            // (t2 = tile of own k-block n - 2.)  The release must come before the wait below, or the single-accumulator
+            // pipeline would wait for itself.
+            if (C::HELP && n >= 2) {
+                while (dq_ok && helped < t2) dq_ok = help_tile(helped++);
+                if (!dq_ok) break;
+                if (++in2 == per_tile) { in2 = 0; ++t2; }
+            }
             // its TMEM stage (i % SA) is free once the MMAs of k-block i - SA have completed
             if constexpr (C::SA == 8) {
                 if (n >= 2 && !wait_bar<false>(done(sr), (phr ^ 1u), abort_flag, p.status)) break;
@@ -495,6 +582,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             QG_ACC(7);
             if (warp == 8 && lane == 0) { QG_TRACE(7, 4 * n); }
         }
+        while (C::HELP && dq_ok && helped < static_cast<uint32_t>(my_tiles)) dq_ok = help_tile(helped++);
         __syncwarp();
         if (warp == 8 && lane == 0) QG_FLUSH();
     } else if (warp >= 4) {
@@ -523,10 +611,16 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + a * BT;
             const int n_epi = (wt < p.n_wt) ? n_mma : 0;
 #ifdef QG_PROFILE
-            const int n_epi2 = (p.dbg & 2) ? 0 : n_epi;
+            int n_epi2 = (p.dbg & 2) ? 0 : n_epi;
 #else
-            const int n_epi2 = n_epi;
+            int n_epi2 = n_epi;
 #endif
+            if (p.mode == QG_MODE_PLAIN || p.mode == QG_MODE_DOWN_WEIGHTED) {
+                // shared with the dequantising warps (participants 1..4 of this lane quarter)
+                drain_plain(p, tl.tok0, tl.tok_end, wt * BW + qd * 32, taddr, n_epi2, 0, C::EPI_PARTS,
+                            stg16 + (16 + qd) * 512, lane);
+                n_epi2 = 0;     // done; the loop below serves the other two modes
+            }
             for (int c = 0; c < n_epi2; c += 32, ++cc) {
                 uint32_t v[32];
                 tmem_ld_32x32(taddr + c, v);
