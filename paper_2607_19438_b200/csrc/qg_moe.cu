@@ -26,19 +26,20 @@ __device__ __forceinline__ bool route_before(float a, int ia, float b, int ib) {
 // One warp per token (each warp walks ROUTE_TOKENS_PER_BLOCK / ROUTE_WARPS tokens).  Lane l owns the
 // logits e = l, l+32, ...; k rounds of (local best, warp arg-best by shuffles, mark taken).
 // Dynamic shared memory: per warp E floats (logits) + k floats (selected logits); then E ints (hist).
-__global__ void __launch_bounds__(ROUTE_WARPS * 32)
+__global__ void __launch_bounds__(1024)
 route_topk_kernel(int M, int E, int k, const float* __restrict__ logits, int32_t* __restrict__ topk_idx,
                   float* __restrict__ topk_w, int32_t* __restrict__ block_hist) {
     extern __shared__ float sm[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nwarps = blockDim.x >> 5;          // 32 (one token per warp) unless E is large, then 8
     float* lg = sm + warp * (E + k);
     float* sel = lg + E;
-    int* hist = reinterpret_cast<int*>(sm + ROUTE_WARPS * (E + k));
+    int* hist = reinterpret_cast<int*>(sm + nwarps * (E + k));
     for (int e = threadIdx.x; e < E; e += blockDim.x) hist[e] = 0;
     __syncthreads();
 
     const int t0 = blockIdx.x * ROUTE_TOKENS_PER_BLOCK;
-    for (int tt = warp; tt < ROUTE_TOKENS_PER_BLOCK; tt += ROUTE_WARPS) {
+    for (int tt = warp; tt < ROUTE_TOKENS_PER_BLOCK; tt += nwarps) {
         const int t = t0 + tt;
         if (t >= M) break;
         const float* row = logits + static_cast<size_t>(t) * E;
@@ -276,7 +277,9 @@ int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* to
         }
         return QG_OK;
     }
-    const size_t sm_topk = (static_cast<size_t>(qg::ROUTE_WARPS) * (E + k) + E) * sizeof(float);
+    // one token per warp when 32 warps' rows fit in 64 KB of shared memory, else 8 warps take 4 tokens each
+    const int topk_warps = (32 * static_cast<size_t>(E + k) * sizeof(float) <= 64 * 1024) ? 32 : qg::ROUTE_WARPS;
+    const size_t sm_topk = (static_cast<size_t>(topk_warps) * (E + k) + E) * sizeof(float);
     if (sm_topk > 48 * 1024) {
         if (cudaFuncSetAttribute(qg::route_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(sm_topk)) != cudaSuccess) {
@@ -284,7 +287,7 @@ int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* to
             return QG_ERR_CUDA;
         }
     }
-    qg::route_topk_kernel<<<nb, qg::ROUTE_WARPS * 32, sm_topk, st>>>(M, E, k, logits, topk_idx, topk_w, hist);
+    qg::route_topk_kernel<<<nb, topk_warps * 32, sm_topk, st>>>(M, E, k, logits, topk_idx, topk_w, hist);
     qg::route_scan_kernel<<<1, 1024, 0, st>>>(nb, E, hist, expert_counts, expert_offsets);
     qg::route_scatter_kernel<<<nb, qg::ROUTE_WARPS * 32, E * sizeof(int), st>>>(M, E, k, topk_idx, expert_offsets, hist,
                                                                                row_pair, pair_row);
@@ -333,7 +336,9 @@ int moe_route_static(qg_ctx* ctx, int M, int E, int k, const float* logits, int3
         }
         return QG_OK;
     }
-    const size_t sm_topk = (static_cast<size_t>(qg::ROUTE_WARPS) * (E + k) + E) * sizeof(float);
+    // one token per warp when 32 warps' rows fit in 64 KB of shared memory, else 8 warps take 4 tokens each
+    const int topk_warps = (32 * static_cast<size_t>(E + k) * sizeof(float) <= 64 * 1024) ? 32 : qg::ROUTE_WARPS;
+    const size_t sm_topk = (static_cast<size_t>(topk_warps) * (E + k) + E) * sizeof(float);
     if (sm_topk > 48 * 1024) {
         if (cudaFuncSetAttribute(qg::route_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(sm_topk)) != cudaSuccess) {
@@ -344,7 +349,7 @@ int moe_route_static(qg_ctx* ctx, int M, int E, int k, const float* logits, int3
     // every entry hist[b, e] that the scan and the scatter read is written by the first kernel of this call, so
     // whatever an earlier call left in the shared array does not matter
     const int nbi = static_cast<int>(nb);
-    qg::route_topk_kernel<<<nbi, qg::ROUTE_WARPS * 32, sm_topk, st>>>(M, E, k, logits, topk_idx, topk_w, hist);
+    qg::route_topk_kernel<<<nbi, topk_warps * 32, sm_topk, st>>>(M, E, k, logits, topk_idx, topk_w, hist);
     qg::route_scan_kernel<<<1, 1024, 0, st>>>(nbi, E, hist, expert_counts, expert_offsets);
     qg::route_scatter_kernel<<<nbi, qg::ROUTE_WARPS * 32, E * sizeof(int), st>>>(M, E, k, topk_idx, expert_offsets, hist,
                                                                                 row_pair, pair_row);

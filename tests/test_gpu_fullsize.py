@@ -1,0 +1,84 @@
+"""GPU parity at the benchmark's full sizes, in the launch configurations bench.py times, on sampled outputs the oracle
+can compute one by one (dense) or on whole expert segments (MoE)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2607_19438_b200 import binding as qg, synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+
+def _sampled_dense(qbits, M, N, K, seed, per_tile=2, tile=128):
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=seed)
+    out = qg.qgemm_dense(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws))
+    qg.poll_status()
+    out = util.host_bf16_f64(out)
+    rng = np.random.default_rng(seed)
+    rows, cols = [], []
+    for rt in range((M + tile - 1) // tile):
+        for ct in range((N + tile - 1) // tile):
+            rows.append(np.minimum(rt * tile + rng.integers(0, tile, per_tile), M - 1))
+            cols.append(np.minimum(ct * tile + rng.integers(0, tile, per_tile), N - 1))
+    # plus the last row / column (ragged edges) and the first ones
+    rows.append(np.array([0, M - 1, M - 1, 0])); cols.append(np.array([0, N - 1, 0, N - 1]))
+    rows = np.concatenate(rows); cols = np.concatenate(cols)
+    ref = orc.qgemm_dense_sample(qbits, A, Wq, Ws, rows, cols)
+    assert np.all(np.isfinite(out))
+    return util.assert_close(out[rows, cols], ref, f"q{qbits} {M}x{N}x{K}")
+
+
+# config 1 (2B-class Q8), config 2 (Llama-3.2-3B-shaped Q4), config 4 (8B-class Q8): one GEMM of each kind
+FULL = [
+    (8, 2048, 2560, 2048), (8, 2048, 2048, 8192), (8, 1024, 16384, 2048), (8, 1000, 2048, 2048),
+    (4, 2048, 5120, 3072), (4, 2048, 3072, 8192), (4, 512, 16384, 3072),
+    (8, 2048, 6144, 4096), (8, 4096, 4096, 14336), (8, 8192, 4096, 4096),
+]
+
+
+@pytest.mark.parametrize("qbits,M,N,K", FULL, ids=[f"q{c[0]}-{c[1]}x{c[2]}x{c[3]}" for c in FULL])
+def test_dense_full_size_sampled(qbits, M, N, K):
+    _sampled_dense(qbits, M, N, K, seed=0, per_tile=1 if M * N > 2 ** 24 else 2)
+
+
+@pytest.mark.parametrize("M,skewed", [(2048, False), (2048, True), (1024, False)], ids=["uniform-2048", "skewed-2048", "uniform-1024"])
+def test_moe_config3_full_size_selected_experts(M, skewed):
+    """Config 3 (H=2048, E=128, top-8, F=768, Q4) at the bench's token counts.  Routing and permutation are compared in
+    full (bit exact); the two GEMM stages are compared on every row of a few experts (the busiest, the least busy and
+    two others), each stage fed with exactly what the GPU stage consumed; the layer output is then checked through
+    the combine stage on the GPU's own weighted rows."""
+    qbits, H, E, F, k = 4, 2048, 128, 768, 8
+    logits, X, W1q, W1s, W2q, W2s = synth.moe_problem(qbits, M, H, E, F, seed=0, skewed=skewed)
+    d = dict(logits=util.dev(logits), X=util.dev_bf16(X), W1q=util.dev(W1q), W1s=util.dev_f16(W1s),
+             W2q=util.dev(W2q), W2s=util.dev_f16(W2s))
+    r = qg.moe_route(d["logits"], k, X=d["X"])
+    Hh = qg.moe_grouped_qgemm(qg.MODE_GATE_UP_SILU, qbits, r["Xperm"], r["offsets"], d["W1q"], d["W1s"])
+    Dw = qg.moe_grouped_qgemm(qg.MODE_DOWN_WEIGHTED, qbits, Hh, r["offsets"], d["W2q"], d["W2s"],
+                              topk_w=r["topk_w"].view(-1), row_pair=r["row_pair"], k=k)
+    y = qg.moe_combine(Dw, r["pair_row"], k)
+    qg.poll_status()
+    idx, w, _ = orc.route(logits, k)
+    counts, offsets = orc.counts_offsets(idx, E)
+    row_pair, pair_row = orc.permutation(idx, offsets)
+    assert np.array_equal(r["topk_idx"].cpu().numpy(), idx)
+    assert np.array_equal(r["offsets"].cpu().numpy(), offsets)
+    assert np.array_equal(r["row_pair"].cpu().numpy(), row_pair)
+    assert np.array_equal(r["pair_row"].cpu().numpy(), pair_row)
+    Xp = orc.permute(X, row_pair, k)
+    assert np.array_equal(util.host_bf16_bits(r["Xperm"]), Xp)
+    Hh_g = util.host_bf16_f64(Hh); Dw_g = util.host_bf16_f64(Dw)
+    w_gpu = r["topk_w"].cpu().numpy().astype(np.float64).reshape(-1)
+    experts = sorted({int(np.argmax(counts)), int(np.argmin(counts)), 5, 64})
+    for e in experts:
+        seg = slice(int(offsets[e]), int(offsets[e + 1]))
+        if seg.stop == seg.start:
+            continue
+        off1 = np.array([0, seg.stop - seg.start], np.int32)
+        GU = orc.grouped_gemm(qbits, orc.bf16_to_f64(Xp[seg]), off1, W1q[e:e + 1], W1s[e:e + 1])
+        util.assert_close(Hh_g[seg], orc.silu_mul(GU), f"gate/up expert {e}")
+        Dn = orc.grouped_gemm(qbits, Hh_g[seg], off1, W2q[e:e + 1], W2s[e:e + 1])
+        util.assert_close(Dw_g[seg], Dn * w_gpu[row_pair[seg]][:, None], f"down expert {e}")
+    util.assert_close(util.host_bf16_f64(y), orc.combine(Dw_g, pair_row, k), "combine")
+    assert np.all(np.isfinite(util.host_bf16_f64(y)))
