@@ -147,39 +147,68 @@ __device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&b);
 }
 
+// Two fp32 fused multiply-adds in one instruction (fma.rn.f32x2, each lane IEEE-exact as fmaf) followed by the
+// packed round-to-nearest-even conversion to bf16x2: returns bf16(a0 * m.lo + c.lo) | bf16(a1 * m.hi + c.hi) << 16.
+// One issue slot per two weights instead of two.
+__device__ __forceinline__ uint32_t fma2_bf16x2(uint32_t a0, uint32_t a1, uint64_t m, uint64_t c) {
+    uint32_t r;
+    asm("{\n\t.reg .b64 t;\n\t.reg .b32 lo, hi;\n\t"
+        "mov.b64 t, {%1, %2};\n\t"
+        "fma.rn.f32x2 t, t, %3, %4;\n\t"
+        "mov.b64 {lo, hi}, t;\n\t"
+        "cvt.rn.bf16x2.f32 %0, hi, lo;\n\t}"
+        : "=r"(r) : "r"(a0), "r"(a1), "l"(m), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    return static_cast<uint64_t>(__float_as_uint(lo)) | (static_cast<uint64_t>(__float_as_uint(hi)) << 32);
+}
+
 // 4 int8 codes (one 32-bit word) -> 4 bf16 = q * scale, exact product rounded once.
 // The byte u = q + 128 is dropped into a float's mantissa: 0x4300uu00 = 128 + u/256, so
 // q * s = fma(f, 256 s, -32896 s); both constants and the result are exact in fp32.
-__device__ __forceinline__ void dq8_word(uint32_t x, float s256, float c, uint32_t& o0, uint32_t& o1) {
+// m2 = {256 s, 256 s}, c2 = {-32896 s, -32896 s}.
+__device__ __forceinline__ void dq8_word(uint32_t x, uint64_t m2, uint64_t c2, uint32_t& o0, uint32_t& o1) {
     x ^= 0x80808080u;
-    const float f0 = __uint_as_float(__byte_perm(x, 0x43000000u, 0x7604));
-    const float f1 = __uint_as_float(__byte_perm(x, 0x43000000u, 0x7614));
-    const float f2 = __uint_as_float(__byte_perm(x, 0x43000000u, 0x7624));
-    const float f3 = __uint_as_float(__byte_perm(x, 0x43000000u, 0x7634));
-    o0 = bf16x2(fmaf(f0, s256, c), fmaf(f1, s256, c));
-    o1 = bf16x2(fmaf(f2, s256, c), fmaf(f3, s256, c));
+    const uint32_t f0 = __byte_perm(x, 0x43000000u, 0x7604);
+    const uint32_t f1 = __byte_perm(x, 0x43000000u, 0x7614);
+    const uint32_t f2 = __byte_perm(x, 0x43000000u, 0x7624);
+    const uint32_t f3 = __byte_perm(x, 0x43000000u, 0x7634);
+    o0 = fma2_bf16x2(f0, f1, m2, c2);
+    o1 = fma2_bf16x2(f2, f3, m2, c2);
 }
 
-// 8 4-bit codes (one word, nibble i = weight i, code u = q + 8) -> 8 bf16.  A nibble at bit p of
-// 0x43000000 reads 128 + u 2^(p-16); for p in {8, 12, 16}: q s = fma(f, s 2^(16-p), -(2^(23-p) + 8) s),
-// again exact in fp32.
-__device__ __forceinline__ void dq4_word(uint32_t x, float s, uint32_t (&o)[4]) {
+// Constants of the 4-bit conversion for one scale s.  A nibble at bit p of 0x43000000 reads 128 + u 2^(p-16); for
+// p in {8, 12, 16}: q s = fma(f, s 2^(16-p), -(2^(23-p) + 8) s), exact in fp32.  The eight nibbles of a word sit at
+// p = 8, 12 (after << 8), 8, 12, 16 (in place), 8, 12, 16 (after >> 12); the pairs below follow that order.
+struct Dq4Consts {
+    uint64_t m_8_12, c_8_12, m_16_8, c_16_8, m_12_16, c_12_16;
+};
+__device__ __forceinline__ Dq4Consts dq4_consts(float s) {
     const float m8 = 256.f * s, c8 = -32776.f * s;
     const float m12 = 16.f * s, c12 = -2056.f * s;
     const float m16 = s, c16 = -136.f * s;
+    Dq4Consts k;
+    k.m_8_12 = pack_f32x2(m8, m12);   k.c_8_12 = pack_f32x2(c8, c12);
+    k.m_16_8 = pack_f32x2(m16, m8);   k.c_16_8 = pack_f32x2(c16, c8);
+    k.m_12_16 = pack_f32x2(m12, m16); k.c_12_16 = pack_f32x2(c12, c16);
+    return k;
+}
+// 8 4-bit codes (one word, nibble i = weight i, code u = q + 8) -> 8 bf16.
+__device__ __forceinline__ void dq4_word(uint32_t x, const Dq4Consts& k, uint32_t (&o)[4]) {
     const uint32_t y = x << 8, z = x >> 12;
-    const float f0 = __uint_as_float((y & 0x00000F00u) | 0x43000000u);
-    const float f1 = __uint_as_float((y & 0x0000F000u) | 0x43000000u);
-    const float f2 = __uint_as_float((x & 0x00000F00u) | 0x43000000u);
-    const float f3 = __uint_as_float((x & 0x0000F000u) | 0x43000000u);
-    const float f4 = __uint_as_float((x & 0x000F0000u) | 0x43000000u);
-    const float f5 = __uint_as_float((z & 0x00000F00u) | 0x43000000u);
-    const float f6 = __uint_as_float((z & 0x0000F000u) | 0x43000000u);
-    const float f7 = __uint_as_float((z & 0x000F0000u) | 0x43000000u);
-    o[0] = bf16x2(fmaf(f0, m8, c8), fmaf(f1, m12, c12));
-    o[1] = bf16x2(fmaf(f2, m8, c8), fmaf(f3, m12, c12));
-    o[2] = bf16x2(fmaf(f4, m16, c16), fmaf(f5, m8, c8));
-    o[3] = bf16x2(fmaf(f6, m12, c12), fmaf(f7, m16, c16));
+    const uint32_t f0 = (y & 0x00000F00u) | 0x43000000u;
+    const uint32_t f1 = (y & 0x0000F000u) | 0x43000000u;
+    const uint32_t f2 = (x & 0x00000F00u) | 0x43000000u;
+    const uint32_t f3 = (x & 0x0000F000u) | 0x43000000u;
+    const uint32_t f4 = (x & 0x000F0000u) | 0x43000000u;
+    const uint32_t f5 = (z & 0x00000F00u) | 0x43000000u;
+    const uint32_t f6 = (z & 0x0000F000u) | 0x43000000u;
+    const uint32_t f7 = (z & 0x000F0000u) | 0x43000000u;
+    o[0] = fma2_bf16x2(f0, f1, k.m_8_12, k.c_8_12);
+    o[1] = fma2_bf16x2(f2, f3, k.m_8_12, k.c_8_12);
+    o[2] = fma2_bf16x2(f4, f5, k.m_16_8, k.c_16_8);
+    o[3] = fma2_bf16x2(f6, f7, k.m_12_16, k.c_12_16);
 }
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
@@ -211,11 +240,24 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
     uint32_t v[16];
     int b = pid;
     if (b < nblk) tmem_ld_32x32_x16(taddr + 16 * b, v);
+    // Routing weights of the whole tile, fetched once (two dependent global loads, all in flight together): lane l
+    // holds the weights of tokens l, l + 32, ... of the tile.
+    float wt8[8];
+    if (p.mode == QG_MODE_DOWN_WEIGHTED) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int tokl = tok0 + 32 * j + lane;
+            wt8[j] = (32 * j < n_epi && tokl < tok_end) ? p.topk_w[p.row_pair[tokl]] : 0.f;
+        }
+    }
     while (b < nblk) {
         float wv = 1.0f;
         if (p.mode == QG_MODE_DOWN_WEIGHTED) {
-            const int tokl = tok0 + 16 * b + (lane & 15);
-            wv = (tokl < tok_end) ? p.topk_w[p.row_pair[tokl]] : 0.f;
+            const int j = b >> 1;        // tokens 16 b .. 16 b + 15 live in register j, lanes 16 (b & 1) ..
+            wv = wt8[0];
+#pragma unroll
+            for (int jj = 1; jj < 8; ++jj) wv = (j == jj) ? wt8[jj] : wv;
+            wv = __shfl_sync(0xFFFFFFFFu, wv, 16 * (b & 1) + (lane & 15));
         }
         tmem_ld_wait();
         uint32_t h[16];
@@ -245,7 +287,9 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
     }
 }
 
-template <int QBITS, int BT>
+// EPI: 0 plain / routing-weighted bf16 store, 1 gate/up + SiLU, 2 weighted fp32 atomic accumulate (compiled apart so
+// that each instantiation carries one epilogue only).
+template <int QBITS, int BT, int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const __grid_constant__ CUtensorMap tm_s, const GemmParams p) {
@@ -316,7 +360,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     const uint32_t tmem_base = static_cast<uint32_t>(misc[0]);
     const int total_tiles = prefix[p.E];
     const int nkb = p.K / BK;     // a multiple of 4
-    const bool gate_up = (p.mode == QG_MODE_GATE_UP_SILU);
+    constexpr bool gate_up = (EPI == 1);
 
     // Control warps walk their loops with all 32 lanes (converged) and keep the per-k-block instruction count small:
     // a lone thread retires only one dependent instruction every few cycles and an mbarrier round trip costs a few
@@ -479,7 +523,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         uint32_t helped = 0;                                           // tiles whose accumulator this warp released
         uint32_t t2 = 0, in2 = 0;                                      // tile of own k-block n - 2, position in it
         const uint32_t acc_empty_leader = map_to_cta(acc_empty(0), 0);
-        const bool plain_ep = (p.mode == QG_MODE_PLAIN || p.mode == QG_MODE_DOWN_WEIGHTED);
+        constexpr bool plain_ep = (EPI == 0);
         __nv_bfloat16* my_st = stg16 + (warp - 8) * 512;               // private 1 KB transposition buffer
         bool dq_ok = true;
         auto help_tile = [&](uint32_t jt) -> bool {
@@ -528,21 +572,23 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     const uint4 v0 = lds128(raw + (((2 * h) ^ swz) << 4));
                     const uint4 v1 = lds128(raw + (((2 * h + 1) ^ swz) << 4));
                     const float s256 = 256.f * sc, c = -32896.f * sc;
-                    dq8_word(v0.x, s256, c, oh[0], oh[1]);
-                    dq8_word(v0.y, s256, c, oh[2], oh[3]);
-                    dq8_word(v0.z, s256, c, oh[4], oh[5]);
-                    dq8_word(v0.w, s256, c, oh[6], oh[7]);
-                    dq8_word(v1.x, s256, c, oh[8], oh[9]);
-                    dq8_word(v1.y, s256, c, oh[10], oh[11]);
-                    dq8_word(v1.z, s256, c, oh[12], oh[13]);
-                    dq8_word(v1.w, s256, c, oh[14], oh[15]);
+                    const uint64_t m2 = pack_f32x2(s256, s256), c2 = pack_f32x2(c, c);
+                    dq8_word(v0.x, m2, c2, oh[0], oh[1]);
+                    dq8_word(v0.y, m2, c2, oh[2], oh[3]);
+                    dq8_word(v0.z, m2, c2, oh[4], oh[5]);
+                    dq8_word(v0.w, m2, c2, oh[6], oh[7]);
+                    dq8_word(v1.x, m2, c2, oh[8], oh[9]);
+                    dq8_word(v1.y, m2, c2, oh[10], oh[11]);
+                    dq8_word(v1.z, m2, c2, oh[12], oh[13]);
+                    dq8_word(v1.w, m2, c2, oh[14], oh[15]);
                 } else {
                     const uint4 v = lds128(raw + ((h ^ swz) << 4));
                     uint32_t w4[4];
-                    dq4_word(v.x, sc, w4); oh[0] = w4[0]; oh[1] = w4[1]; oh[2] = w4[2]; oh[3] = w4[3];
-                    dq4_word(v.y, sc, w4); oh[4] = w4[0]; oh[5] = w4[1]; oh[6] = w4[2]; oh[7] = w4[3];
-                    dq4_word(v.z, sc, w4); oh[8] = w4[0]; oh[9] = w4[1]; oh[10] = w4[2]; oh[11] = w4[3];
-                    dq4_word(v.w, sc, w4); oh[12] = w4[0]; oh[13] = w4[1]; oh[14] = w4[2]; oh[15] = w4[3];
+                    const Dq4Consts kc = dq4_consts(sc);
+                    dq4_word(v.x, kc, w4); oh[0] = w4[0]; oh[1] = w4[1]; oh[2] = w4[2]; oh[3] = w4[3];
+                    dq4_word(v.y, kc, w4); oh[4] = w4[0]; oh[5] = w4[1]; oh[6] = w4[2]; oh[7] = w4[3];
+                    dq4_word(v.z, kc, w4); oh[8] = w4[0]; oh[9] = w4[1]; oh[10] = w4[2]; oh[11] = w4[3];
+                    dq4_word(v.w, kc, w4); oh[12] = w4[0]; oh[13] = w4[1]; oh[14] = w4[2]; oh[15] = w4[3];
                 }
             }
             __syncwarp();
@@ -592,7 +638,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         __nv_bfloat16* outb = static_cast<__nv_bfloat16*>(p.out);
         float* outf = static_cast<float*>(p.out);
         const uint32_t acc_empty_base = map_to_cta(acc_empty(0), 0);
-        uint32_t j = 0, cc = 0;
+        uint32_t j = 0;
         QG_DECL();
         for (int t = pair; t < total_tiles; t += n_pairs, ++j) {
             const Tile tl = decode_tile(t, prefix, p, BT);
@@ -615,88 +661,62 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
 #else
             int n_epi2 = n_epi;
 #endif
-            if (p.mode == QG_MODE_PLAIN || p.mode == QG_MODE_DOWN_WEIGHTED) {
-                // shared with the dequantising warps (participants 1..4 of this lane quarter)
+            if constexpr (EPI == 0) {
+                // shared with the dequantising warps (participants 1..4 of this lane quarter) when they help
                 drain_plain(p, tl.tok0, tl.tok_end, wt * BW + qd * 32, taddr, n_epi2, 0, C::EPI_PARTS,
                             stg16 + (16 + qd) * 512, lane);
-                n_epi2 = 0;     // done; the loop below serves the other two modes
-            }
-            for (int c = 0; c < n_epi2; c += 32, ++cc) {
-                uint32_t v[32];
-                tmem_ld_32x32(taddr + c, v);
-                tmem_ld_wait();
-                const int row = qd * 32 + lane;          // weight row of this thread inside the tile
-                if (p.mode == QG_MODE_DOWN_ACCUM_F32) {
-                    // y[token, n] += w * acc: lanes are consecutive n, so each warp-wide red covers 128 bytes
-                    const int n = wt * BW + row;
-                    const int tokl = tl.tok0 + c + lane;
-                    int trow = 0;
-                    float wv = 0.f;
-                    if (tokl < tl.tok_end) {
-                        const int pr = p.row_pair[tokl];
-                        wv = p.topk_w[pr];
-                        trow = pr / p.k;
-                    }
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        const float w = __shfl_sync(0xFFFFFFFFu, wv, jj);
-                        const int tr = __shfl_sync(0xFFFFFFFFu, trow, jj);
-                        if (tl.tok0 + c + jj < tl.tok_end && n < p.N)
-                            atomicAdd(outf + static_cast<size_t>(tr) * p.N + n, w * __uint_as_float(v[jj]));
-                    }
-                } else if (gate_up) {
-                    // lanes 0..63 hold gate rows, 64..127 the matching up rows: transpose through shared memory
-                    // ([32 tokens][128 rows] fp32), then every thread finishes 16 outputs of one token.
-                    const int F = p.N / 2;
-#pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) stg32[jj * 128 + row] = __uint_as_float(v[jj]);
-                    named_bar_sync(2, 128);
-                    const int tk = et >> 2, f0 = (et & 3) * 16;
-                    const int tok = tl.tok0 + c + tk;
-                    const float4* g4 = reinterpret_cast<const float4*>(stg32 + tk * 128 + f0);
-                    const float4* u4 = reinterpret_cast<const float4*>(stg32 + tk * 128 + 64 + f0);
-                    uint32_t o[8];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float4 g = g4[i], u = u4[i];
-                        const float h0 = __fdividef(g.x, 1.0f + __expf(-g.x)) * u.x;
-                        const float h1 = __fdividef(g.y, 1.0f + __expf(-g.y)) * u.y;
-                        const float h2 = __fdividef(g.z, 1.0f + __expf(-g.z)) * u.z;
-                        const float h3 = __fdividef(g.w, 1.0f + __expf(-g.w)) * u.w;
-                        o[2 * i] = bf16x2(h0, h1);
-                        o[2 * i + 1] = bf16x2(h2, h3);
-                    }
-                    if (tok < tl.tok_end) {
-                        uint4* dst = reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * F + wt * 64 + f0);
-                        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
-                    }
-                    named_bar_sync(2, 128);
-                } else {
-                    // bf16 [32 tokens][128 rows] staging (two buffers, one barrier per chunk), then 16-byte stores
-                    // that cover 256 contiguous bytes per token.
-                    float wv = 1.0f;
-                    if (p.mode == QG_MODE_DOWN_WEIGHTED) {
+            } else {
+                for (int c = 0; c < n_epi2; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(taddr + c, v);
+                    tmem_ld_wait();
+                    const int row = qd * 32 + lane;          // weight row of this thread inside the tile
+                    if constexpr (EPI == 2) {
+                        // y[token, n] += w * acc: lanes are consecutive n, so each warp-wide red covers 128 bytes
+                        const int n = wt * BW + row;
                         const int tokl = tl.tok0 + c + lane;
-                        wv = (tokl < tl.tok_end) ? p.topk_w[p.row_pair[tokl]] : 0.f;
-                    }
-                    __nv_bfloat16* st = stg16 + (cc & 1u) * 4096;
+                        int trow = 0;
+                        float wv = 0.f;
+                        if (tokl < tl.tok_end) {
+                            const int pr = p.row_pair[tokl];
+                            wv = p.topk_w[pr];
+                            trow = pr / p.k;
+                        }
 #pragma unroll
-                    for (int jj = 0; jj < 32; ++jj) {
-                        float val = __uint_as_float(v[jj]);
-                        if (p.mode == QG_MODE_DOWN_WEIGHTED) val *= __shfl_sync(0xFFFFFFFFu, wv, jj);
-                        st[jj * 128 + row] = __float2bfloat16_rn(val);
-                    }
-                    named_bar_sync(2, 128);
+                        for (int jj = 0; jj < 32; ++jj) {
+                            const float w = __shfl_sync(0xFFFFFFFFu, wv, jj);
+                            const int tr = __shfl_sync(0xFFFFFFFFu, trow, jj);
+                            if (tl.tok0 + c + jj < tl.tok_end && n < p.N)
+                                atomicAdd(outf + static_cast<size_t>(tr) * p.N + n, w * __uint_as_float(v[jj]));
+                        }
+                    } else {
+                        // lanes 0..63 hold gate rows, 64..127 the matching up rows: transpose through shared memory
+                        // ([32 tokens][128 rows] fp32), then every thread finishes 16 outputs of one token.
+                        const int F = p.N / 2;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int piece = i * 128 + et;
-                        const int tk = piece >> 4, c16 = piece & 15;
+                        for (int jj = 0; jj < 32; ++jj) stg32[jj * 128 + row] = __uint_as_float(v[jj]);
+                        named_bar_sync(2, 128);
+                        const int tk = et >> 2, f0 = (et & 3) * 16;
                         const int tok = tl.tok0 + c + tk;
-                        const int n = wt * BW + c16 * 8;
-                        if (tok < tl.tok_end && n < p.N)
-                            *reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * p.N + n) =
-                                *reinterpret_cast<const uint4*>(st + tk * 128 + c16 * 8);
+                        const float4* g4 = reinterpret_cast<const float4*>(stg32 + tk * 128 + f0);
+                        const float4* u4 = reinterpret_cast<const float4*>(stg32 + tk * 128 + 64 + f0);
+                        uint32_t o[8];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float4 g = g4[i], u = u4[i];
+                            const float h0 = __fdividef(g.x, 1.0f + __expf(-g.x)) * u.x;
+                            const float h1 = __fdividef(g.y, 1.0f + __expf(-g.y)) * u.y;
+                            const float h2 = __fdividef(g.z, 1.0f + __expf(-g.z)) * u.z;
+                            const float h3 = __fdividef(g.w, 1.0f + __expf(-g.w)) * u.w;
+                            o[2 * i] = bf16x2(h0, h1);
+                            o[2 * i + 1] = bf16x2(h2, h3);
+                        }
+                        if (tok < tl.tok_end) {
+                            uint4* dst = reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * F + wt * 64 + f0);
+                            dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                            dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                        }
+                        named_bar_sync(2, 128);
                     }
                 }
             }
@@ -720,7 +740,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     if (warp == 3) tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
 }
 
-template <int QBITS, int BT>
+template <int QBITS, int BT, int EPI>
 static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const void* Wq, const void* Ws,
                        cudaStream_t st) {
     using C = Cfg<QBITS, BT>;
@@ -736,7 +756,7 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const vo
         rc = make_tmap_2d(ctx, &tm_s, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, Ws, p.K / 32, wrows, 8, 64,
                           CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc != QG_OK) return rc;
-    auto kern = qgemm_kernel<QBITS, BT>;
+    auto kern = qgemm_kernel<QBITS, BT, EPI>;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
@@ -788,14 +808,22 @@ static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in,
     p.stats = g_stats;
     if (const char* d = getenv("QG_DBG")) p.dbg = atoi(d);
 #endif
+    const int epi = (p.mode == QG_MODE_GATE_UP_SILU) ? 1 : (p.mode == QG_MODE_DOWN_ACCUM_F32) ? 2 : 0;
+#define QG_LAUNCH(Q, B)                                                                 \
+    do {                                                                                \
+        if (epi == 0) return launch_gemm<Q, B, 0>(ctx, p, X, Wq, Ws, st);               \
+        if (epi == 1) return launch_gemm<Q, B, 1>(ctx, p, X, Wq, Ws, st);               \
+        return launch_gemm<Q, B, 2>(ctx, p, X, Wq, Ws, st);                             \
+    } while (0)
     if (qbits == QG_Q8) {
-        if (bt == 256) return launch_gemm<8, 256>(ctx, p, X, Wq, Ws, st);
-        if (bt == 192) return launch_gemm<8, 192>(ctx, p, X, Wq, Ws, st);
-        return launch_gemm<8, 128>(ctx, p, X, Wq, Ws, st);
+        if (bt == 256) QG_LAUNCH(8, 256);
+        if (bt == 192) QG_LAUNCH(8, 192);
+        QG_LAUNCH(8, 128);
     }
-    if (bt == 256) return launch_gemm<4, 256>(ctx, p, X, Wq, Ws, st);
-    if (bt == 192) return launch_gemm<4, 192>(ctx, p, X, Wq, Ws, st);
-    return launch_gemm<4, 128>(ctx, p, X, Wq, Ws, st);
+    if (bt == 256) QG_LAUNCH(4, 256);
+    if (bt == 192) QG_LAUNCH(4, 192);
+    QG_LAUNCH(4, 128);
+#undef QG_LAUNCH
 }
 
 }  // namespace qg
