@@ -94,10 +94,12 @@ def run_reference(args):
     from oracle import oracle as orc
     dense, moe = host_inputs(M_TOKENS, seed=0)
     # calibrate on a tiny sample, then size a step so that the whole run stays within a few minutes
-    t = time.perf_counter(); fl = oracle_sample_step(dense, moe, 2, 2); rate = fl / (time.perf_counter() - t)
-    budget = min(3.0, 150.0 / max(1, args.steps + args.warmup))
+    # (the oracle parallelises over rows, so the sample has at least as many rows as threads)
+    nthr = orc.num_threads()
+    t = time.perf_counter(); fl = oracle_sample_step(dense, moe, nthr, nthr); rate = fl / (time.perf_counter() - t)
+    budget = min(6.0, 150.0 / max(1, args.steps + args.warmup))
     per_tok = dense_flops(1) + moe_flops(1)
-    m = int(max(1, min(128, rate * budget / per_tok)))
+    m = int(max(nthr, min(128, rate * budget / per_tok)))
     for _ in range(args.warmup):
         oracle_sample_step(dense, moe, m, m)
     t0 = time.perf_counter()
@@ -351,7 +353,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()

@@ -5,12 +5,13 @@
 //
 // Mapping onto the tensor cores.  The weight rows are the UMMA "M" side and the tokens the "N" side.  Two CTAs
 // on neighbouring SMs form a pair (cluster of 2, tcgen05 cta_group::2): the pair's tile is 256 weight rows x BT
-// tokens (BT = 128 or 192).  Each CTA dequantises its own 128 weight rows straight into tensor memory, where the
-// MMA reads them as its A operand, and stages half of the token tile in shared memory as its half of the B
+// tokens (BT = 128, 192 or 256).  Each CTA dequantises its own 128 weight rows straight into tensor memory, where
+// the MMA reads them as its A operand, and stages half of the token tile in shared memory as its half of the B
 // operand, so per SM only half of the activation bytes cross L2 -> SM and shared memory.
 //
-// Persistent CTA of 24 warps, one tile at a time, two TMEM accumulators (epilogue of tile j overlaps the main
-// loop of tile j+1):
+// Persistent CTA of 24 warps, one tile at a time.  BT <= 192: two TMEM accumulators (the epilogue of tile j overlaps
+// the main loop of tile j+1); BT = 256: one accumulator and eight TMEM weight stages, the exposed epilogue is shared
+// with the dequantising warps.
 //   warp 0      TMA producer of this CTA's half activation tile X[BT/2, 64] (128-byte swizzle)    -> x ring
 //   warp 2      TMA producer of packed weights [128, 64] (+ scales every 4 k-blocks)              -> raw ring
 //   warps 8-23  dequantise raw -> bf16, written with tcgen05.st into TMEM weight stages (4 groups x 4 warps,
