@@ -71,7 +71,8 @@ struct Cfg {
                                                                    // weights (TMEM) and the full/done barriers
     static constexpr int SR = SX;
     static constexpr int NACC = (BT > 192) ? 1 : 2;                // accumulators in tensor memory
-    static constexpr int SA = ((512 - NACC * BT) / 32 >= 8) ? 8 : 4;   // dequantised-weight stages in tensor memory
+    static constexpr int SA = ((512 - NACC * BT) / 32 >= 8) ? 8 : (512 - NACC * BT) / 32;   // dequantised-weight stages in
+                                                                   // tensor memory (8, or what two accumulators leave)
     // With a single accumulator the epilogue is exposed, so the dequantising warps share it (they would idle at the
     // tile boundary); with two accumulators it overlaps the next main loop and the dequantising warps stay on theirs.
     static constexpr bool HELP = (NACC == 1);
@@ -99,6 +100,7 @@ struct Cfg {
     static_assert(NACC * BT + SA * 32 <= 512, "tensor memory budget");
     static_assert(X_BYTES % 1024 == 0, "swizzled stages must stay 1024-byte aligned");
     static_assert(SX == 8, "stage arithmetic below assumes a ring of eight");
+    static_assert(SA >= 4 && (!HELP || SA == 8), "weight stages");
 };
 
 struct Tile {
@@ -478,6 +480,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 QG_ACC(2);
                 const uint32_t d_tmem = tmem_base + a * BT;
                 uint32_t i = i0 + w;
+                uint32_t ta = i % C::SA;                                     // TMEM weight stage of k-block i
                 bool ready = mbar_test_wait_cluster(full(i & 7u), (i >> 3) & 1u);
                 for (int kb = static_cast<int>(w); kb < nkb; kb += 2, i += 2) {
                     const uint32_t st = i & 7u;
@@ -488,12 +491,17 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     // start the wait for this warp's next k-block before issuing, so its latency is hidden
                     ready = (kb + 2 < nkb) && mbar_test_wait_cluster(full((i + 2) & 7u), ((i + 2) >> 3) & 1u);
                     if (lane == 0) {
-                        umma_kblock_ts_pair(d_tmem, tmem_base + C::A_COL0 + (st & (C::SA - 1)) * C::A_COLS,
+#ifdef QG_PROFILE
+                        if (!(p.dbg & 64))
+#endif
+                        umma_kblock_ts_pair(d_tmem, tmem_base + C::A_COL0 + ta * C::A_COLS,
                                             b_lo0 + st * (C::X_BYTES >> 4), b_hi, idesc, kb != 0 ? 1u : 0u);
                         umma_commit_pair(done(st));
                     }
                     __syncwarp();
                     QG_ACC(10);
+                    ta += 2;
+                    if (ta >= C::SA) ta -= C::SA;
                 }
                 if (ok && lane == 0) umma_commit_pair(acc_full(a));
                 __syncwarp();
@@ -526,6 +534,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         const uint32_t acc_empty_leader = map_to_cta(acc_empty(0), 0);
         constexpr bool plain_ep = (EPI == 0);
         __nv_bfloat16* my_st = stg16 + (warp - 8) * 512;               // private 1 KB transposition buffer
+        uint32_t ta = static_cast<uint32_t>(g) % C::SA;                 // TMEM weight stage of own k-block i = i % SA
         bool dq_ok = true;
         auto help_tile = [&](uint32_t jt) -> bool {
             const Tile tl = decode_tile(pair + static_cast<int>(jt) * n_pairs, prefix, p, BT);
@@ -603,10 +612,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 if (++in2 == per_tile) { in2 = 0; ++t2; }
             }
             // its TMEM stage (i % SA) is free once the MMAs of k-block i - SA have completed
-            if constexpr (C::SA == 8) {
-                if (n >= 2 && !wait_bar<false>(done(sr), (phr ^ 1u), abort_flag, p.status)) break;
-            } else {
-                if (n >= 1 && !wait_bar<false>(done((((n - 1) & 1u) << 2) + g), ((n - 1) >> 1) & 1u, abort_flag, p.status)) break;
+            {
+                const uint32_t i = 4u * n + g;
+                if (i >= C::SA && !wait_bar<false>(done((i - C::SA) & 7u), ((i - C::SA) >> 3) & 1u, abort_flag, p.status)) break;
             }
             QG_ACC(6);
             if (warp == 8 && lane == 0) { QG_TRACE(6, 4 * n); }
@@ -618,14 +626,16 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 if (!(p.dbg & 1) || n < 2)
 #endif
                 {
-                    tmem_st_32x32_x16(a_taddr + (sr & (C::SA - 1)) * C::A_COLS, o0);
-                    tmem_st_32x32_x16(a_taddr + (sr & (C::SA - 1)) * C::A_COLS + 16, o1);
+                    tmem_st_32x32_x16(a_taddr + ta * C::A_COLS, o0);
+                    tmem_st_32x32_x16(a_taddr + ta * C::A_COLS + 16, o1);
                 }
             }
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(full_leader + 8u * sr);
+            ta += 4;
+            if (ta >= C::SA) ta -= C::SA;
             QG_ACC(7);
             if (warp == 8 && lane == 0) { QG_TRACE(7, 4 * n); }
         }
