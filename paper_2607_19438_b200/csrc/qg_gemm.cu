@@ -90,7 +90,9 @@ struct Cfg {
     static constexpr int OFF_SC = OFF_RAW + SR * RAW_BYTES;
     static constexpr int OFF_STG = OFF_SC + NSB * SC_BYTES;
     static constexpr int OFF_PREFIX = OFF_STG + STG_BYTES;
-    static constexpr int OFF_BAR = OFF_PREFIX + (MAX_E + 4) * 4;
+    static constexpr int TAB_N = 128;                              // decoded tiles of this pair kept in shared memory
+    static constexpr int OFF_TAB = OFF_PREFIX + (MAX_E + 4) * 4;
+    static constexpr int OFF_BAR = OFF_TAB + TAB_N * 16;
     static constexpr int NBAR = 2 * SX + 2 * SR + 4;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;        // + slack for 1024-byte alignment
@@ -103,7 +105,7 @@ struct Cfg {
     static_assert(SA >= 4 && (!HELP || SA == 8), "weight stages");
 };
 
-struct Tile {
+struct __align__(16) Tile {
     int e, pw, tok0, tok_end;   // expert, pair weight tile (weight tiles 2 pw and 2 pw + 1), token range
 };
 
@@ -363,6 +365,16 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     const uint32_t tmem_base = static_cast<uint32_t>(misc[0]);
     const int total_tiles = prefix[p.E];
     const int nkb = p.K / BK;     // a multiple of 4
+    // The pair's j-th tile is tile pair + j n_pairs.  Decoding one costs a binary search and two global loads, far
+    // too much for the control warps to repeat at every tile boundary, so the first TAB_N are decoded once, here.
+    const int my_tiles = (total_tiles > pair) ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
+    Tile* tab = reinterpret_cast<Tile*>(sgen + C::OFF_TAB);
+    for (int j = threadIdx.x; j < min(my_tiles, C::TAB_N); j += NTHREADS)
+        tab[j] = decode_tile(pair + j * n_pairs, prefix, p, BT);
+    __syncthreads();
+    auto tile_at = [&](int j) -> Tile {
+        return (j < C::TAB_N) ? tab[j] : decode_tile(pair + j * n_pairs, prefix, p, BT);
+    };
     constexpr bool gate_up = (EPI == 1);
 
     // Control warps walk their loops with all 32 lanes (converged) and keep the per-k-block instruction count small:
@@ -375,8 +387,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         const uint32_t full_leader = map_to_cta(full(0), 0);
         bool ok = true;
         QG_DECL();
-        for (int t = pair; t < total_tiles && ok; t += n_pairs) {
-            const Tile tl = decode_tile(t, prefix, p, BT);
+        for (int jt = 0; jt < my_tiles && ok; ++jt) {
+            const Tile tl = tile_at(jt);
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const int row0 = tl.tok0 + static_cast<int>(rank) * (n_mma >> 1);   // B rows split at N / 2
             for (int kb = 0; kb < nkb; kb += 2) {
@@ -411,8 +423,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         uint32_t s = 0, ph = 0, sg = 0;     // first raw stage of the batch (0 or 4), parity, scale buffer
         bool ok = true;
         QG_DECL();
-        for (int t = pair; t < total_tiles && ok; t += n_pairs) {
-            const Tile tl = decode_tile(t, prefix, p, BT);
+        for (int jt = 0; jt < my_tiles && ok; ++jt) {
+            const Tile tl = tile_at(jt);
             const int wt = 2 * tl.pw + static_cast<int>(rank);
             const int row_a = tl.e * p.N + wt * (gate_up ? 64 : 128);
             const int row_b = row_a + (gate_up ? (p.N / 2) : 64);
@@ -464,8 +476,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const uint32_t b_hi = (1024u >> 4) | (1u << 14) | (2u << 29);   // stride, version, 128-byte swizzle
             const uint32_t b_lo0 = ((sbase + C::OFF_X) >> 4) | (1u << 16);
             uint32_t j = 0;
-            for (int t = pair; t < total_tiles && ok; t += n_pairs, ++j) {
-                const Tile tl = decode_tile(t, prefix, p, BT);
+            for (; static_cast<int>(j) < my_tiles && ok; ++j) {
+                const Tile tl = tile_at(static_cast<int>(j));
                 const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
                 const uint32_t idesc = umma_idesc_bf16(2 * BW, n_mma);
                 const uint32_t a = (C::NACC == 2) ? (j & 1u) : 0u;
@@ -522,7 +534,6 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         const uint32_t raw_row = row * C::RAW_ROW;
         const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + C::A_COL0;
         const uint32_t full_leader = map_to_cta(full(0), 0);
-        const int my_tiles = (total_tiles > pair) ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
         const uint32_t n_own = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(nkb >> 2);
         QG_DECL();
         // Helping with the epilogue.  Before this warp waits for the MMAs of own k-block n - 2 (to reuse their TMEM
@@ -537,7 +548,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         uint32_t ta = static_cast<uint32_t>(g) % C::SA;                 // TMEM weight stage of own k-block i = i % SA
         bool dq_ok = true;
         auto help_tile = [&](uint32_t jt) -> bool {
-            const Tile tl = decode_tile(pair + static_cast<int>(jt) * n_pairs, prefix, p, BT);
+            const Tile tl = tile_at(static_cast<int>(jt));
             const int wt = 2 * tl.pw + static_cast<int>(rank);
             const uint32_t a = (C::NACC == 2) ? (jt & 1u) : 0u;
             const uint32_t aph = (C::NACC == 2) ? ((jt >> 1) & 1u) : (jt & 1u);
@@ -651,8 +662,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         const uint32_t acc_empty_base = map_to_cta(acc_empty(0), 0);
         uint32_t j = 0;
         QG_DECL();
-        for (int t = pair; t < total_tiles; t += n_pairs, ++j) {
-            const Tile tl = decode_tile(t, prefix, p, BT);
+        for (; static_cast<int>(j) < my_tiles; ++j) {
+            const Tile tl = tile_at(static_cast<int>(j));
             const int wt = 2 * tl.pw + static_cast<int>(rank);     // may be one past the last tile: nothing is stored
             const uint32_t a = (C::NACC == 2) ? (j & 1u) : 0u;
             const uint32_t aph = (C::NACC == 2) ? ((j >> 1) & 1u) : (j & 1u);
