@@ -16,24 +16,30 @@ constexpr int ROUTE_WARPS = 8;
 
 // Order of experts for one token: larger logit first, equal logits (IEEE ==, so -0 == +0) by lower
 // index; NaN after every number.
-__device__ __forceinline__ bool route_before(float a, int ia, float b, int ib) {
-    const bool na = (a != a), nb = (b != b);
-    if (na || nb) return (na == nb) ? (ia < ib) : nb;
-    if (a != b) return a > b;
-    return ia < ib;
+// Order-preserving key of a logit: larger key = earlier in the order above.  Numbers map monotonically onto
+// [0x007FFFFF, 0xFF800000] (-0 and +0 share a key), NaN onto 1; key 0 marks an expert already selected.
+__device__ __forceinline__ uint32_t route_key(float v) {
+    if (v != v) return 1u;
+    const uint32_t b = __float_as_uint(v + 0.0f);            // -0 + 0 = +0
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float route_unkey(uint32_t key) {
+    if (key == 1u) return __int_as_float(0x7FC00000);
+    return __uint_as_float((key & 0x80000000u) ? (key ^ 0x80000000u) : ~key);
 }
 
-// One warp per token (each warp walks ROUTE_TOKENS_PER_BLOCK / ROUTE_WARPS tokens).  Lane l owns the
-// logits e = l, l+32, ...; k rounds of (local best, warp arg-best by shuffles, mark taken).
-// Dynamic shared memory: per warp E floats (logits) + k floats (selected logits); then E ints (hist).
+// One warp per token (each warp walks ROUTE_TOKENS_PER_BLOCK / warps tokens).  The token's logits sit in shared
+// memory as keys; lane l owns the experts e = l, l+32, ...  Each of the k rounds takes the largest remaining key
+// with one warp-wide max and, among the lanes that hold it, the lowest expert index with one warp-wide min, then
+// zeroes that key.  Dynamic shared memory: per warp E keys + k floats (selected logits); then E ints (hist).
 __global__ void __launch_bounds__(1024)
 route_topk_kernel(int M, int E, int k, const float* __restrict__ logits, int32_t* __restrict__ topk_idx,
                   float* __restrict__ topk_w, int32_t* __restrict__ block_hist) {
     extern __shared__ float sm[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nwarps = blockDim.x >> 5;          // 32 (one token per warp) unless E is large, then 8
-    float* lg = sm + warp * (E + k);
-    float* sel = lg + E;
+    uint32_t* keys = reinterpret_cast<uint32_t*>(sm) + warp * (E + k);
+    float* sel = reinterpret_cast<float*>(keys + E);
     int* hist = reinterpret_cast<int*>(sm + nwarps * (E + k));
     for (int e = threadIdx.x; e < E; e += blockDim.x) hist[e] = 0;
     __syncthreads();
@@ -43,28 +49,22 @@ route_topk_kernel(int M, int E, int k, const float* __restrict__ logits, int32_t
         const int t = t0 + tt;
         if (t >= M) break;
         const float* row = logits + static_cast<size_t>(t) * E;
-        for (int e = lane; e < E; e += 32) lg[e] = row[e];
+        for (int e = lane; e < E; e += 32) keys[e] = route_key(row[e]);
         __syncwarp();
-        uint32_t taken = 0;  // bit i: element lane + 32 i already selected
         for (int s = 0; s < k; ++s) {
-            float bv = 0.f;
-            int bi = -1;
-            for (int e = lane, i = 0; e < E; e += 32, ++i) {
-                if ((taken >> i) & 1u) continue;
-                const float v = lg[e];
-                if (bi < 0 || route_before(v, e, bv, bi)) { bv = v; bi = e; }
+            uint32_t bk = 0u;                    // best key among this lane's experts and the first expert holding it
+            int bi = 0x7FFFFFFF;
+            for (int e = lane; e < E; e += 32) {
+                const uint32_t key = keys[e];
+                if (key > bk) { bk = key; bi = e; }
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, off);
-                const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, off);
-                if (oi >= 0 && (bi < 0 || route_before(ov, oi, bv, bi))) { bv = ov; bi = oi; }
-            }
-            if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
+            const uint32_t wk = __reduce_max_sync(0xFFFFFFFFu, bk);
+            const int wi = static_cast<int>(__reduce_min_sync(0xFFFFFFFFu, static_cast<uint32_t>(bk == wk ? bi : 0x7FFFFFFF)));
+            if ((wi & 31) == lane) keys[wi] = 0u;
             if (lane == 0) {
-                sel[s] = bv;
-                topk_idx[static_cast<size_t>(t) * k + s] = bi;
-                atomicAdd(&hist[bi], 1);
+                sel[s] = route_unkey(wk);
+                topk_idx[static_cast<size_t>(t) * k + s] = wi;
+                atomicAdd(&hist[wi], 1);
             }
         }
         __syncwarp();
@@ -194,10 +194,23 @@ combine_kernel(int M, int k, int H8, const int4* __restrict__ D, const int32_t* 
     const int t = blockIdx.x;
     for (int v = threadIdx.x; v < H8; v += blockDim.x) {
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int s = 0; s < k; ++s) {
-            const int row = pair_row[static_cast<size_t>(t) * k + s];
-            const float w = topk_w ? topk_w[static_cast<size_t>(t) * k + s] : 1.0f;
-            add8(acc, __ldg(D + static_cast<size_t>(row) * H8 + v), w);
+        // Eight slots at a time: all row indices, then all rows, are in flight together; the sum stays in slot order.
+        for (int s0 = 0; s0 < k; s0 += 8) {
+            int row[8];
+            float w[8];
+            int4 d[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const bool on = s0 + j < k;
+                row[j] = on ? pair_row[static_cast<size_t>(t) * k + s0 + j] : -1;
+                w[j] = (on && topk_w) ? topk_w[static_cast<size_t>(t) * k + s0 + j] : 1.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                d[j] = (row[j] >= 0) ? __ldg(D + static_cast<size_t>(row[j]) * H8 + v) : make_int4(0, 0, 0, 0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (row[j] >= 0) add8(acc, d[j], w[j]);
         }
         int4 o;
         o.x = pack_bf16x2(acc[0], acc[1]); o.y = pack_bf16x2(acc[2], acc[3]);
