@@ -233,65 +233,80 @@ __device__ __forceinline__ float lds_scale(uint32_t addr) {
 }
 
 // Plain / routing-weighted epilogue of one warp: drains the 16-column (token) blocks b = pid, pid + npart, ... of
-// its 32 TMEM lanes (weight rows), rounds to bf16, transposes through a private [16 tokens][32 rows] buffer and
-// writes 16-byte pieces (64 contiguous bytes per token).  The next block's TMEM load is in flight while the current
-// one is processed.  Called by the four epilogue warps and by the sixteen dequantising warps, which would otherwise
-// idle at a tile boundary: a single warp retires only about one dependent instruction every few cycles, so the
-// drain time of a tile scales inversely with the number of warps that share it.
+// its 32 TMEM lanes (weight rows).  The block is read in accumulator-fragment layout (thread T: rows T/4 + 8 m,
+// token pairs), scaled, packed to bf16x2 and written with two transposing matrix stores into a private
+// [16 tokens][32 rows] buffer (16-byte chunks XOR-swizzled by the token pair, conflict-free both ways), from which
+// every thread moves two 16-byte pieces to global memory (64 contiguous bytes per token).  The next block's TMEM
+// loads are in flight while the current one is stored.  Called by the four epilogue warps and, for a
+// single-accumulator tile, by the sixteen dequantising warps, which would otherwise idle at the tile boundary.
 __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int tok_end, int n_base, uint32_t taddr,
                                             int n_epi, int pid, int npart, __nv_bfloat16* st, int lane) {
     __nv_bfloat16* outb = static_cast<__nv_bfloat16*>(p.out);
     const int nblk = n_epi >> 4;
-    uint32_t v[16];
+    const bool weighted = (p.mode == QG_MODE_DOWN_WEIGHTED);
+    uint32_t v0[8], v1[8];                       // TMEM lanes 0-15 / 16-31 of this warp's quarter
     int b = pid;
-    if (b < nblk) tmem_ld_32x32_x16(taddr + 16 * b, v);
+    if (b < nblk) {
+        tmem_ld_16x256_x2(taddr + 16 * b, v0);
+        tmem_ld_16x256_x2(taddr + (16u << 16) + 16 * b, v1);
+    }
     // Routing weights of the whole tile, fetched once (two dependent global loads, all in flight together): lane l
     // holds the weights of tokens l, l + 32, ... of the tile.
     float wt8[8];
-    if (p.mode == QG_MODE_DOWN_WEIGHTED) {
+    if (weighted) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int tokl = tok0 + 32 * j + lane;
             wt8[j] = (32 * j < n_epi && tokl < tok_end) ? p.topk_w[p.row_pair[tokl]] : 0.f;
         }
     }
+    const uint32_t st_s = smem_u32(st);
+    const uint32_t st_row = st_s + (lane & 7) * 64 + (((lane >> 3) ^ ((lane >> 1) & 3)) << 4);   // matrix lane>>3, token lane&7
+    const int c = 2 * (lane & 3);                // this thread's token pairs: c, c + 1 and 8 + c, 9 + c of the block
     while (b < nblk) {
-        float wv = 1.0f;
-        if (p.mode == QG_MODE_DOWN_WEIGHTED) {
-            const int j = b >> 1;        // tokens 16 b .. 16 b + 15 live in register j, lanes 16 (b & 1) ..
-            wv = wt8[0];
+        float w0 = 1.f, w1 = 1.f, w2 = 1.f, w3 = 1.f;
+        if (weighted) {
+            const int j = b >> 1;                // tokens 16 b .. 16 b + 15 live in register j, lanes 16 (b & 1) ..
+            float wv = wt8[0];
 #pragma unroll
             for (int jj = 1; jj < 8; ++jj) wv = (j == jj) ? wt8[jj] : wv;
-            wv = __shfl_sync(0xFFFFFFFFu, wv, 16 * (b & 1) + (lane & 15));
+            const int src = 16 * (b & 1) + c;
+            w0 = __shfl_sync(0xFFFFFFFFu, wv, src);
+            w1 = __shfl_sync(0xFFFFFFFFu, wv, src + 1);
+            w2 = __shfl_sync(0xFFFFFFFFu, wv, src + 8);
+            w3 = __shfl_sync(0xFFFFFFFFu, wv, src + 9);
         }
         tmem_ld_wait();
-        uint32_t h[16];
+        uint32_t pk[8];
 #pragma unroll
-        for (int jj = 0; jj < 16; ++jj) {
-            float val = __uint_as_float(v[jj]);
-            if (p.mode == QG_MODE_DOWN_WEIGHTED) val *= __shfl_sync(0xFFFFFFFFu, wv, jj);
-            h[jj] = __float_as_uint(val);
+        for (int g = 0; g < 2; ++g) {            // tokens 8 g .. 8 g + 7
+            const float wa = g ? w2 : w0, wb = g ? w3 : w1;
+            pk[4 * g + 0] = bf16x2(__uint_as_float(v0[4 * g + 0]) * wa, __uint_as_float(v0[4 * g + 1]) * wb);
+            pk[4 * g + 1] = bf16x2(__uint_as_float(v0[4 * g + 2]) * wa, __uint_as_float(v0[4 * g + 3]) * wb);
+            pk[4 * g + 2] = bf16x2(__uint_as_float(v1[4 * g + 0]) * wa, __uint_as_float(v1[4 * g + 1]) * wb);
+            pk[4 * g + 3] = bf16x2(__uint_as_float(v1[4 * g + 2]) * wa, __uint_as_float(v1[4 * g + 3]) * wb);
         }
         const int bn = b + npart;
-        if (bn < nblk) tmem_ld_32x32_x16(taddr + 16 * bn, v);      // next block, overlapped with the stores below
-#pragma unroll
-        for (int jj = 0; jj < 16; ++jj) st[jj * 32 + lane] = __float2bfloat16_rn(__uint_as_float(h[jj]));
+        if (bn < nblk) {                         // next block, overlapped with the stores below
+            tmem_ld_16x256_x2(taddr + 16 * bn, v0);
+            tmem_ld_16x256_x2(taddr + (16u << 16) + 16 * bn, v1);
+        }
+        stmatrix_x4_trans(st_row, pk[0], pk[1], pk[2], pk[3]);
+        stmatrix_x4_trans(st_row + 512, pk[4], pk[5], pk[6], pk[7]);
         __syncwarp();
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-            const int piece = i * 32 + lane;
-            const int tk = piece >> 2, c4 = piece & 3;
+            const int tk = i * 8 + (lane >> 2), c4 = lane & 3;
             const int tok = tok0 + 16 * b + tk;
             const int n = n_base + c4 * 8;
             if (tok < tok_end && n < p.N)
                 *reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * p.N + n) =
-                    *reinterpret_cast<const uint4*>(st + tk * 32 + c4 * 8);
+                    *reinterpret_cast<const uint4*>(st + tk * 32 + ((c4 ^ ((tk >> 1) & 3)) << 3));
         }
         __syncwarp();
         b = bn;
     }
 }
-
 // EPI: 0 plain / routing-weighted bf16 store, 1 gate/up + SiLU, 2 weighted fp32 atomic accumulate (compiled apart so
 // that each instantiation carries one epilogue only).
 template <int QBITS, int BT, int EPI>
@@ -567,6 +582,14 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         for (uint32_t n = 0; n < n_own && dq_ok; ++n) {       // own k-block i = 4 n + g
             const uint32_t sr = ((n & 1u) << 2) + g;               // ring stage i % 8
             const uint32_t phr = (n >> 1) & 1u;                    // parity of (i / 8)
+            // (t2 = tile of own k-block n - 2.)  The release must come before this iteration's wait for the MMAs of
+            // own k-block n - 2, or the single-accumulator pipeline would wait for itself; it is done first, while
+            // no converted weights are held in registers.
+            if (C::HELP && n >= 2) {
+                while (dq_ok && helped < t2) dq_ok = help_tile(helped++);
+                if (!dq_ok) break;
+                if (++in2 == per_tile) { in2 = 0; ++t2; }
+            }
             QG_T0();
             // the scales of this group of four k-blocks arrive with the first of them (stage 0 or 4)
             if (!wait_bar<false>(r_full((n & 1u) << 2), phr, abort_flag, p.status)) break;
@@ -615,13 +638,6 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             __syncwarp();
             if (lane == 0) mbar_arrive(r_empty(sr));             // the packed codes are in registers now
             QG_ACC(7);
-            // (t2 = tile of own k-block n - 2.)  The release must come before the wait below, or the single-accumulator
-            // pipeline would wait for itself.
-            if (C::HELP && n >= 2) {
-                while (dq_ok && helped < t2) dq_ok = help_tile(helped++);
-                if (!dq_ok) break;
-                if (++in2 == per_tile) { in2 = 0; ++t2; }
-            }
             // its TMEM stage (i % SA) is free once the MMAs of k-block i - SA have completed
             {
                 const uint32_t i = 4u * n + g;
@@ -806,7 +822,7 @@ static long long* g_stats = nullptr;   // device buffer supplied by the profilin
 static int pick_token_tile(const qg_ctx* ctx, int M, int n_wt, int K) {
     if (M <= 128) return 128;
     const int cand[3] = {128, 192, 256};
-    const double period[3] = {670.0, 700.0, 720.0}, epilogue[3] = {0.0, 0.0, 8000.0};
+    const double period[3] = {625.0, 665.0, 720.0}, epilogue[3] = {0.0, 0.0, 6000.0};
     const long long pairs = ctx->sm_count / 2, n_pw = (n_wt + 1) / 2;
     int best = 256;
     double best_cost = 1e300;

@@ -220,6 +220,23 @@ __device__ __forceinline__ void tmem_ld_32x32_x16(uint32_t taddr, uint32_t (&v)[
         : "r"(taddr)
         : "memory");
 }
+// 16 lanes x 16 columns in the layout of an MMA accumulator fragment: thread T holds, for the column groups
+// g = 0, 1 (columns 8 g ..), v[4 g + 0..1] = lane T/4, columns 8 g + 2 (T%4) + {0, 1} and v[4 g + 2..3] = the same
+// columns of lane T/4 + 8.
+__device__ __forceinline__ void tmem_ld_16x256_x2(uint32_t taddr, uint32_t (&v)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+// Four 8x8 matrices of 16-bit elements, stored transposed.  Register m of thread T holds row T/4, columns
+// 2 (T%4) + {0, 1} of matrix m; thread 8 m + j supplies the shared-memory address of the 16 bytes that receive
+// column j of matrix m (its eight rows, in order).
+__device__ __forceinline__ void stmatrix_x4_trans(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1, %2, %3, %4};"
+                 ::"r"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+                 : "memory");
+}
 // Thread i of the warp writes 8 consecutive 32-bit columns of lane (base + i).
 __device__ __forceinline__ void tmem_st_32x32_x8(uint32_t taddr, const uint32_t (&v)[8]) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
