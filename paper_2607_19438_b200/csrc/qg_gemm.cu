@@ -152,11 +152,13 @@ __device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&b);
 }
 
-// Two fp32 fused multiply-adds in one instruction (fma.rn.f32x2, each lane IEEE-exact as fmaf) followed by the
-// packed round-to-nearest-even conversion to bf16x2: returns bf16(a0 * m.lo + c.lo) | bf16(a1 * m.hi + c.hi) << 16.
-// One issue slot per two weights instead of two.
+// Dequantisation arithmetic.  A code byte c (0..255) dropped into byte 1 of 0x43000000 reads as the float
+// 128 + c / 256, so q * s = fma(f, 256 s, -(32768 + 256 z) s) for the code's zero point z (128 for the sign-flipped
+// int8 byte, 8 for a nibble): both constants and the result are exact in fp32, one rounding (to bf16) follows.
+// Per weight: one byte permute builds f from a code byte and the magic word, half a packed two-float fused
+// multiply-add (fma.rn.f32x2, each lane IEEE-exact as fmaf) converts, half a packed conversion rounds to bf16x2.
 __device__ __forceinline__ uint32_t fma2_bf16x2(uint32_t a0, uint32_t a1, uint64_t m, uint64_t c) {
-    uint32_t r;
+    uint32_t r;     // bf16(a0 * m.lo + c.lo) | bf16(a1 * m.hi + c.hi) << 16
     asm("{\n\t.reg .b64 t;\n\t.reg .b32 lo, hi;\n\t"
         "mov.b64 t, {%1, %2};\n\t"
         "fma.rn.f32x2 t, t, %3, %4;\n\t"
@@ -168,52 +170,26 @@ __device__ __forceinline__ uint32_t fma2_bf16x2(uint32_t a0, uint32_t a1, uint64
 __device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
     return static_cast<uint64_t>(__float_as_uint(lo)) | (static_cast<uint64_t>(__float_as_uint(hi)) << 32);
 }
-
-// 4 int8 codes (one 32-bit word) -> 4 bf16 = q * scale, exact product rounded once.
-// The byte u = q + 128 is dropped into a float's mantissa: 0x4300uu00 = 128 + u/256, so
-// q * s = fma(f, 256 s, -32896 s); both constants and the result are exact in fp32.
-// m2 = {256 s, 256 s}, c2 = {-32896 s, -32896 s}.
-__device__ __forceinline__ void dq8_word(uint32_t x, uint64_t m2, uint64_t c2, uint32_t& o0, uint32_t& o1) {
-    x ^= 0x80808080u;
-    const uint32_t f0 = __byte_perm(x, 0x43000000u, 0x7604);
-    const uint32_t f1 = __byte_perm(x, 0x43000000u, 0x7614);
-    const uint32_t f2 = __byte_perm(x, 0x43000000u, 0x7624);
-    const uint32_t f3 = __byte_perm(x, 0x43000000u, 0x7634);
-    o0 = fma2_bf16x2(f0, f1, m2, c2);
-    o1 = fma2_bf16x2(f2, f3, m2, c2);
+template <int BYTE>
+__device__ __forceinline__ uint32_t code_byte_to_float(uint32_t x, uint32_t magic) {   // bits of 128 + byte BYTE of x / 256
+    return __byte_perm(x, magic, 0x7404 + (BYTE << 4));
 }
 
-// Constants of the 4-bit conversion for one scale s.  A nibble at bit p of 0x43000000 reads 128 + u 2^(p-16); for
-// p in {8, 12, 16}: q s = fma(f, s 2^(16-p), -(2^(23-p) + 8) s), exact in fp32.  The eight nibbles of a word sit at
-// p = 8, 12 (after << 8), 8, 12, 16 (in place), 8, 12, 16 (after >> 12); the pairs below follow that order.
-struct Dq4Consts {
-    uint64_t m_8_12, c_8_12, m_16_8, c_16_8, m_12_16, c_12_16;
-};
-__device__ __forceinline__ Dq4Consts dq4_consts(float s) {
-    const float m8 = 256.f * s, c8 = -32776.f * s;
-    const float m12 = 16.f * s, c12 = -2056.f * s;
-    const float m16 = s, c16 = -136.f * s;
-    Dq4Consts k;
-    k.m_8_12 = pack_f32x2(m8, m12);   k.c_8_12 = pack_f32x2(c8, c12);
-    k.m_16_8 = pack_f32x2(m16, m8);   k.c_16_8 = pack_f32x2(c16, c8);
-    k.m_12_16 = pack_f32x2(m12, m16); k.c_12_16 = pack_f32x2(c12, c16);
-    return k;
+// 4 int8 codes (one word) -> 4 bf16 = q * scale.  m2 = {256 s, 256 s}, c2 = {-32896 s, -32896 s}.
+__device__ __forceinline__ void dq8_word(uint32_t x, uint64_t m2, uint64_t c2, uint32_t magic, uint32_t& o0, uint32_t& o1) {
+    x ^= 0x80808080u;                            // byte = q + 128
+    o0 = fma2_bf16x2(code_byte_to_float<0>(x, magic), code_byte_to_float<1>(x, magic), m2, c2);
+    o1 = fma2_bf16x2(code_byte_to_float<2>(x, magic), code_byte_to_float<3>(x, magic), m2, c2);
 }
-// 8 4-bit codes (one word, nibble i = weight i, code u = q + 8) -> 8 bf16.
-__device__ __forceinline__ void dq4_word(uint32_t x, const Dq4Consts& k, uint32_t (&o)[4]) {
-    const uint32_t y = x << 8, z = x >> 12;
-    const uint32_t f0 = (y & 0x00000F00u) | 0x43000000u;
-    const uint32_t f1 = (y & 0x0000F000u) | 0x43000000u;
-    const uint32_t f2 = (x & 0x00000F00u) | 0x43000000u;
-    const uint32_t f3 = (x & 0x0000F000u) | 0x43000000u;
-    const uint32_t f4 = (x & 0x000F0000u) | 0x43000000u;
-    const uint32_t f5 = (z & 0x00000F00u) | 0x43000000u;
-    const uint32_t f6 = (z & 0x0000F000u) | 0x43000000u;
-    const uint32_t f7 = (z & 0x000F0000u) | 0x43000000u;
-    o[0] = fma2_bf16x2(f0, f1, k.m_8_12, k.c_8_12);
-    o[1] = fma2_bf16x2(f2, f3, k.m_8_12, k.c_8_12);
-    o[2] = fma2_bf16x2(f4, f5, k.m_16_8, k.c_16_8);
-    o[3] = fma2_bf16x2(f6, f7, k.m_12_16, k.c_12_16);
+
+// 8 4-bit codes (one word, nibble i = weight i, code u = q + 8) -> 8 bf16.  The even and the odd nibbles are
+// spread into the bytes of two words first.  m2 = {256 s, 256 s}, c2 = {-32776 s, -32776 s}.
+__device__ __forceinline__ void dq4_word(uint32_t x, uint64_t m2, uint64_t c2, uint32_t magic, uint32_t* o) {
+    const uint32_t xe = x & 0x0F0F0F0Fu, xo = (x >> 4) & 0x0F0F0F0Fu;
+    o[0] = fma2_bf16x2(code_byte_to_float<0>(xe, magic), code_byte_to_float<0>(xo, magic), m2, c2);
+    o[1] = fma2_bf16x2(code_byte_to_float<1>(xe, magic), code_byte_to_float<1>(xo, magic), m2, c2);
+    o[2] = fma2_bf16x2(code_byte_to_float<2>(xe, magic), code_byte_to_float<2>(xo, magic), m2, c2);
+    o[3] = fma2_bf16x2(code_byte_to_float<3>(xe, magic), code_byte_to_float<3>(xo, magic), m2, c2);
 }
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
@@ -514,6 +490,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     QG_T0();
                     if (!ready && !spin_wait_bar(full(st), (i >> 3) & 1u, abort_flag, p.status)) { ok = false; break; }
                     QG_ACC(3);
+                    if (lane == 0) { QG_TRACE(2, i); }
                     tc_fence_after_sync();
                     // start the wait for this warp's next k-block before issuing, so its latency is hidden
                     ready = (kb + 2 < nkb) && mbar_test_wait_cluster(full((i + 2) & 7u), ((i + 2) >> 3) & 1u);
@@ -527,6 +504,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     }
                     __syncwarp();
                     QG_ACC(10);
+                    if (lane == 0) { QG_TRACE(4, i); }
                     ta += 2;
                     if (ta >= C::SA) ta -= C::SA;
                 }
@@ -550,6 +528,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + C::A_COL0;
         const uint32_t full_leader = map_to_cta(full(0), 0);
         const uint32_t n_own = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(nkb >> 2);
+        constexpr uint32_t magic = 0x43000000u;
         QG_DECL();
         // Helping with the epilogue.  Before this warp waits for the MMAs of own k-block n - 2 (to reuse their TMEM
         // stage) it must have released every accumulator of an earlier tile, otherwise a single-accumulator pipeline
@@ -595,7 +574,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             if (!wait_bar<false>(r_full((n & 1u) << 2), phr, abort_flag, p.status)) break;
             if (!wait_bar<false>(r_full(sr), phr, abort_flag, p.status)) break;
             QG_ACC(5);
-            if (warp == 8 && lane == 0) { QG_TRACE(5, 4 * n); }
+            if (q == 0 && lane == 0) { QG_TRACE(5, 4 * n + g); }
             const uint32_t raw = sbase + C::OFF_RAW + sr * C::RAW_BYTES + raw_row;
             const uint32_t scw = *reinterpret_cast<const uint32_t*>(
                 sgen + C::OFF_SC + (n % C::NSB) * C::SC_BYTES + row * 16 + g * 4);
@@ -615,36 +594,37 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 if constexpr (QBITS == 8) {
                     const uint4 v0 = lds128(raw + (((2 * h) ^ swz) << 4));
                     const uint4 v1 = lds128(raw + (((2 * h + 1) ^ swz) << 4));
-                    const float s256 = 256.f * sc, c = -32896.f * sc;
-                    const uint64_t m2 = pack_f32x2(s256, s256), c2 = pack_f32x2(c, c);
-                    dq8_word(v0.x, m2, c2, oh[0], oh[1]);
-                    dq8_word(v0.y, m2, c2, oh[2], oh[3]);
-                    dq8_word(v0.z, m2, c2, oh[4], oh[5]);
-                    dq8_word(v0.w, m2, c2, oh[6], oh[7]);
-                    dq8_word(v1.x, m2, c2, oh[8], oh[9]);
-                    dq8_word(v1.y, m2, c2, oh[10], oh[11]);
-                    dq8_word(v1.z, m2, c2, oh[12], oh[13]);
-                    dq8_word(v1.w, m2, c2, oh[14], oh[15]);
+                    const float m1 = 256.f * sc, c1 = -32896.f * sc;
+                    const uint64_t m = pack_f32x2(m1, m1), c = pack_f32x2(c1, c1);
+                    dq8_word(v0.x, m, c, magic, oh[0], oh[1]);
+                    dq8_word(v0.y, m, c, magic, oh[2], oh[3]);
+                    dq8_word(v0.z, m, c, magic, oh[4], oh[5]);
+                    dq8_word(v0.w, m, c, magic, oh[6], oh[7]);
+                    dq8_word(v1.x, m, c, magic, oh[8], oh[9]);
+                    dq8_word(v1.y, m, c, magic, oh[10], oh[11]);
+                    dq8_word(v1.z, m, c, magic, oh[12], oh[13]);
+                    dq8_word(v1.w, m, c, magic, oh[14], oh[15]);
                 } else {
                     const uint4 v = lds128(raw + ((h ^ swz) << 4));
-                    uint32_t w4[4];
-                    const Dq4Consts kc = dq4_consts(sc);
-                    dq4_word(v.x, kc, w4); oh[0] = w4[0]; oh[1] = w4[1]; oh[2] = w4[2]; oh[3] = w4[3];
-                    dq4_word(v.y, kc, w4); oh[4] = w4[0]; oh[5] = w4[1]; oh[6] = w4[2]; oh[7] = w4[3];
-                    dq4_word(v.z, kc, w4); oh[8] = w4[0]; oh[9] = w4[1]; oh[10] = w4[2]; oh[11] = w4[3];
-                    dq4_word(v.w, kc, w4); oh[12] = w4[0]; oh[13] = w4[1]; oh[14] = w4[2]; oh[15] = w4[3];
+                    const float m1 = 256.f * sc, c1 = -32776.f * sc;
+                    const uint64_t m = pack_f32x2(m1, m1), c = pack_f32x2(c1, c1);
+                    dq4_word(v.x, m, c, magic, oh);
+                    dq4_word(v.y, m, c, magic, oh + 4);
+                    dq4_word(v.z, m, c, magic, oh + 8);
+                    dq4_word(v.w, m, c, magic, oh + 12);
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(r_empty(sr));             // the packed codes are in registers now
             QG_ACC(7);
+            if (q == 0 && lane == 0) { QG_TRACE(9, 4 * n + g); }
             // its TMEM stage (i % SA) is free once the MMAs of k-block i - SA have completed
             {
                 const uint32_t i = 4u * n + g;
                 if (i >= C::SA && !wait_bar<false>(done((i - C::SA) & 7u), ((i - C::SA) >> 3) & 1u, abort_flag, p.status)) break;
             }
             QG_ACC(6);
-            if (warp == 8 && lane == 0) { QG_TRACE(6, 4 * n); }
+            if (q == 0 && lane == 0) { QG_TRACE(6, 4 * n + g); }
             tc_fence_after_sync();
             {
                 uint32_t (&o0)[16] = *reinterpret_cast<uint32_t (*)[16]>(o);
@@ -664,7 +644,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             ta += 4;
             if (ta >= C::SA) ta -= C::SA;
             QG_ACC(7);
-            if (warp == 8 && lane == 0) { QG_TRACE(7, 4 * n); }
+            if (q == 0 && lane == 0) { QG_TRACE(7, 4 * n + g); }
         }
         while (C::HELP && dq_ok && helped < static_cast<uint32_t>(my_tiles)) dq_ok = help_tile(helped++);
         __syncwarp();
