@@ -35,7 +35,7 @@ DENSE_SET = [("qkv", 2560, 2048), ("o", 2048, 2048), ("gate_up", 16384, 2048), (
 MOE = dict(H=2048, E=128, k=8, F=768)
 # DRAM bytes (read + written) per launch of qgemm_kernel from one ncu capture of this step, averaged over the captured
 # launches (profiles/qgemm_kernel_bench_step_ncu_full.md).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 152.0e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 107.0e6
 
 
 def dense_flops(M):
