@@ -69,7 +69,8 @@ struct Cfg {
     static constexpr int SX = 8;                                   // k-block stages: one ring index for the activation tile
                                                                    // (smem), the packed weights (smem), the dequantised
                                                                    // weights (TMEM) and the full/done barriers
-    static constexpr int SR = SX;
+    static constexpr int SR = (QBITS == 4 && BT <= 192) ? 16 : 8;   // packed-weight stages (refilled four at a time); the
+                                                                   // 4-bit tile is half the size, so its ring can be twice as deep
     static constexpr int NACC = (BT > 192) ? 1 : 2;                // accumulators in tensor memory
     static constexpr int SA = ((512 - NACC * BT) / 32 >= 8) ? 8 : (512 - NACC * BT) / 32;   // dequantised-weight stages in
                                                                    // tensor memory (8, or what two accumulators leave)
@@ -77,7 +78,7 @@ struct Cfg {
     // tile boundary); with two accumulators it overlaps the next main loop and the dequantising warps stay on theirs.
     static constexpr bool HELP = (NACC == 1);
     static constexpr int EPI_PARTS = HELP ? 5 : 1;                  // warps per TMEM lane quarter that drain a tile
-    static constexpr int NSB = 3;                                  // scale buffers (one per 4 k-blocks)
+    static constexpr int NSB = SR / 4 + 1;                         // scale buffers (one per 4 k-blocks)
     static constexpr int XH_ROWS = BT / 2;                         // token rows this CTA stages per k-block
     static constexpr int X_BYTES = XH_ROWS * 128;
     static constexpr int RAW_ROW = (QBITS == 8) ? 64 : 32;         // packed bytes per row per stage
@@ -447,7 +448,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 }
                 __syncwarp();
                 if (++sg == C::NSB) sg = 0;
-                s ^= 4u;
+                s = (s + 4u) & (C::SR - 1);
                 if (s == 0) ph ^= 1u;
             }
         }
@@ -559,8 +560,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             return true;
         };
         for (uint32_t n = 0; n < n_own && dq_ok; ++n) {       // own k-block i = 4 n + g
-            const uint32_t sr = ((n & 1u) << 2) + g;               // ring stage i % 8
-            const uint32_t phr = (n >> 1) & 1u;                    // parity of (i / 8)
+            constexpr uint32_t NB = C::SR / 4;                     // batches of four stages in the packed-weight ring
+            const uint32_t sr = ((n % NB) << 2) + g;               // ring stage i % SR
+            const uint32_t phr = (n / NB) & 1u;                    // parity of (i / SR)
             // (t2 = tile of own k-block n - 2.)  The release must come before this iteration's wait for the MMAs of
             // own k-block n - 2, or the single-accumulator pipeline would wait for itself; it is done first, while
             // no converted weights are held in registers.
@@ -571,7 +573,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             }
             QG_T0();
             // the scales of this group of four k-blocks arrive with the first of them (stage 0 or 4)
-            if (!wait_bar<false>(r_full((n & 1u) << 2), phr, abort_flag, p.status)) break;
+            if (!wait_bar<false>(r_full((n % NB) << 2), phr, abort_flag, p.status)) break;
             if (!wait_bar<false>(r_full(sr), phr, abort_flag, p.status)) break;
             QG_ACC(5);
             if (q == 0 && lane == 0) { QG_TRACE(5, 4 * n + g); }
@@ -640,7 +642,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(full_leader + 8u * sr);
+            if (lane == 0) mbar_arrive_cluster(full_leader + 8u * (((n & 1u) << 2) + g));   // k-block stage i % 8
             ta += 4;
             if (ta >= C::SA) ta -= C::SA;
             QG_ACC(7);
