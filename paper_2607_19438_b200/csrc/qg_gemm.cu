@@ -714,16 +714,22 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                         // ([32 tokens][128 rows] fp32), then every thread finishes 16 outputs of one token.
                         const int F = p.N / 2;
 #pragma unroll
-                        for (int jj = 0; jj < 32; ++jj) stg32[jj * 128 + row] = __uint_as_float(v[jj]);
+                        // The 16-byte chunk index of a row is XOR-ed with (chunk / 8) % 2 and 2 (token % 2), so that
+                        // the eight threads of a quarter warp below (two tokens x four 64-byte spans) hit eight
+                        // different bank groups instead of two.
+                        const int wchunk = ((row >> 2) ^ ((row >> 5) & 1)) << 2 | (row & 3);
+#pragma unroll
+                        for (int jj = 0; jj < 32; ++jj) stg32[jj * 128 + (wchunk ^ ((jj & 1) << 3))] = __uint_as_float(v[jj]);
                         named_bar_sync(2, 128);
                         const int tk = et >> 2, f0 = (et & 3) * 16;
                         const int tok = tl.tok0 + c + tk;
+                        const int rsw = ((et & 3) >> 1) ^ ((tk & 1) << 1);      // swizzle of this thread's chunks 4 (et & 3) + i
                         const float4* g4 = reinterpret_cast<const float4*>(stg32 + tk * 128 + f0);
                         const float4* u4 = reinterpret_cast<const float4*>(stg32 + tk * 128 + 64 + f0);
                         uint32_t o[8];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            const float4 g = g4[i], u = u4[i];
+                            const float4 g = g4[i ^ rsw], u = u4[i ^ rsw];
                             const float h0 = __fdividef(g.x, 1.0f + __expf(-g.x)) * u.x;
                             const float h1 = __fdividef(g.y, 1.0f + __expf(-g.y)) * u.y;
                             const float h2 = __fdividef(g.z, 1.0f + __expf(-g.z)) * u.z;
