@@ -77,7 +77,6 @@ struct Cfg {
     // With a single accumulator the epilogue is exposed, so the dequantising warps share it (they would idle at the
     // tile boundary); with two accumulators it overlaps the next main loop and the dequantising warps stay on theirs.
     static constexpr bool HELP = (NACC == 1);
-    static constexpr int EPI_PARTS = HELP ? 5 : 1;                  // warps per TMEM lane quarter that drain a tile
     static constexpr int NSB = SR / 4 + 1;                         // scale buffers (one per 4 k-blocks)
     static constexpr int XH_ROWS = BT / 2;                         // token rows this CTA stages per k-block
     static constexpr int X_BYTES = XH_ROWS * 128;
@@ -542,7 +541,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         __nv_bfloat16* my_st = stg16 + (warp - 8) * 512;               // private 1 KB transposition buffer
         uint32_t ta = static_cast<uint32_t>(g) % C::SA;                 // TMEM weight stage of own k-block i = i % SA
         bool dq_ok = true;
-        auto help_tile = [&](uint32_t jt) -> bool {
+        auto help_tile = [&](uint32_t jt, bool release) -> bool {
             const Tile tl = tile_at(static_cast<int>(jt));
             const int wt = 2 * tl.pw + static_cast<int>(rank);
             const uint32_t a = (C::NACC == 2) ? (jt & 1u) : 0u;
@@ -556,7 +555,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8u * a);
+            if (release && lane == 0) mbar_arrive_cluster(acc_empty_leader + 8u * a);
             return true;
         };
         for (uint32_t n = 0; n < n_own && dq_ok; ++n) {       // own k-block i = 4 n + g
@@ -567,7 +566,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             // own k-block n - 2, or the single-accumulator pipeline would wait for itself; it is done first, while
             // no converted weights are held in registers.
             if (C::HELP && n >= 2) {
-                while (dq_ok && helped < t2) dq_ok = help_tile(helped++);
+                while (dq_ok && helped < t2) dq_ok = help_tile(helped++, true);
                 if (!dq_ok) break;
                 if (++in2 == per_tile) { in2 = 0; ++t2; }
             }
@@ -648,7 +647,10 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             QG_ACC(7);
             if (q == 0 && lane == 0) { QG_TRACE(7, 4 * n + g); }
         }
-        while (C::HELP && dq_ok && helped < static_cast<uint32_t>(my_tiles)) dq_ok = help_tile(helped++);
+        while (C::HELP && dq_ok && helped < static_cast<uint32_t>(my_tiles)) dq_ok = help_tile(helped++, true);
+        // With two accumulators the epilogues overlap the main loops, except the last one: these warps have nothing
+        // left to do then and take four fifths of it (nobody waits for that accumulator again: no release).
+        if (!C::HELP && plain_ep && dq_ok && my_tiles > 0) help_tile(static_cast<uint32_t>(my_tiles - 1), false);
         __syncwarp();
         if (warp == 8 && lane == 0) QG_FLUSH();
     } else if (warp >= 4) {
@@ -683,7 +685,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
 #endif
             if constexpr (EPI == 0) {
                 // shared with the dequantising warps (participants 1..4 of this lane quarter) when they help
-                drain_plain(p, tl.tok0, tl.tok_end, wt * BW + qd * 32, taddr, n_epi2, 0, C::EPI_PARTS,
+                drain_plain(p, tl.tok0, tl.tok_end, wt * BW + qd * 32, taddr, n_epi2, 0,
+                            (C::HELP || static_cast<int>(j) == my_tiles - 1) ? 5 : 1,
                             stg16 + (16 + qd) * 512, lane);
             } else {
                 for (int c = 0; c < n_epi2; c += 32) {
