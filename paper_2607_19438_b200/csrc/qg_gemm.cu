@@ -716,7 +716,6 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                         // lanes 0..63 hold gate rows, 64..127 the matching up rows: transpose through shared memory
                         // ([32 tokens][128 rows] fp32), then every thread finishes 16 outputs of one token.
                         const int F = p.N / 2;
-#pragma unroll
                         // The 16-byte chunk index of a row is XOR-ed with (chunk / 8) % 2 and 2 (token % 2), so that
                         // the eight threads of a quarter warp below (two tokens x four 64-byte spans) hit eight
                         // different bank groups instead of two.
