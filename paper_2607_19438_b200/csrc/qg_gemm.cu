@@ -182,14 +182,19 @@ __device__ __forceinline__ void dq8_word(uint32_t x, uint64_t m2, uint64_t c2, u
     o1 = fma2_bf16x2(code_byte_to_float<2>(x, magic), code_byte_to_float<3>(x, magic), m2, c2);
 }
 
-// 8 4-bit codes (one word, nibble i = weight i, code u = q + 8) -> 8 bf16.  The even and the odd nibbles are
-// spread into the bytes of two words first.  m2 = {256 s, 256 s}, c2 = {-32776 s, -32776 s}.
+// 8 4-bit codes (one word, nibble i = weight i, code u = q + 8) -> 8 bf16.  The nibbles are first spread into
+// the bytes of two words in k order (mask the even and the odd nibbles, interleave their bytes), then converted like
+// the 8-bit codes.  Both permutes of a packed multiply-add read the same word: with operands from two different
+// words the compiler needs a register move per weight to form the pair (measured with the opcode counters).
+// m2 = {256 s, 256 s}, c2 = {-32776 s, -32776 s}.
 __device__ __forceinline__ void dq4_word(uint32_t x, uint64_t m2, uint64_t c2, uint32_t magic, uint32_t* o) {
     const uint32_t xe = x & 0x0F0F0F0Fu, xo = (x >> 4) & 0x0F0F0F0Fu;
-    o[0] = fma2_bf16x2(code_byte_to_float<0>(xe, magic), code_byte_to_float<0>(xo, magic), m2, c2);
-    o[1] = fma2_bf16x2(code_byte_to_float<1>(xe, magic), code_byte_to_float<1>(xo, magic), m2, c2);
-    o[2] = fma2_bf16x2(code_byte_to_float<2>(xe, magic), code_byte_to_float<2>(xo, magic), m2, c2);
-    o[3] = fma2_bf16x2(code_byte_to_float<3>(xe, magic), code_byte_to_float<3>(xo, magic), m2, c2);
+    const uint32_t w03 = __byte_perm(xe, xo, 0x5140);        // codes 0, 1, 2, 3
+    const uint32_t w47 = __byte_perm(xe, xo, 0x7362);        // codes 4, 5, 6, 7
+    o[0] = fma2_bf16x2(code_byte_to_float<0>(w03, magic), code_byte_to_float<1>(w03, magic), m2, c2);
+    o[1] = fma2_bf16x2(code_byte_to_float<2>(w03, magic), code_byte_to_float<3>(w03, magic), m2, c2);
+    o[2] = fma2_bf16x2(code_byte_to_float<0>(w47, magic), code_byte_to_float<1>(w47, magic), m2, c2);
+    o[3] = fma2_bf16x2(code_byte_to_float<2>(w47, magic), code_byte_to_float<3>(w47, magic), m2, c2);
 }
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
