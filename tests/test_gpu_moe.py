@@ -78,3 +78,25 @@ def test_moe_config3_shape_reduced_tokens():
     assert o["counts"].min() <= 2 and o["counts"].max() >= 20      # short and long segments in one launch
     util.assert_close(util.host_bf16_f64(Hh), o["Hh"], "gate/up+silu cfg3")
     util.assert_close(util.host_bf16_f64(y), o["y"], "layer cfg3")
+
+
+def test_grouped_more_tiles_per_pair_than_the_tile_table():
+    """512 experts x 20 pairs of weight tiles = about 10,000 pair tiles, i.e. more per SM pair (about 138) than the
+    128 entries of the kernel's shared-memory tile table: the tiles past the table are decoded on the fly.  Ragged
+    segments, some experts empty; plain grouped mode, every output row against the oracle."""
+    qbits, E, N, K = 4, 512, 5120, 256
+    rng = np.random.default_rng(5)
+    counts = rng.integers(1, 12, size=E).astype(np.int32)
+    counts[rng.integers(0, E, size=6)] = 0
+    offsets = np.zeros(E + 1, np.int32)
+    offsets[1:] = np.cumsum(counts)
+    R = int(offsets[-1])
+    A = synth.activations(R, K, 3, 21)
+    Wq = synth.weights_q4(E * N, K, 3, 22).reshape(E, N, K // 2)
+    Ws = synth.scales(E * N, K // 32, 7, 3, 23).reshape(E, N, K // 32)
+    n_tiles = int(np.count_nonzero(counts)) * ((N // 128 + 1) // 2)
+    assert n_tiles > 128 * 74
+    out = qg.moe_grouped_qgemm(qg.MODE_PLAIN, qbits, util.dev_bf16(A), util.dev(offsets), util.dev(Wq), util.dev_f16(Ws))
+    qg.poll_status()
+    ref = orc.grouped_gemm(qbits, orc.bf16_to_f64(A), offsets, Wq, Ws)
+    util.assert_close(util.host_bf16_f64(out), ref, "grouped plain, tiles beyond the table")
