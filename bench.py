@@ -289,6 +289,12 @@ def run_ours(args):
     detail = {lab: {"launches": v[2], "avg_us": v[1] / v[2] * 1e3, "tflops": (v[0] / (v[1] * 1e-3) / 1e12) if v[0] else None}
               for lab, v in agg.items()}
     peak_tf, peak_hbm, peak_src = measured_peaks()
+    # the HBM-bound calls: algorithmic bytes (route: logits in, indices/weights/permutation out; permute: X in, permuted
+    # rows out; combine: weighted rows in, y out) against the measured copy bandwidth
+    hbm_bytes = {"route_permute": 4.0 * M * E + 16.0 * R + 2.0 * M * H + 2.0 * R * H, "combine": 2.0 * R * H + 2.0 * M * H}
+    for lab, nbytes in hbm_bytes.items():
+        gbs = nbytes / (detail[lab]["avg_us"] * 1e-6) / 1e9
+        detail[lab].update({"bound": "hbm", "algorithmic_bytes": nbytes, "gbs": gbs, "frac_of_measured_hbm": gbs / peak_hbm})
     dq = [0.0, 0.0, 0]
     for lab, v in agg.items():
         if lab.startswith("dense_q8_"):
