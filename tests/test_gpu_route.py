@@ -21,11 +21,20 @@ def _ties_logits(M, E, seed):
     return l
 
 
+def _extreme_logits(M, E, seed):
+    """Finite extremes: huge magnitudes of both signs, subnormals, both zeros, ordinary values, many ties."""
+    rng = np.random.default_rng(seed)
+    pool = np.array([3.0e38, -3.0e38, 1.0e-45, -1.0e-45, 0.0, -0.0, 1.5, -1.5, 1.17549435e-38, -7.0, 65504.0],
+                    dtype=np.float32)
+    return pool[rng.integers(0, pool.size, size=(M, E))]
+
+
 CASES = [
     ("uniform-2048", 2048, 128, 8, "uniform"), ("skewed-2048", 2048, 128, 8, "skewed"),
     ("skewed-128", 128, 128, 8, "skewed"), ("ties", 257, 128, 8, "ties"), ("ragged", 33, 16, 16, "ties"),
     ("k1", 100, 8, 1, "uniform"), ("odd-E", 77, 5, 3, "ties"), ("E1024", 40, 1024, 8, "uniform"),
     ("k40", 65, 64, 40, "uniform"), ("one-token", 1, 128, 8, "uniform"), ("uniform-8192", 8192, 128, 8, "uniform"),
+    ("extremes", 200, 96, 6, "extremes"),
 ]
 
 
@@ -33,6 +42,8 @@ CASES = [
 def test_route_bit_exact(name, M, E, k, kind):
     if kind == "ties":
         logits = _ties_logits(M, E, seed=M + E)
+    elif kind == "extremes":
+        logits = _extreme_logits(M, E, seed=M + E)
     else:
         logits = synth.router_logits(M, E, seed=0, hot_bias=synth.SKEW_HOT_BIAS if kind == "skewed" else 0.0)
     H = 64
