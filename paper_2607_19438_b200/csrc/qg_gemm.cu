@@ -66,11 +66,10 @@ struct GemmParams {
 
 template <int QBITS, int BT>
 struct Cfg {
-    static constexpr int SX = 8;                                   // k-block stages: one ring index for the activation tile
-                                                                   // (smem), the packed weights (smem), the dequantised
-                                                                   // weights (TMEM) and the full/done barriers
-    static constexpr int SR = (QBITS == 4 && BT <= 192) ? 16 : 8;   // packed-weight stages (refilled four at a time); the
-                                                                   // 4-bit tile is half the size, so its ring can be twice as deep
+    static constexpr int SX = 8;                                   // k-block stages: ring of the activation tile (smem)
+                                                                   // and of the full/done barriers
+    static constexpr int SR = (QBITS == 4 && BT <= 192) ? 16 : 8;  // packed-weight stages (smem, refilled four at a time):
+                                                                   // twice as deep for 4-bit tiles where shared memory allows
     static constexpr int NACC = (BT > 192) ? 1 : 2;                // accumulators in tensor memory
     static constexpr int SA = ((512 - NACC * BT) / 32 >= 8) ? 8 : (512 - NACC * BT) / 32;   // dequantised-weight stages in
                                                                    // tensor memory (8, or what two accumulators leave)
