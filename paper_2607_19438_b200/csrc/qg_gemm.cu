@@ -789,13 +789,14 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const vo
                           CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc != QG_OK) return rc;
     auto kern = qgemm_kernel<QBITS, BT, EPI>;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {false};      // per device: the attribute belongs to the function on one device
+    const int dv = ctx->device;
+    if (dv < 0 || dv >= 64 || !attr_set[dv]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
             cudaGetLastError();
             return QG_ERR_CUDA;
         }
-        attr_set = true;
+        if (dv >= 0 && dv < 64) attr_set[dv] = true;
     }
     // Upper bound on the number of pair tiles (the exact count lives on the device for grouped calls).
     const long long max_tiles =
