@@ -318,16 +318,18 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     volatile int* abort_flag = misc + 1;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < C::SX; ++s) { mbar_init(full(s), 1 + 8); mbar_init(done(s), 1); }
-        for (int s = 0; s < C::SR; ++s) { mbar_init(r_full(s), 1); mbar_init(r_empty(s), 4); }
+    if (warp == 0) {   // barrier initialisation spread over the lanes of one warp (a single thread needs ~50 steps)
+        if (lane < C::SX) { mbar_init(full(lane), 1 + 8); mbar_init(done(lane), 1); }
+        if (lane < C::SR) { mbar_init(r_full(lane), 1); mbar_init(r_empty(lane), 4); }
         // an accumulator is released by the 4 epilogue + 16 dequantising warps of both CTAs
-        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 2); mbar_init(acc_empty(s), C::HELP ? 40 : 8); }
-        misc[1] = 0;
+        if (lane >= 16 && lane < 18) { mbar_init(acc_full(lane - 16), 2); mbar_init(acc_empty(lane - 16), C::HELP ? 40 : 8); }
+        if (lane == 31) misc[1] = 0;
         fence_mbar_init();
         fence_proxy_async_smem();
+        if (lane == 30) prefetch_tmap(&tm_x);
+        if (lane == 29) prefetch_tmap(&tm_w);
+        if (lane == 28) prefetch_tmap(&tm_s);
     }
-    if (warp == 0 && lane == 0) { prefetch_tmap(&tm_x); prefetch_tmap(&tm_w); prefetch_tmap(&tm_s); }
     if (warp == 3) {
         tmem_alloc_pair(sbase + C::OFF_MISC, C::TMEM_COLS);
         tmem_relinquish_pair();
