@@ -115,10 +115,32 @@ route_scan_kernel(int nb, int E, int32_t* __restrict__ block_hist, int32_t* __re
         if (g == 0) { counts[e] = total; tot[e] = total; }
     }
     __syncthreads();
-    if (threadIdx.x == 0) {  // E <= 1024: a serial prefix over shared memory is a few microseconds
-        int run = 0;
-        for (int i = 0; i < E; ++i) { offsets[i] = run; run += tot[i]; }
-        offsets[E] = run;
+    // offsets = exclusive prefix of the totals over the experts: warp scans, then a scan of the 32 warp sums
+    {
+        const int i = threadIdx.x, lane = i & 31, wp = i >> 5;
+        const int v = (i < E) ? tot[i] : 0;
+        int inc = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int u = __shfl_up_sync(0xFFFFFFFFu, inc, off);
+            if (lane >= off) inc += u;
+        }
+        __syncthreads();                       // tot is re-used for the warp sums
+        if (lane == 31) part[wp] = inc;
+        __syncthreads();
+        if (wp == 0) {
+            const int ws = part[lane];
+            int winc = ws;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int u = __shfl_up_sync(0xFFFFFFFFu, winc, off);
+                if (lane >= off) winc += u;
+            }
+            part[32 + lane] = winc - ws;        // exclusive prefix of the warp sums
+            if (lane == 31) offsets[E] = winc;
+        }
+        __syncthreads();
+        if (i < E) offsets[i] = part[32 + wp] + inc - v;
     }
 }
 
