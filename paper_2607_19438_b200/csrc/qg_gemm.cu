@@ -221,15 +221,15 @@ __device__ __forceinline__ float lds_scale(uint32_t addr) {
 // single-accumulator tile, by the sixteen dequantising warps, which would otherwise idle at the tile boundary.
 __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int tok_end, int n_base, uint32_t taddr,
                                             int n_epi, int pid, int npart, __nv_bfloat16* st, int lane) {
-    __nv_bfloat16* outb = static_cast<__nv_bfloat16*>(p.out);
+    // The loop is issue-bound (five warps of a scheduler drain together), so everything that does not depend on the
+    // block is computed once: the lane's two shared-memory read addresses, its global pointer and its token limit.
     const int nblk = n_epi >> 4;
+    int b = pid;
+    if (b >= nblk) return;
     const bool weighted = (p.mode == QG_MODE_DOWN_WEIGHTED);
     uint32_t v0[8], v1[8];                       // TMEM lanes 0-15 / 16-31 of this warp's quarter
-    int b = pid;
-    if (b < nblk) {
-        tmem_ld_16x256_x2(taddr + 16 * b, v0);
-        tmem_ld_16x256_x2(taddr + (16u << 16) + 16 * b, v1);
-    }
+    tmem_ld_16x256_x2(taddr + 16 * b, v0);
+    tmem_ld_16x256_x2(taddr + (16u << 16) + 16 * b, v1);
     // Routing weights of the whole tile, fetched once (two dependent global loads, all in flight together): lane l
     // holds the weights of tokens l, l + 32, ... of the tile.
     float wt8[8];
@@ -240,31 +240,45 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
             wt8[j] = (32 * j < n_epi && tokl < tok_end) ? p.topk_w[p.row_pair[tokl]] : 0.f;
         }
     }
-    const uint32_t st_s = smem_u32(st);
-    const uint32_t st_row = st_s + (lane & 7) * 64 + (((lane >> 3) ^ ((lane >> 1) & 3)) << 4);   // matrix lane>>3, token lane&7
+    const uint32_t st_row = smem_u32(st) + (lane & 7) * 64 + (((lane >> 3) ^ ((lane >> 1) & 3)) << 4);   // matrix lane>>3, token lane&7
     const int c = 2 * (lane & 3);                // this thread's token pairs: c, c + 1 and 8 + c, 9 + c of the block
+    // store side: this lane moves tokens tk and 8 + tk of every block, 16 bytes (8 rows from n) each
+    const int tk = lane >> 2, c4 = lane & 3;
+    const int n = n_base + c4 * 8;
+    const uint4* s_lo = reinterpret_cast<const uint4*>(st + tk * 32 + ((c4 ^ ((tk >> 1) & 3)) << 3));
+    const uint4* s_hi = s_lo + 32;               // token 8 + tk: 512 bytes on, same swizzle
+    const size_t row8 = static_cast<size_t>(8) * p.N;
+    __nv_bfloat16* g = static_cast<__nv_bfloat16*>(p.out) + static_cast<size_t>(tok0 + 16 * b + tk) * p.N + n;
+    const size_t g_step = 2 * row8 * npart;
+    int left = (n < p.N) ? (tok_end - tok0 - 16 * b - tk) : 0;   // tokens tk, 8 + tk of the block are stored if 0, 8 < left
+    const int left_step = 16 * npart;
     while (b < nblk) {
-        float w0 = 1.f, w1 = 1.f, w2 = 1.f, w3 = 1.f;
+        tmem_ld_wait();
+        uint32_t pk[8];
         if (weighted) {
             const int j = b >> 1;                // tokens 16 b .. 16 b + 15 live in register j, lanes 16 (b & 1) ..
             float wv = wt8[0];
 #pragma unroll
             for (int jj = 1; jj < 8; ++jj) wv = (j == jj) ? wt8[jj] : wv;
             const int src = 16 * (b & 1) + c;
-            w0 = __shfl_sync(0xFFFFFFFFu, wv, src);
-            w1 = __shfl_sync(0xFFFFFFFFu, wv, src + 1);
-            w2 = __shfl_sync(0xFFFFFFFFu, wv, src + 8);
-            w3 = __shfl_sync(0xFFFFFFFFu, wv, src + 9);
-        }
-        tmem_ld_wait();
-        uint32_t pk[8];
+            const float w0 = __shfl_sync(0xFFFFFFFFu, wv, src), w1 = __shfl_sync(0xFFFFFFFFu, wv, src + 1);
+            const float w2 = __shfl_sync(0xFFFFFFFFu, wv, src + 8), w3 = __shfl_sync(0xFFFFFFFFu, wv, src + 9);
 #pragma unroll
-        for (int g = 0; g < 2; ++g) {            // tokens 8 g .. 8 g + 7
-            const float wa = g ? w2 : w0, wb = g ? w3 : w1;
-            pk[4 * g + 0] = bf16x2(__uint_as_float(v0[4 * g + 0]) * wa, __uint_as_float(v0[4 * g + 1]) * wb);
-            pk[4 * g + 1] = bf16x2(__uint_as_float(v0[4 * g + 2]) * wa, __uint_as_float(v0[4 * g + 3]) * wb);
-            pk[4 * g + 2] = bf16x2(__uint_as_float(v1[4 * g + 0]) * wa, __uint_as_float(v1[4 * g + 1]) * wb);
-            pk[4 * g + 3] = bf16x2(__uint_as_float(v1[4 * g + 2]) * wa, __uint_as_float(v1[4 * g + 3]) * wb);
+            for (int gq = 0; gq < 2; ++gq) {     // tokens 8 gq .. 8 gq + 7
+                const float wa = gq ? w2 : w0, wb = gq ? w3 : w1;
+                pk[4 * gq + 0] = bf16x2(__uint_as_float(v0[4 * gq + 0]) * wa, __uint_as_float(v0[4 * gq + 1]) * wb);
+                pk[4 * gq + 1] = bf16x2(__uint_as_float(v0[4 * gq + 2]) * wa, __uint_as_float(v0[4 * gq + 3]) * wb);
+                pk[4 * gq + 2] = bf16x2(__uint_as_float(v1[4 * gq + 0]) * wa, __uint_as_float(v1[4 * gq + 1]) * wb);
+                pk[4 * gq + 3] = bf16x2(__uint_as_float(v1[4 * gq + 2]) * wa, __uint_as_float(v1[4 * gq + 3]) * wb);
+            }
+        } else {
+#pragma unroll
+            for (int gq = 0; gq < 2; ++gq) {
+                pk[4 * gq + 0] = bf16x2(__uint_as_float(v0[4 * gq + 0]), __uint_as_float(v0[4 * gq + 1]));
+                pk[4 * gq + 1] = bf16x2(__uint_as_float(v0[4 * gq + 2]), __uint_as_float(v0[4 * gq + 3]));
+                pk[4 * gq + 2] = bf16x2(__uint_as_float(v1[4 * gq + 0]), __uint_as_float(v1[4 * gq + 1]));
+                pk[4 * gq + 3] = bf16x2(__uint_as_float(v1[4 * gq + 2]), __uint_as_float(v1[4 * gq + 3]));
+            }
         }
         const int bn = b + npart;
         if (bn < nblk) {                         // next block, overlapped with the stores below
@@ -274,19 +288,15 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
         stmatrix_x4_trans(st_row, pk[0], pk[1], pk[2], pk[3]);
         stmatrix_x4_trans(st_row + 512, pk[4], pk[5], pk[6], pk[7]);
         __syncwarp();
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-            const int tk = i * 8 + (lane >> 2), c4 = lane & 3;
-            const int tok = tok0 + 16 * b + tk;
-            const int n = n_base + c4 * 8;
-            if (tok < tok_end && n < p.N)
-                *reinterpret_cast<uint4*>(outb + static_cast<size_t>(tok) * p.N + n) =
-                    *reinterpret_cast<const uint4*>(st + tk * 32 + ((c4 ^ ((tk >> 1) & 3)) << 3));
-        }
+        if (left > 0) *reinterpret_cast<uint4*>(g) = *s_lo;
+        if (left > 8) *reinterpret_cast<uint4*>(g + row8) = *s_hi;
         __syncwarp();
+        g += g_step;
+        left -= left_step;
         b = bn;
     }
 }
+
 // EPI: 0 plain / routing-weighted bf16 store, 1 gate/up + SiLU, 2 weighted fp32 atomic accumulate (compiled apart so
 // that each instantiation carries one epilogue only).
 template <int QBITS, int BT, int EPI>
