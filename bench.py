@@ -35,9 +35,17 @@ METRIC = "Q4/Q8 prefill GEMM TFLOP/s & tok/s (dense+MoE), % of B200 bf16 tensor 
 M_TOKENS = 2048
 DENSE_SET = [("qkv", 2560, 2048), ("o", 2048, 2048), ("gate_up", 16384, 2048), ("down", 2048, 8192)]  # (name, N, K)
 MOE = dict(H=2048, E=128, k=8, F=768)
-# DRAM bytes (read + written) per launch of qgemm_kernel from one ncu capture of this step, averaged over the captured
-# launches (profiles/qgemm_kernel_bench_step_ncu_full.md).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 107.0e6
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "qgemm_kernel_bench_step_traffic.json")
+
+
+def ncu_traffic():
+    """DRAM bytes (read + written) per launch of the GEMM kernel, quoted from the ncu capture of this step that the
+    tracked data file records (with the commit it was taken at); None if the file is missing."""
+    try:
+        d = json.load(open(TRAFFIC_FILE))
+        return float(d["dram_bytes_per_launch"]), d.get("captured_at_commit"), d.get("source")
+    except Exception:
+        return None, None, None
 
 
 def dense_flops(M):
@@ -46,6 +54,13 @@ def dense_flops(M):
 
 def moe_flops(M):
     return 2.0 * M * MOE["k"] * 3 * MOE["F"] * MOE["H"]
+
+
+def sustained_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path)).get("bf16_tflops_sustained", 1400.0))
+    return 1400.0
 
 
 def measured_peaks():
@@ -161,6 +176,137 @@ class ClockSampler:
         return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "power_w_max": float(max(pw)),
                 "samples": len(sm), "reasons": sorted(reasons)}
 
+
+
+# ------------------------------------------------------------------------------------------ config sweep
+LAYER_SETS = {   # (label, N, K) of the four projections of one transformer layer
+    "cfg1_q8": (8, [("qkv", 2560, 2048), ("o", 2048, 2048), ("gate_up", 16384, 2048), ("down", 2048, 8192)]),
+    "cfg2_q4": (4, [("qkv", 5120, 3072), ("o", 3072, 3072), ("gate_up", 16384, 3072), ("down", 3072, 8192)]),
+    "cfg4_q8": (8, [("qkv", 6144, 4096), ("o", 4096, 4096), ("gate_up", 28672, 4096), ("down", 4096, 14336)]),
+}
+SWEEP_DENSE = [("cfg1_q8", 1024), ("cfg1_q8", 2048), ("cfg2_q4", 1024), ("cfg2_q4", 2048), ("cfg4_q8", 2048), ("cfg4_q8", 8192)]
+SWEEP_MOE = [(1024, False), (2048, False), (2048, True), (8192, False), (8192, True)]
+L2_BYTES = 126e6
+
+
+def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
+    """Every configuration of the config list beside the headline one, each call timed with its own CUDA-event pair on
+    the launching stream.  Inputs are seeded and drawn on the device (torch generator, seed 0) with the value
+    distributions of the host generator: int8 uniform -127..127 / nibbles uniform 0..15, fp16 scales |N(0,0.02)|/qmax,
+    bf16 N(0,1) activations, fp32 N(0,1) logits (+0.80 on every fourth expert when skewed).  Dense weights rotate
+    through enough copies that the working set exceeds twice the L2; the MoE layer streams 340 MB per pass."""
+    import ctypes as C
+    P = lambda t: C.c_void_p(t.data_ptr())
+    S = C.c_void_p(stream.cuda_stream)
+    g = torch.Generator(device=dev); g.manual_seed(0)
+
+    def chk(rc, what):
+        if rc != 0:
+            raise qg.QGemmError(rc, what)
+
+    def weights(qbits, N, K):
+        if qbits == 8:
+            q = torch.randint(-127, 128, (N, K), dtype=torch.int8, device=dev, generator=g)
+        else:
+            q = torch.randint(0, 256, (N, K // 2), dtype=torch.uint8, device=dev, generator=g)
+        sc = (torch.randn((N, K // 32), device=dev, generator=g).abs() * (0.02 / (127 if qbits == 8 else 7))).to(torch.float16)
+        return q, sc
+
+    def timed_calls(calls, n_iter):
+        """calls: list of (label, flops, bytes, fn(it)).  Returns {label: [total_ms, flops, bytes]} over n_iter passes."""
+        for it in range(3):
+            for _, _, _, fn in calls:
+                fn(it)
+        torch.cuda.synchronize()
+        evs = []
+        for it in range(n_iter):
+            for lab, fl, nb, fn in calls:
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(stream); fn(it); e1.record(stream)
+                evs.append((lab, fl, nb, e0, e1))
+        torch.cuda.synchronize()
+        agg = {}
+        for lab, fl, nb, e0, e1 in evs:
+            d = agg.setdefault(lab, [0.0, fl, nb])
+            d[0] += e0.elapsed_time(e1)
+        return agg
+
+    out = {"method": "one CUDA-event pair per call on the launching stream, 3 warm-up + %d timed passes per configuration, "
+                     "dense weights rotated through copies exceeding 2x L2, inputs drawn on the device (seed 0)" % iters,
+           "peak_tflops": peak_tf, "dense": [], "moe": []}
+    for name, M in SWEEP_DENSE:
+        qbits, layers = LAYER_SETS[name]
+        wbytes = sum(N * K * (1.0625 if qbits == 8 else 0.5625) for _, N, K in layers)
+        ncopy = max(2, int(2 * L2_BYTES // wbytes) + 1)
+        W = [[weights(qbits, N, K) for _, N, K in layers] for _ in range(ncopy)]
+        A = {K: torch.randn((M, K), device=dev, generator=g).to(torch.bfloat16) for K in {K for _, _, K in layers}}
+        Cs = [torch.empty((M, N), dtype=torch.bfloat16, device=dev) for _, N, _ in layers]
+        calls = []
+        for i, (lab, N, K) in enumerate(layers):
+            def fn(it, i=i, N=N, K=K):
+                q, sc = W[it % ncopy][i]
+                chk(lib.qgemm_dense(ctx, qbits, M, N, K, P(A[K]), P(q), P(sc), P(Cs[i]), S), "qgemm_dense")
+            calls.append((lab, 2.0 * M * N * K, 0.0, fn))
+        n_it = iters if M * sum(N * K for _, N, K in layers) < 2e12 else max(5, iters // 2)
+        agg = timed_calls(calls, n_it)
+        tot_ms = sum(v[0] for v in agg.values()); tot_fl = sum(v[1] for v in agg.values()) * n_it
+        row = {"set": name, "M": M, "weight_copies": ncopy,
+               "gemm_tflops": {lab: v[1] * n_it / (v[0] * 1e-3) / 1e12 for lab, v in agg.items()},
+               "gemm_us": {lab: v[0] / n_it * 1e3 for lab, v in agg.items()},
+               "set_tflops": tot_fl / (tot_ms * 1e-3) / 1e12, "tok_per_s": M * n_it / (tot_ms * 1e-3)}
+        row["frac_of_measured_peak"] = row["set_tflops"] / peak_tf
+        out["dense"].append(row)
+        del W, A, Cs
+        torch.cuda.empty_cache()
+
+    H, E, k, F = MOE["H"], MOE["E"], MOE["k"], MOE["F"]
+    W1q, W1s = weights(4, E * 2 * F, H); W2q, W2s = weights(4, E * H, F)
+    i32 = dict(dtype=torch.int32, device=dev)
+    for M, skewed in SWEEP_MOE:
+        R = M * k
+        L = torch.randn((M, E), device=dev, generator=g)
+        if skewed:
+            L[:, ::4] += 0.80
+        X = torch.randn((M, H), device=dev, generator=g).to(torch.bfloat16)
+        ws = torch.empty(max(16, qg.route_workspace_bytes(M, E, k)), dtype=torch.uint8, device=dev)
+        o = dict(idx=torch.empty((M, k), **i32), w=torch.empty((M, k), dtype=torch.float32, device=dev),
+                 counts=torch.empty(E, **i32), offsets=torch.empty(E + 1, **i32), row_pair=torch.empty(R, **i32),
+                 pair_row=torch.empty(R, **i32), Xp=torch.empty((R, H), dtype=torch.bfloat16, device=dev),
+                 Hh=torch.empty((R, F), dtype=torch.bfloat16, device=dev),
+                 Dw=torch.empty((R, H), dtype=torch.bfloat16, device=dev), y=torch.empty((M, H), dtype=torch.bfloat16, device=dev))
+        calls = [
+            ("route_permute", 0.0, 4.0 * M * E + 16.0 * R + 2.0 * M * H + 2.0 * R * H, lambda it: chk(lib.moe_route(
+                ctx, M, E, k, P(L), P(o["idx"]), P(o["w"]), P(o["counts"]), P(o["offsets"]), P(o["row_pair"]),
+                P(o["pair_row"]), P(X), P(o["Xp"]), H, P(ws), ws.numel(), S), "moe_route")),
+            ("gate_up", 2.0 * R * 2 * F * H, 0.0, lambda it: chk(lib.moe_grouped_qgemm(
+                ctx, qg.MODE_GATE_UP_SILU, 4, R, E, 2 * F, H, P(o["Xp"]), P(o["offsets"]), P(W1q), P(W1s), None, None, k,
+                P(o["Hh"]), S), "gate/up")),
+            ("down", 2.0 * R * F * H, 0.0, lambda it: chk(lib.moe_grouped_qgemm(
+                ctx, qg.MODE_DOWN_WEIGHTED, 4, R, E, H, F, P(o["Hh"]), P(o["offsets"]), P(W2q), P(W2s), P(o["w"]),
+                P(o["row_pair"]), k, P(o["Dw"]), S), "down")),
+            ("combine", 0.0, 2.0 * R * H + 2.0 * M * H, lambda it: chk(lib.moe_combine(
+                ctx, M, k, H, P(o["Dw"]), qg.D_BF16, P(o["pair_row"]), None, P(o["y"]), S), "combine")),
+        ]
+        n_it = iters if M <= 2048 else max(5, iters // 2)
+        agg = timed_calls(calls, n_it)
+        gemm_ms = agg["gate_up"][0] + agg["down"][0]
+        gemm_fl = (agg["gate_up"][1] + agg["down"][1]) * n_it
+        tot_ms = sum(v[0] for v in agg.values())
+        # composite bound of the two grouped GEMMs: the tensor time at the measured peak or the time to stream the
+        # 340 MB of expert weights once from HBM, whichever is longer
+        t_tensor = gemm_fl / n_it / (peak_tf * 1e12)
+        t_hbm = (E * 3 * F * H * 0.5625) / (peak_hbm * 1e9)
+        row = {"M": M, "routing": "skewed" if skewed else "uniform", "rows_per_expert": R / E,
+               "gemm_tflops": {lab: agg[lab][1] * n_it / (agg[lab][0] * 1e-3) / 1e12 for lab in ("gate_up", "down")},
+               "call_us": {lab: v[0] / n_it * 1e3 for lab, v in agg.items()},
+               "gemms_tflops": gemm_fl / (gemm_ms * 1e-3) / 1e12, "layer_tok_per_s": M * n_it / (tot_ms * 1e-3),
+               "hbm_gbs": {lab: agg[lab][2] * n_it / (agg[lab][0] * 1e-3) / 1e9 for lab in ("route_permute", "combine")},
+               "composite_bound_us": max(t_tensor, t_hbm) * 1e6,
+               "bound": "hbm (expert weights)" if t_hbm > t_tensor else "tensor"}
+        row["frac_of_measured_peak"] = row["gemms_tflops"] / peak_tf
+        row["frac_of_composite_bound"] = max(t_tensor, t_hbm) / (gemm_ms / n_it * 1e-3)
+        out["moe"].append(row)
+    return out
 
 # ------------------------------------------------------------------------------------------ GPU arm
 def run_ours(args):
@@ -290,6 +436,14 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
     qg.poll_status()
     flops_step = dense_flops(M) + moe_flops(M)
+    # sustained: the same step back to back for at least two seconds, with its own clock record (the board's power
+    # cap pulls the SM clock down after a few hundred milliseconds of this load)
+    sus_steps = int(min(20000, max(200, 2200.0 / (ms / args.steps))))
+    sampler2 = ClockSampler(local) if rank == 0 else None
+    ms_sus = timed(lambda: step(dA, dL, dX), sus_steps)
+    clocks_sus = sampler2.stop() if sampler2 else None
+    qg.poll_status()
+    time.sleep(1.0)
     value = world * flops_step * args.steps / (ms * 1e-3) / 1e12
 
     # per-kernel figures from the events recorded inside the timed region
@@ -316,9 +470,17 @@ def run_ours(args):
         if v[0]:
             gk[0] += v[0]; gk[1] += v[1]; gk[2] += v[2]
     achieved = gk[0] / (gk[1] * 1e-3) / 1e12
+    # algorithmic bytes of the six GEMM launches (weights + scales + activations in + output), averaged per launch
+    alg = [N * K * 1.0625 + 2.0 * M * K + 2.0 * M * N for _, N, K in DENSE_SET]
+    alg.append(E * 2 * F * H * 0.5625 + 2.0 * R * H + 2.0 * R * F)
+    alg.append(E * H * F * 0.5625 + 2.0 * R * F + 2.0 * R * H)
+    alg_bytes_per_launch = sum(alg) / len(alg)
     roofline = {"kernel": "qgemm_kernel (all instantiations: 4 qgemm_dense + 2 moe_grouped_qgemm launches per step)",
                 "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
-                "peak_source": peak_src, "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "peak_source": peak_src, "traffic": ncu_traffic()[0],
+                "traffic_source": {"kind": "quoted from an ncu capture, not measured by this run", "file": os.path.relpath(TRAFFIC_FILE, ROOT),
+                                   "captured_at_commit": ncu_traffic()[1]},
+                "algorithmic_bytes_per_launch": alg_bytes_per_launch,
                 "avg_launch_us": gk[1] / gk[2] * 1e3, "flops_per_launch": gk[0] / gk[2],
                 "dense_q8_only": {"achieved": dq[0] / (dq[1] * 1e-3) / 1e12, "frac": dq[0] / (dq[1] * 1e-3) / 1e12 / peak_tf}}
     gemm_ms = sum(v[1] for lab, v in agg.items() if v[0])
@@ -383,6 +545,12 @@ def run_ours(args):
     d2h = sum(c.numel() * 2 for c in hC) + hY.numel() * 2
     e2e_val = world * flops_step * e2e_steps / (ms_e2e * 1e-3) / 1e12
 
+    sweep = None
+    if world == 1 and not args.no_sweep:
+        del inA, inL, inX, outC2, outY2
+        torch.cuda.empty_cache()
+        sweep = run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm)
+        qg.poll_status()
     if rank == 0:
         dense_h0, moe_h0 = dense_h, moe_h
         cpu = cpu_baseline(dense_h0, moe_h0) if world == 1 else None
@@ -398,6 +566,12 @@ def run_ours(args):
             "gemm_only": {"tflops": gemm_fl / (gemm_ms * 1e-3) / 1e12, "frac_of_peak": gemm_fl / (gemm_ms * 1e-3) / 1e12 / peak_tf},
             "frac_of_measured_bf16_peak": value / world / peak_tf, "frac_of_nominal_2250": value / world / 2250.0,
             "roofline": roofline, "kernels": detail, "clocks": clocks,
+            "per_kernel_region": "a separate region of %d steps with an event pair around every call, started after a "
+                                 "1 s pause so that it runs at burst clocks like the headline region" % ev_steps,
+            "sustained": {"steps": sus_steps, "seconds": ms_sus * 1e-3, "ms_per_step": ms_sus / sus_steps,
+                          "tflops": world * flops_step * sus_steps / (ms_sus * 1e-3) / 1e12,
+                          "frac_of_sustained_peak": flops_step * sus_steps / (ms_sus * 1e-3) / 1e12 / sustained_peak(),
+                          "sustained_peak_tflops": sustained_peak(), "clocks": clocks_sus},
             "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": ms_e2e / e2e_steps, "steps": e2e_steps,
                     "overlap": "steps pipelined on three streams (copy in / compute / copy out), two buffer sets"},
@@ -405,6 +579,8 @@ def run_ours(args):
         }
         if cpu is not None:
             line["cpu_baseline"] = cpu
+        if sweep is not None:
+            line["sweep"] = sweep
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -416,6 +592,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-sweep", action="store_true", help="skip the per-configuration sweep block")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

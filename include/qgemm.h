@@ -12,10 +12,13 @@
  *   - all data pointers are DEVICE pointers owned by the caller; the library never allocates,
  *     frees or synchronises inside a compute call; the call is asynchronous on `stream`
  *     (a cudaStream_t passed as void*; NULL = the legacy default stream);
+ *   - the context's device must be the calling thread's current device (else QG_ERR_DEVICE); a
+ *     context and its calls belong to one host thread and one stream at a time (it caches tensor
+ *     maps and owns the split-K scratch of qgemm_dense);
  *   - return value: QG_OK (0) or a negative QG_ERR_* code; an error is detected before anything is
  *     launched, so the outputs are untouched; nothing aborts, traps or throws;
  *   - there is no fallback path: a shape the kernels do not accept is an error (the paper's
- *     Sec. 3.2 "shape constraints" check, without its SIMD fallback);
+ *     Sec. 3.2 dispatch-time shape check, without the fallback kernels it falls back to);
  *   - device-side waits are bounded; a wait that expires records QG_ERR_TIMEOUT in the context's
  *     status word, the kernel exits cleanly and qg_poll_status() reports it.
  *
@@ -54,7 +57,8 @@ enum {
     QG_ERR_ARCH = -5,      /* the device is not compute capability 10.x */
     QG_ERR_CUDA = -6,      /* a CUDA runtime / driver call failed */
     QG_ERR_TIMEOUT = -7,   /* a bounded device-side wait expired (reported by qg_poll_status) */
-    QG_ERR_TOO_LARGE = -8  /* the problem does not fit the library's built-in scratch (moe_route_static) */
+    QG_ERR_TOO_LARGE = -8, /* the problem does not fit the library's built-in scratch (moe_route_static) */
+    QG_ERR_DEVICE = -9     /* the calling thread's current CUDA device is not the context's device */
 };
 enum { QG_Q8 = 8, QG_Q4 = 4 };
 enum {
@@ -65,7 +69,8 @@ enum {
 };
 enum { QG_D_BF16 = 0, QG_D_F32_ACC = 1 };
 
-/* Create / destroy a context for `device` (these two may allocate a few bytes of device memory). */
+/* Create / destroy a context for `device`.  Only these two allocate device memory (the status word and the
+ * split-K scratch of qgemm_dense, about 20 MB); qg_create leaves the caller's current device as it was. */
 int qg_create(qg_ctx** out, int device);
 int qg_destroy(qg_ctx* ctx);
 const char* qg_strerror(int code);
@@ -75,15 +80,25 @@ int qg_poll_status(qg_ctx* ctx, void* stream);
 size_t qg_route_workspace_bytes(int M, int E, int k);
 
 /*
- * Dense quantised GEMM (Sec. 3.1, "Dense GEMM ... in 4-bit and 8-bit quantisation, reading the
- * packed-quant weight layout"):  C[m, n] = sum_k A[m, k] * q[n, k] * scale[n, k/32].
+ * Testing hook (no counterpart in the paper): the GEMM kernels' device-side waits give up after
+ * `wait_limit_polls` polls (0 restores the default, about a second), and the next GEMM launch on this
+ * context leaves out the activation load of k-block `skip_kblock` of each CTA's first tile (-1: none), so
+ * that a wait in that launch runs out.  The launch then returns normally and qg_poll_status() reports
+ * QG_ERR_TIMEOUT; the context stays usable.  Never needed in production.
+ */
+int qg_test_inject(qg_ctx* ctx, unsigned wait_limit_polls, int skip_kblock);
+
+/*
+ * Dense quantised GEMM (Sec. 3.1: the dense projection over 4-bit / 8-bit block-quantised weights, read in
+ * their packed layout without a separate dequantisation pass):
+ *   C[m, n] = sum_k A[m, k] * q[n, k] * scale[n, k/32].
  *   qbits QG_Q8 or QG_Q4; A bf16 [M, K]; Wq / Wscale as above; C bf16 [M, N] (overwritten).
  */
 int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq,
                 const void* Wscale, void* C, void* stream);
 
 /*
- * Routing (the paper only says "routed tokens", Sec. 3.1; defined here): for every token the k
+ * Routing (Sec. 3.1 only presupposes that tokens have been assigned to experts; defined here): for every token the k
  * experts that come first in the order (logit descending, expert index ascending), in that order;
  * topk_w = softmax over those k logits (fp32).  Then the per-expert histogram, its exclusive
  * prefix sum (expert_offsets[E] = M*k) and the stable counting sort of the pair ids p = t*k + s by
@@ -127,8 +142,9 @@ int moe_permute(qg_ctx* ctx, int M, int k, int H, const void* X, const int32_t* 
                 void* stream);
 
 /*
- * Grouped quantised GEMM over expert segments (Sec. 3.1, "MoE expert GEMM" and "Fused MoE gate/up
- * projection ... applies the SiLU activation on the tensor-core accumulators"): rows
+ * Grouped quantised GEMM over expert segments (Sec. 3.1: the per-expert projection over that expert's routed
+ * tokens, and the gate/up projection whose SiLU gating is applied to the accumulators before anything is
+ * written out): rows
  * r in [expert_offsets[e], expert_offsets[e+1]) of Ain (bf16 [R, K], permuted order) are multiplied
  * by expert e's weights (Wq [E, N, K or K/2], Wscale fp16 [E, N, K/32]).  `mode` selects the epilogue
  * (see QG_MODE_*).  In mode 1 rows 0..F-1 of an expert's weights are the gate and F..2F-1 the up

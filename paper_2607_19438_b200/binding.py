@@ -18,7 +18,8 @@ QG_Q8, QG_Q4 = 8, 4
 MODE_PLAIN, MODE_GATE_UP_SILU, MODE_DOWN_WEIGHTED, MODE_DOWN_ACCUM_F32 = 0, 1, 2, 3
 D_BF16, D_F32_ACC = 0, 1
 
-EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_route_workspace_bytes", "qgemm_dense",
+EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_route_workspace_bytes",
+           "qgemm_dense",
            "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_combine"]
 
 
@@ -46,6 +47,7 @@ def load():
         lib.qg_create.argtypes = [C.POINTER(C.c_void_p), C.c_int]
         lib.qg_destroy.argtypes = [C.c_void_p]
         lib.qg_poll_status.argtypes = [C.c_void_p, C.c_void_p]
+        lib.qg_test_inject.argtypes = [C.c_void_p, C.c_uint, C.c_int]
         vp, ci = C.c_void_p, C.c_int
         lib.qgemm_dense.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
         lib.moe_route.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp, C.c_size_t, vp]
@@ -95,6 +97,17 @@ def poll_status():
     _check(load().qg_poll_status(context(), _stream()), "qg_poll_status")
 
 
+def poll_status_code() -> int:
+    """Synchronises the current stream; returns (and clears) the device status word instead of raising."""
+    return int(load().qg_poll_status(context(), _stream()))
+
+
+def test_inject(wait_limit_polls: int = 0, skip_kblock: int = -1):
+    """Testing hook: bounded-wait limit in polls (0 = default) and the k-block whose activation load the next GEMM
+    launch leaves out (-1 = none)."""
+    _check(load().qg_test_inject(context(), wait_limit_polls, skip_kblock), "qg_test_inject")
+
+
 def route_workspace_bytes(M, E, k) -> int:
     return int(load().qg_route_workspace_bytes(M, E, k))
 
@@ -110,48 +123,45 @@ def qgemm_dense(qbits, A, Wq, Wscale, out=None):
     return out
 
 
-def moe_route(logits, k, X=None, ws=None):
+def _route_outputs(M, E, k, H, dev, X, out):
+    """The output tensors of a routing call: the caller's (`out`, a dict with the same keys) or fresh ones."""
+    if out is not None:
+        return out
+    i32 = dict(dtype=torch.int32, device=dev)
+    o = dict(topk_idx=torch.empty((M, k), **i32), topk_w=torch.empty((M, k), dtype=torch.float32, device=dev),
+             counts=torch.empty(E, **i32), offsets=torch.empty(E + 1, **i32),
+             row_pair=torch.empty(M * k, **i32), pair_row=torch.empty(M * k, **i32))
+    if X is not None:
+        o["Xperm"] = torch.empty((M * k, H), dtype=torch.bfloat16, device=dev)
+    return o
+
+
+def moe_route(logits, k, X=None, ws=None, out=None):
     """logits f32 [M,E] -> dict(topk_idx, topk_w, counts, offsets, row_pair, pair_row[, Xperm])."""
     M, E = logits.shape
-    dev = logits.device
-    i32 = dict(dtype=torch.int32, device=dev)
-    out = dict(topk_idx=torch.empty((M, k), **i32), topk_w=torch.empty((M, k), dtype=torch.float32, device=dev),
-               counts=torch.empty(E, **i32), offsets=torch.empty(E + 1, **i32),
-               row_pair=torch.empty(M * k, **i32), pair_row=torch.empty(M * k, **i32))
-    H = 0
-    Xp = None
-    if X is not None:
-        H = X.shape[1]
-        Xp = torch.empty((M * k, H), dtype=torch.bfloat16, device=dev)
-        out["Xperm"] = Xp
+    H = X.shape[1] if X is not None else 0
+    out = _route_outputs(M, E, k, H, logits.device, X, out)
     need = route_workspace_bytes(M, E, k)
     if ws is None:
-        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=logits.device)
     _check(load().moe_route(context(), M, E, k, _ptr(logits), _ptr(out["topk_idx"]), _ptr(out["topk_w"]),
                             _ptr(out["counts"]), _ptr(out["offsets"]), _ptr(out["row_pair"]), _ptr(out["pair_row"]),
-                            _ptr(X), _ptr(Xp), H, _ptr(ws), ws.numel(), _stream()), "moe_route")
+                            _ptr(X), _ptr(out.get("Xperm")), H, _ptr(ws), ws.numel(), _stream()), "moe_route")
     return out
 
 
-def moe_route_static(logits, k, X=None):
+def moe_route_static(logits, k, X=None, out=None):
     """moe_route for callers that cannot supply scratch memory: the block histograms live in a fixed array inside
-    the library (limit ceil(M/32)*E <= 65536, else QGemmError -8).  The output tensors are still the caller's; this
-    wrapper allocates them only for convenience.  Calls that overlap on the GPU share the array and would race."""
+    the library (limit ceil(M/32)*E <= 65536, else QGemmError -8).  The output tensors are still the caller's: pass
+    them as `out` (a dict with the keys moe_route returns) and this wrapper allocates nothing either; without `out`
+    it allocates them for convenience.  Calls that overlap on the GPU share the array and would race."""
     M, E = logits.shape
-    dev = logits.device
-    i32 = dict(dtype=torch.int32, device=dev)
-    out = dict(topk_idx=torch.empty((M, k), **i32), topk_w=torch.empty((M, k), dtype=torch.float32, device=dev),
-               counts=torch.empty(E, **i32), offsets=torch.empty(E + 1, **i32),
-               row_pair=torch.empty(M * k, **i32), pair_row=torch.empty(M * k, **i32))
-    H = 0
-    Xp = None
-    if X is not None:
-        H = X.shape[1]
-        Xp = torch.empty((M * k, H), dtype=torch.bfloat16, device=dev)
-        out["Xperm"] = Xp
+    H = X.shape[1] if X is not None else 0
+    out = _route_outputs(M, E, k, H, logits.device, X, out)
     _check(load().moe_route_static(context(), M, E, k, _ptr(logits), _ptr(out["topk_idx"]), _ptr(out["topk_w"]),
                                    _ptr(out["counts"]), _ptr(out["offsets"]), _ptr(out["row_pair"]),
-                                   _ptr(out["pair_row"]), _ptr(X), _ptr(Xp), H, _stream()), "moe_route_static")
+                                   _ptr(out["pair_row"]), _ptr(X), _ptr(out.get("Xperm")), H, _stream()),
+           "moe_route_static")
     return out
 
 

@@ -1,5 +1,6 @@
 // Context management, error strings and tensor-map encoding for the quantised GEMM library.
 #include <new>
+#include <stdlib.h>
 
 #include "qg_internal.h"
 
@@ -16,6 +17,7 @@ const char* qg_strerror(int code) {
         case QG_ERR_CUDA: return "CUDA runtime or driver call failed";
         case QG_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case QG_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of moe_route_static (ceil(M/32)*E <= 65536)";
+        case QG_ERR_DEVICE: return "the current CUDA device is not the context's device";
         default: return "unknown error code";
     }
 }
@@ -26,11 +28,23 @@ int qg_create(qg_ctx** out, int device) {
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { cudaGetLastError(); return QG_ERR_CUDA; }
     if (prop.major != 10) return QG_ERR_ARCH;
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) { cudaGetLastError(); return QG_ERR_CUDA; }
     if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return QG_ERR_CUDA; }
+    struct Restore {       // the caller's current device is left as it was
+        int dev;
+        ~Restore() { if (dev >= 0) cudaSetDevice(dev); }
+    } restore{prev};
     qg_ctx* ctx = new (std::nothrow) qg_ctx();
     if (!ctx) return QG_ERR_CUDA;
     ctx->device = device;
     ctx->sm_count = prop.multiProcessorCount;
+    ctx->wait_limit = qg::DEFAULT_WAIT_LIMIT;
+    ctx->skip_kb = -1;
+    if (const char* f = getenv("QG_FORCE_BT")) {   // tile-shape override for sweeps, read once
+        const int v = atoi(f);
+        if (v == 128 || v == 192 || v == 256) ctx->force_bt = v;
+    }
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
@@ -52,6 +66,7 @@ int qg_create(qg_ctx** out, int device) {
 int qg_destroy(qg_ctx* ctx) {
     if (!ctx) return QG_ERR_NULL;
     cudaFree(ctx->d_status);
+    if (ctx->d_ws) cudaFree(ctx->d_ws);
     delete ctx;
     return QG_OK;
 }
@@ -66,18 +81,47 @@ int qg_poll_status(qg_ctx* ctx, void* stream) {
     return host;
 }
 
+int qg_test_inject(qg_ctx* ctx, unsigned wait_limit_polls, int skip_kblock) {
+    if (!ctx) return QG_ERR_NULL;
+    ctx->wait_limit = wait_limit_polls ? wait_limit_polls : qg::DEFAULT_WAIT_LIMIT;
+    ctx->skip_kb = skip_kblock;
+    return QG_OK;
+}
+
 }  // extern "C"
 
 namespace qg {
-int make_tmap_2d(qg_ctx* ctx, CUtensorMap* out, CUtensorMapDataType dt, int elem_bytes, const void* base,
-                 uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz) {
+int check_device(const qg_ctx* ctx) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return QG_ERR_CUDA; }
+    return dev == ctx->device ? QG_OK : QG_ERR_DEVICE;
+}
+
+int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
+                uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz) {
+    for (int i = 0; i < ctx->tmap_count; ++i) {
+        const TmapEntry& e = ctx->tmaps[i];
+        if (e.base == base && e.inner == inner && e.rows == rows && e.box_inner == box_inner && e.box_rows == box_rows &&
+            e.dt == static_cast<int>(dt) && e.elem_bytes == elem_bytes && e.swz == static_cast<int>(swz)) {
+            *out = &e.map;
+            return QG_OK;
+        }
+    }
+    TmapEntry& e = ctx->tmaps[ctx->tmap_next];
     cuuint64_t dims[2] = {inner, rows};
     cuuint64_t strides[1] = {inner * static_cast<uint64_t>(elem_bytes)};
     cuuint32_t box[2] = {box_inner, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = ctx->encode_tiled(out, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
+    e.base = nullptr;      // not a valid entry while it is being rewritten
+    CUresult r = ctx->encode_tiled(&e.map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
                                    CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? QG_OK : QG_ERR_CUDA;
+    if (r != CUDA_SUCCESS) return QG_ERR_CUDA;
+    e.base = base; e.inner = inner; e.rows = rows; e.box_inner = box_inner; e.box_rows = box_rows;
+    e.dt = static_cast<int>(dt); e.elem_bytes = elem_bytes; e.swz = static_cast<int>(swz);
+    *out = &e.map;
+    ctx->tmap_next = (ctx->tmap_next + 1) % TMAP_CACHE;
+    if (ctx->tmap_count < TMAP_CACHE) ++ctx->tmap_count;
+    return QG_OK;
 }
 }  // namespace qg

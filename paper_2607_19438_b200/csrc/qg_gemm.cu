@@ -24,10 +24,10 @@
 // Every mbarrier wait is bounded; when one expires the CTA records QG_ERR_TIMEOUT and leaves.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
-#include <stdlib.h>
 
 #include "qg_internal.h"
 #include "qg_ptx.cuh"
+#include "qg_profile.cuh"
 
 namespace qg {
 
@@ -35,22 +35,6 @@ constexpr int BW = 128;        // weight rows per CTA tile (one UMMA M half)
 constexpr int BK = 64;         // k per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int NTHREADS = 768;
 constexpr int MAX_E = 1024;
-constexpr uint32_t WAIT_LIMIT = 1u << 18;   // polls; an unsatisfied try_wait poll lasts about 4 us, so about a second
-
-// Profiling builds (-DQG_PROFILE) accumulate, per CTA, the cycles each role spends in each wait.
-#if defined(QG_PROFILE) && !defined(QG_NOSTATS)
-#define QG_T0() long long qg_t0_ = clock64()
-#define QG_ACC(slot) do { if (p.stats) { long long now_ = clock64(); qg_stat_[slot] += now_ - qg_t0_; qg_t0_ = now_; } } while (0)
-#define QG_DECL() long long qg_stat_[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
-#define QG_FLUSH() do { if (p.stats) for (int i_ = 0; i_ < 12; ++i_) if (qg_stat_[i_]) atomicAdd(reinterpret_cast<unsigned long long*>(p.stats) + blockIdx.x * 12 + i_, static_cast<unsigned long long>(qg_stat_[i_])); } while (0)
-#define QG_TRACE(ev, i) do { if (p.stats && blockIdx.x == 0 && (i) < 256) p.stats[148 * 12 + (ev) * 256 + (i)] = clock64(); } while (0)
-#else
-#define QG_TRACE(ev, i) do {} while (0)
-#define QG_T0() do {} while (0)
-#define QG_ACC(slot) do {} while (0)
-#define QG_DECL() do {} while (0)
-#define QG_FLUSH() do {} while (0)
-#endif
 
 struct GemmParams {
     int mode, R, N, K, E, k;
@@ -60,8 +44,11 @@ struct GemmParams {
     const float* topk_w;
     const int32_t* row_pair;
     int* status;
-    long long* stats;           // optional per-CTA cycle counters (profiling builds only), else nullptr
-    int dbg;                    // profiling builds only
+    uint32_t wait_limit;        // polls per bounded wait (an unsatisfied poll lasts about 4 us)
+    int skip_kb;                // test hook: k-block of the first tile whose activation load is left out (-1: none)
+#ifdef QG_PROFILE
+    long long* stats;           // per-CTA cycle counters of a profiling build
+#endif
 };
 
 template <int QBITS, int BT>
@@ -92,7 +79,7 @@ struct Cfg {
     static constexpr int TAB_N = 128;                              // decoded tiles of this pair kept in shared memory
     static constexpr int OFF_TAB = OFF_PREFIX + (MAX_E + 4) * 4;
     static constexpr int OFF_BAR = OFF_TAB + TAB_N * 16;
-    static constexpr int NBAR = 2 * SX + 2 * SR + 4;
+    static constexpr int NBAR = 2 * SX + 2 * SR + 5;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;        // + slack for 1024-byte alignment
     static constexpr int TMEM_COLS = 512;                          // accumulator(s) + SX weight stages
@@ -128,22 +115,23 @@ __device__ __forceinline__ Tile decode_tile(int t, const int* prefix, const Gemm
 
 // Bounded wait on an mbarrier phase.  Returns false if the CTA is giving up.
 template <bool CLUSTER>
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, const GemmParams& p) {
+    const uint32_t limit = p.wait_limit;
+    for (uint32_t it = 0; it < limit; ++it) {
         if (CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
     *abort_flag = 1;
-    atomicCAS(status, 0, QG_ERR_TIMEOUT);
+    atomicCAS(p.status, 0, QG_ERR_TIMEOUT);
     return false;
 }
 
 // Same for the MMA warps: a short non-blocking spin first (the barrier is usually complete or about to be), then
 // the bounded blocking wait.
-__device__ __forceinline__ bool spin_wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool spin_wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, const GemmParams& p) {
     for (int it = 0; it < 64; ++it)
         if (mbar_test_wait_cluster(bar, parity)) return true;
-    return wait_bar<true>(bar, parity, abort_flag, status);
+    return wait_bar<true>(bar, parity, abort_flag, p);
 }
 
 __device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
@@ -322,6 +310,10 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     auto r_empty = [&](int s) { return bar0 + 8u * (2 * C::SX + C::SR + s); };
     auto acc_full = [&](int s) { return bar0 + 8u * (2 * C::SX + 2 * C::SR + s); };
     auto acc_empty = [&](int s) { return bar0 + 8u * (2 * C::SX + 2 * C::SR + 2 + s); };
+    // last_full (this CTA, one phase): the epilogue warps, which consume every accumulator phase in order, have seen the
+    // last tile's accumulator complete.  The dequantising warps that help with that last epilogue wait here instead
+    // of on acc_full, whose parity they cannot tell apart from the phase two tiles earlier when K is short.
+    const uint32_t last_full = bar0 + 8u * (2 * C::SX + 2 * C::SR + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();          // 0: issues the MMAs, 1: its peer
@@ -333,7 +325,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         if (lane < C::SR) { mbar_init(r_full(lane), 1); mbar_init(r_empty(lane), 4); }
         // an accumulator is released by the 4 epilogue + 16 dequantising warps of both CTAs
         if (lane >= 16 && lane < 18) { mbar_init(acc_full(lane - 16), 2); mbar_init(acc_empty(lane - 16), C::HELP ? 40 : 8); }
-        if (lane == 31) misc[1] = 0;
+        if (lane == 31) { misc[1] = 0; mbar_init(last_full, 1); }
         fence_mbar_init();
         fence_proxy_async_smem();
         if (lane == 30) prefetch_tmap(&tm_x);
@@ -402,17 +394,13 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 QG_T0();
                 // a stage is free once the MMAs that read it eight k-blocks ago are done (even and odd stages
                 // belong to different MMA warps, so both are checked)
-                if (!wait_bar<false>(done(s), ph ^ 1u, abort_flag, p.status) ||
-                    !wait_bar<false>(done(s + 1), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                if (!wait_bar<false>(done(s), ph ^ 1u, abort_flag, p) ||
+                    !wait_bar<false>(done(s + 1), ph ^ 1u, abort_flag, p)) { ok = false; break; }
                 QG_ACC(0);
-#ifdef QG_PROFILE
-                if (p.dbg & 8) {
-                    if (lane == 0 && rank == 0) { mbar_arrive(full(s)); mbar_arrive(full(s + 1)); }
-                } else
-#endif
                 if (lane == 0) {
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
+                        if (jt == 0 && kb + j == p.skip_kb) continue;      // test hook: this stage never fills
                         if (rank == 0) mbar_arrive_expect_tx(full(s + j), 2 * C::X_BYTES);
                         tma_load_2d_pair(sbase + C::OFF_X + (s + j) * C::X_BYTES, &tm_x, (kb + j) * BK, row0,
                                          full_leader + 8u * (s + j));
@@ -439,14 +427,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 QG_T0();
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    if (ok && !wait_bar<false>(r_empty(s + j), ph ^ 1u, abort_flag, p.status)) ok = false;
+                    if (ok && !wait_bar<false>(r_empty(s + j), ph ^ 1u, abort_flag, p)) ok = false;
                 if (!ok) break;
                 QG_ACC(1);
-#ifdef QG_PROFILE
-                if (p.dbg & 32) {
-                    if (lane == 0) { for (int j = 0; j < 4; ++j) mbar_arrive(r_full(s + j)); }
-                } else
-#endif
                 if (lane == 0) {
                     const uint32_t sd = sbase + C::OFF_SC + sg * C::SC_BYTES;
 #pragma unroll
@@ -492,9 +475,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 const uint32_t i0 = j * static_cast<uint32_t>(nkb);          // first k-block of the tile (ring index)
                 QG_T0();
                 if (w == 0) {
-                    if (!spin_wait_bar(acc_empty(a), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    if (!spin_wait_bar(acc_empty(a), aph ^ 1u, abort_flag, p)) { ok = false; break; }
                 } else {
-                    if (!spin_wait_bar(done(i0 & 7u), (i0 >> 3) & 1u, abort_flag, p.status)) { ok = false; break; }
+                    if (!spin_wait_bar(done(i0 & 7u), (i0 >> 3) & 1u, abort_flag, p)) { ok = false; break; }
                 }
                 QG_ACC(2);
                 const uint32_t d_tmem = tmem_base + a * BT;
@@ -504,23 +487,18 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 for (int kb = static_cast<int>(w); kb < nkb; kb += 2, i += 2) {
                     const uint32_t st = i & 7u;
                     QG_T0();
-                    if (!ready && !spin_wait_bar(full(st), (i >> 3) & 1u, abort_flag, p.status)) { ok = false; break; }
+                    if (!ready && !spin_wait_bar(full(st), (i >> 3) & 1u, abort_flag, p)) { ok = false; break; }
                     QG_ACC(3);
-                    if (lane == 0) { QG_TRACE(2, i); }
                     tc_fence_after_sync();
                     // start the wait for this warp's next k-block before issuing, so its latency is hidden
                     ready = (kb + 2 < nkb) && mbar_test_wait_cluster(full((i + 2) & 7u), ((i + 2) >> 3) & 1u);
                     if (lane == 0) {
-#ifdef QG_PROFILE
-                        if (!(p.dbg & 64))
-#endif
                         umma_kblock_ts_pair(d_tmem, tmem_base + C::A_COL0 + ta * C::A_COLS,
                                             b_lo0 + st * (C::X_BYTES >> 4), b_hi, idesc, kb != 0 ? 1u : 0u);
                         umma_commit_pair(done(st));
                     }
                     __syncwarp();
                     QG_ACC(10);
-                    if (lane == 0) { QG_TRACE(4, i); }
                     ta += 2;
                     if (ta >= C::SA) ta -= C::SA;
                 }
@@ -562,7 +540,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const int wt = 2 * tl.pw + static_cast<int>(rank);
             const uint32_t a = (C::NACC == 2) ? (jt & 1u) : 0u;
             const uint32_t aph = (C::NACC == 2) ? ((jt >> 1) & 1u) : (jt & 1u);
-            if (!wait_bar<false>(acc_full(a), aph, abort_flag, p.status)) return false;
+            // single accumulator: every tile is helped, so the phases of acc_full are consumed in order; two
+            // accumulators: only the last tile is helped, through the one-shot barrier
+            if (!wait_bar<false>(C::HELP ? acc_full(a) : last_full, C::HELP ? aph : 0u, abort_flag, p)) return false;
             tc_fence_after_sync();
             if (plain_ep && wt < p.n_wt) {
                 const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
@@ -588,22 +568,15 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             }
             QG_T0();
             // the scales of this group of four k-blocks arrive with the first of them (stage 0 or 4)
-            if (!wait_bar<false>(r_full((n % NB) << 2), phr, abort_flag, p.status)) break;
-            if (!wait_bar<false>(r_full(sr), phr, abort_flag, p.status)) break;
+            if (!wait_bar<false>(r_full((n % NB) << 2), phr, abort_flag, p)) break;
+            if (!wait_bar<false>(r_full(sr), phr, abort_flag, p)) break;
             QG_ACC(5);
-            if (q == 0 && lane == 0) { QG_TRACE(5, 4 * n + g); }
             const uint32_t raw = sbase + C::OFF_RAW + sr * C::RAW_BYTES + raw_row;
             const uint32_t scw = *reinterpret_cast<const uint32_t*>(
                 sgen + C::OFF_SC + (n % C::NSB) * C::SC_BYTES + row * 16 + g * 4);
             const float s0 = __half2float(__ushort_as_half(static_cast<unsigned short>(scw & 0xFFFFu)));
             const float s1 = __half2float(__ushort_as_half(static_cast<unsigned short>(scw >> 16)));
             uint32_t o[32];
-#ifdef QG_PROFILE
-            if (p.dbg & 16) {
-#pragma unroll
-                for (int z = 0; z < 32; ++z) o[z] = scw + z;
-            } else
-#endif
 #pragma unroll
             for (int h = 0; h < 2; ++h) {            // k = 32 h .. 32 h + 31 share one scale
                 const float sc = h ? s1 : s0;
@@ -634,21 +607,16 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             __syncwarp();
             if (lane == 0) mbar_arrive(r_empty(sr));             // the packed codes are in registers now
             QG_ACC(7);
-            if (q == 0 && lane == 0) { QG_TRACE(9, 4 * n + g); }
             // its TMEM stage (i % SA) is free once the MMAs of k-block i - SA have completed
             {
                 const uint32_t i = 4u * n + g;
-                if (i >= C::SA && !wait_bar<false>(done((i - C::SA) & 7u), ((i - C::SA) >> 3) & 1u, abort_flag, p.status)) break;
+                if (i >= C::SA && !wait_bar<false>(done((i - C::SA) & 7u), ((i - C::SA) >> 3) & 1u, abort_flag, p)) break;
             }
             QG_ACC(6);
-            if (q == 0 && lane == 0) { QG_TRACE(6, 4 * n + g); }
             tc_fence_after_sync();
             {
                 uint32_t (&o0)[16] = *reinterpret_cast<uint32_t (*)[16]>(o);
                 uint32_t (&o1)[16] = *reinterpret_cast<uint32_t (*)[16]>(o + 16);
-#ifdef QG_PROFILE
-                if (!(p.dbg & 1) || n < 2)
-#endif
                 {
                     tmem_st_32x32_x16(a_taddr + ta * C::A_COLS, o0);
                     tmem_st_32x32_x16(a_taddr + ta * C::A_COLS + 16, o1);
@@ -661,7 +629,6 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             ta += 4;
             if (ta >= C::SA) ta -= C::SA;
             QG_ACC(7);
-            if (q == 0 && lane == 0) { QG_TRACE(7, 4 * n + g); }
         }
         while (C::HELP && dq_ok && helped < static_cast<uint32_t>(my_tiles)) dq_ok = help_tile(helped++, true);
         // With two accumulators the epilogues overlap the main loops, except the last one: these warps have nothing
@@ -685,27 +652,23 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const uint32_t aph = (C::NACC == 2) ? ((j >> 1) & 1u) : (j & 1u);
             const uint32_t fl = j & 1u;       // flag slot: alternates so a slow warp never reads a newer flag
             QG_T0();
-            if (et == 0) misc[2 + fl] = wait_bar<false>(acc_full(a), aph, abort_flag, p.status) ? 1 : 0;
+            if (et == 0) misc[2 + fl] = wait_bar<false>(acc_full(a), aph, abort_flag, p) ? 1 : 0;
             tc_fence_before_sync();
             named_bar_sync(1, 128);
             if (!misc[2 + fl]) break;
             tc_fence_after_sync();
+            if (!C::HELP && et == 0 && static_cast<int>(j) == my_tiles - 1) mbar_arrive(last_full);
             QG_ACC(8);
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + a * BT;
             const int n_epi = (wt < p.n_wt) ? n_mma : 0;
-#ifdef QG_PROFILE
-            int n_epi2 = (p.dbg & 2) ? 0 : n_epi;
-#else
-            int n_epi2 = n_epi;
-#endif
             if constexpr (EPI == 0) {
                 // shared with the dequantising warps (participants 1..4 of this lane quarter) when they help
-                drain_plain(p, tl.tok0, tl.tok_end, wt * BW + qd * 32, taddr, n_epi2, 0,
+                drain_plain(p, tl.tok0, tl.tok_end, wt * BW + qd * 32, taddr, n_epi, 0,
                             (C::HELP || static_cast<int>(j) == my_tiles - 1) ? 5 : 1,
                             stg16 + (16 + qd) * 512, lane);
             } else {
-                for (int c = 0; c < n_epi2; c += 32) {
+                for (int c = 0; c < n_epi; c += 32) {
                     uint32_t v[32];
                     tmem_ld_32x32(taddr + c, v);
                     tmem_ld_wait();
@@ -789,39 +752,35 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const vo
                        cudaStream_t st) {
     using C = Cfg<QBITS, BT>;
     static_assert(C::SMEM_BYTES <= 232448, "shared memory budget");
-    CUtensorMap tm_x, tm_w, tm_s;
+    const CUtensorMap *tm_x, *tm_w, *tm_s;       // cached in the context: the same buffers recur every layer and step
     const uint64_t wrows = static_cast<uint64_t>(p.E) * p.N;
-    int rc = make_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, p.R, BK, C::XH_ROWS,
-                          CU_TENSOR_MAP_SWIZZLE_128B);
+    int rc = get_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, p.R, BK, C::XH_ROWS,
+                         CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc == QG_OK)
-        rc = make_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (QBITS == 8) ? p.K : p.K / 2, wrows,
-                          C::RAW_ROW, 64, (QBITS == 8) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+        rc = get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (QBITS == 8) ? p.K : p.K / 2, wrows,
+                         C::RAW_ROW, 64, (QBITS == 8) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
     if (rc == QG_OK)
-        rc = make_tmap_2d(ctx, &tm_s, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, Ws, p.K / 32, wrows, 8, 64,
-                          CU_TENSOR_MAP_SWIZZLE_NONE);
+        rc = get_tmap_2d(ctx, &tm_s, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, Ws, p.K / 32, wrows, 8, 64,
+                         CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc != QG_OK) return rc;
     auto kern = qgemm_kernel<QBITS, BT, EPI>;
-    static bool attr_set[64] = {false};      // per device: the attribute belongs to the function on one device
-    const int dv = ctx->device;
-    if (dv < 0 || dv >= 64 || !attr_set[dv]) {
+    // the shared-memory attribute belongs to the function on one device: set once per context and instantiation
+    constexpr int inst = ((QBITS == 4) ? 9 : 0) + ((BT == 128) ? 0 : (BT == 192) ? 3 : 6) + EPI;
+    if (!ctx->attr_set[inst]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
             cudaGetLastError();
             return QG_ERR_CUDA;
         }
-        if (dv >= 0 && dv < 64) attr_set[dv] = true;
+        ctx->attr_set[inst] = true;
     }
     // Upper bound on the number of pair tiles (the exact count lives on the device for grouped calls).
     const long long max_tiles =
         (static_cast<long long>((p.R + BT - 1) / BT) + (p.offsets ? p.E : 0)) * ((p.n_wt + 1) / 2);
     const long long pairs_hw = ctx->sm_count / 2;
     const int grid = 2 * static_cast<int>(max_tiles < pairs_hw ? max_tiles : pairs_hw);
-    kern<<<grid, NTHREADS, C::SMEM_BYTES, st>>>(tm_x, tm_w, tm_s, p);
+    kern<<<grid, NTHREADS, C::SMEM_BYTES, st>>>(*tm_x, *tm_w, *tm_s, p);
     return cudaGetLastError() == cudaSuccess ? QG_OK : QG_ERR_CUDA;
 }
-
-#ifdef QG_PROFILE
-static long long* g_stats = nullptr;   // device buffer supplied by the profiling harness
-#endif
 
 // Token tile of a dense call: the candidate with the smallest modelled time.  A wave is one pair tile per SM pair;
 // a tile costs nkb k-blocks of about `period` cycles (measured: issue- and latency-bound, nearly independent of
@@ -845,13 +804,13 @@ static int pick_token_tile(const qg_ctx* ctx, int M, int n_wt, int K) {
 static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in, const void* X, const void* Wq,
                          const void* Ws, cudaStream_t st) {
     GemmParams p = p_in;
-    if (const char* f = getenv("QG_FORCE_BT")) {   // tile-shape override for sweeps
-        const int v = atoi(f);
-        if (v == 128 || v == 192 || v == 256) bt = v;
-    }
+    if (ctx->force_bt) bt = ctx->force_bt;       // QG_FORCE_BT, read when the context was created (tile-shape sweeps)
+    p.status = ctx->d_status;
+    p.wait_limit = ctx->wait_limit;
+    p.skip_kb = ctx->skip_kb;
+    ctx->skip_kb = -1;                           // the test hook acts on one launch
 #ifdef QG_PROFILE
-    p.stats = g_stats;
-    if (const char* d = getenv("QG_DBG")) p.dbg = atoi(d);
+    p.stats = ctx->stats;
 #endif
     const int epi = (p.mode == QG_MODE_GATE_UP_SILU) ? 1 : (p.mode == QG_MODE_DOWN_ACCUM_F32) ? 2 : 0;
 #define QG_LAUNCH(Q, B)                                                                 \
@@ -875,10 +834,6 @@ static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in,
 
 extern "C" {
 
-#ifdef QG_PROFILE
-void qg_debug_set_stats(long long* dev_buf) { qg::g_stats = dev_buf; }
-#endif
-
 int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq, const void* Wscale,
                 void* Cout, void* stream) {
     if (!ctx) return QG_ERR_NULL;
@@ -887,10 +842,11 @@ int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, cons
     if (M == 0) return QG_OK;     // nothing to do: empty tensors may carry null pointers
     if (!A || !Wq || !Wscale || !Cout) return QG_ERR_NULL;
     if (!qg::aligned16(A) || !qg::aligned16(Wq) || !qg::aligned16(Wscale) || !qg::aligned16(Cout)) return QG_ERR_ALIGN;
+    if (const int rc = qg::check_device(ctx)) return rc;
     qg::GemmParams p{};
     p.mode = QG_MODE_PLAIN; p.R = M; p.N = N; p.K = K; p.E = 1; p.k = 1;
     p.n_wt = (N + qg::BW - 1) / qg::BW;
-    p.offsets = nullptr; p.out = Cout; p.topk_w = nullptr; p.row_pair = nullptr; p.status = ctx->d_status;
+    p.offsets = nullptr; p.out = Cout; p.topk_w = nullptr; p.row_pair = nullptr;
     const int bt = qg::pick_token_tile(ctx, M, p.n_wt, K);
     return qg::dispatch_gemm(ctx, qbits, bt, p, A, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
@@ -909,10 +865,11 @@ int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int
     if (mode == QG_MODE_DOWN_ACCUM_F32 && k < 1) return QG_ERR_SHAPE;
     if (static_cast<long long>(E) * N > 0x7FFFFFFF) return QG_ERR_SHAPE;
     if (!qg::aligned16(Ain) || !qg::aligned16(Wq) || !qg::aligned16(Wscale) || !qg::aligned16(Out)) return QG_ERR_ALIGN;
+    if (const int rc = qg::check_device(ctx)) return rc;
     qg::GemmParams p{};
     p.mode = mode; p.R = R; p.N = N; p.K = K; p.E = E; p.k = (k < 1) ? 1 : k;
     p.n_wt = (mode == QG_MODE_GATE_UP_SILU) ? (N / 128) : (N + qg::BW - 1) / qg::BW;
-    p.offsets = expert_offsets; p.out = Out; p.topk_w = topk_w; p.row_pair = row_pair; p.status = ctx->d_status;
+    p.offsets = expert_offsets; p.out = Out; p.topk_w = topk_w; p.row_pair = row_pair;
     // expected rows per expert decide the token tile; 192 keeps two accumulators, so the short main loops of
     // expert tiles overlap their epilogues
     const int bt = (R / E > 100) ? 192 : 128;

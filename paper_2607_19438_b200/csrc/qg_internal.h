@@ -6,6 +6,19 @@
 
 #include "../../include/qgemm.h"
 
+namespace qg {
+// One cached tensor map: the key is everything cuTensorMapEncodeTiled was given.
+struct TmapEntry {
+    const void* base;
+    uint64_t inner, rows;
+    uint32_t box_inner, box_rows;
+    int dt, elem_bytes, swz;
+    CUtensorMap map;
+};
+constexpr int TMAP_CACHE = 64;
+constexpr uint32_t DEFAULT_WAIT_LIMIT = 1u << 18;   // polls; an unsatisfied try_wait poll lasts about 4 us: about a second
+}  // namespace qg
+
 struct qg_ctx {
     int device;
     int sm_count;
@@ -13,11 +26,23 @@ struct qg_ctx {
     CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    int force_bt;              // QG_FORCE_BT at creation (0: heuristic)
+    uint32_t wait_limit;       // polls per bounded device wait
+    int skip_kb;               // test hook, consumed by the next GEMM launch (-1: none)
+    bool attr_set[32];         // per kernel instantiation: dynamic shared-memory attribute set on this device
+    qg::TmapEntry tmaps[qg::TMAP_CACHE];   // tensor maps of recent calls (weights and buffers recur every layer)
+    int tmap_count, tmap_next;
+    void* d_ws;                // device workspace owned by the context (split-K partial tiles and their flags)
+    size_t ws_bytes;
+    long long* stats;          // profiling builds only
 };
 
 namespace qg {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
-// Encodes a 2-D row-major tensor map; inner = contiguous extent in elements, box in elements.
-int make_tmap_2d(qg_ctx* ctx, CUtensorMap* out, CUtensorMapDataType dt, int elem_bytes, const void* base,
-                 uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz);
+// QG_OK if the calling thread's current device is the context's, else QG_ERR_DEVICE.
+int check_device(const qg_ctx* ctx);
+// A 2-D row-major tensor map (inner = contiguous extent in elements, box in elements): looked up in the context's
+// cache, encoded on a miss.  The returned pointer stays valid until TMAP_CACHE further misses.
+int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
+                uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz);
 }  // namespace qg

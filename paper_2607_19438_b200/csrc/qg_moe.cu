@@ -281,6 +281,7 @@ int moe_permute(qg_ctx* ctx, int M, int k, int H, const void* X, const int32_t* 
     if (M == 0) return QG_OK;
     if (!X || !row_pair || !Xperm) return QG_ERR_NULL;
     if (!qg::aligned16(X) || !qg::aligned16(Xperm)) return QG_ERR_ALIGN;
+    if (const int rc = qg::check_device(ctx)) return rc;
     const long long R = static_cast<long long>(M) * k;
     if (R == 0) return QG_OK;
     if (R > 0x7FFFFFFF) return QG_ERR_SHAPE;
@@ -290,19 +291,13 @@ int moe_permute(qg_ctx* ctx, int M, int k, int H, const void* X, const int32_t* 
     return qg::launch_ok();
 }
 
-int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
-              int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row, const void* X,
-              void* Xperm, int H, void* ws, size_t ws_bytes, void* stream) {
-    if (!ctx || !expert_counts || !expert_offsets) return QG_ERR_NULL;
-    if (M < 0 || E < 1 || E > 1024 || k < 1 || k > E) return QG_ERR_SHAPE;
-    if (M > 0 && (!logits || !topk_idx || !topk_w || !row_pair || !pair_row)) return QG_ERR_NULL;
-    if (static_cast<long long>(M) * k > 0x7FFFFFFF) return QG_ERR_SHAPE;
-    const bool gather = (X != nullptr) && (Xperm != nullptr);
-    if (gather && (H < 8 || H % 8)) return QG_ERR_SHAPE;
-    if (gather && (!qg::aligned16(X) || !qg::aligned16(Xperm))) return QG_ERR_ALIGN;
-    if (M > 0 && (!ws || ws_bytes < qg_route_workspace_bytes(M, E, k))) return QG_ERR_WORKSPACE;
+// Shared body of moe_route and moe_route_static: validation, then the three routing launches and the optional row
+// gather.  `hist` is the scratch for the per-block expert histograms (the caller's workspace or the built-in array).
+static int route_impl(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
+                      int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row,
+                      const void* X, void* Xperm, int H, int32_t* hist, void* stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int32_t* hist = static_cast<int32_t*>(ws);
+    const bool gather = (X != nullptr) && (Xperm != nullptr);
     const int nb = (M + qg::ROUTE_TOKENS_PER_BLOCK - 1) / qg::ROUTE_TOKENS_PER_BLOCK;
     if (M == 0) {  // no pairs: counts and offsets are all zero
         if (cudaMemsetAsync(expert_counts, 0, sizeof(int32_t) * E, st) != cudaSuccess ||
@@ -322,21 +317,21 @@ int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* to
             return QG_ERR_CUDA;
         }
     }
+    // every entry hist[b, e] that the scan and the scatter read is written by the first kernel, so whatever an
+    // earlier call left in the scratch does not matter
     qg::route_topk_kernel<<<nb, topk_warps * 32, sm_topk, st>>>(M, E, k, logits, topk_idx, topk_w, hist);
     qg::route_scan_kernel<<<1, 1024, 0, st>>>(nb, E, hist, expert_counts, expert_offsets);
     qg::route_scatter_kernel<<<nb, qg::ROUTE_WARPS * 32, E * sizeof(int), st>>>(M, E, k, topk_idx, expert_offsets, hist,
                                                                                row_pair, pair_row);
-    int rc = qg::launch_ok();
+    const int rc = qg::launch_ok();
     if (rc != QG_OK) return rc;
     if (gather) return moe_permute(ctx, M, k, H, X, row_pair, Xperm, stream);
     return QG_OK;
 }
 
-// moe_route with the block histograms in the library's own fixed device array instead of a caller workspace, for
-// callers that cannot allocate.  Same kernels, same results; no allocation of any kind happens here.
-int moe_route_static(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
-                     int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row,
-                     const void* X, void* Xperm, int H, void* stream) {
+static int route_check(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
+                       int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row,
+                       const void* X, void* Xperm, int H) {
     if (!ctx || !expert_counts || !expert_offsets) return QG_ERR_NULL;
     if (M < 0 || E < 1 || E > 1024 || k < 1 || k > E) return QG_ERR_SHAPE;
     if (M > 0 && (!logits || !topk_idx || !topk_w || !row_pair || !pair_row)) return QG_ERR_NULL;
@@ -344,15 +339,34 @@ int moe_route_static(qg_ctx* ctx, int M, int E, int k, const float* logits, int3
     const bool gather = (X != nullptr) && (Xperm != nullptr);
     if (gather && (H < 8 || H % 8)) return QG_ERR_SHAPE;
     if (gather && (!qg::aligned16(X) || !qg::aligned16(Xperm))) return QG_ERR_ALIGN;
+    return qg::check_device(ctx);
+}
+
+int moe_route(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
+              int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row, const void* X,
+              void* Xperm, int H, void* ws, size_t ws_bytes, void* stream) {
+    const int rc = route_check(ctx, M, E, k, logits, topk_idx, topk_w, expert_counts, expert_offsets, row_pair, pair_row,
+                               X, Xperm, H);
+    if (rc != QG_OK) return rc;
+    if (M > 0 && (!ws || ws_bytes < qg_route_workspace_bytes(M, E, k))) return QG_ERR_WORKSPACE;
+    return route_impl(ctx, M, E, k, logits, topk_idx, topk_w, expert_counts, expert_offsets, row_pair, pair_row, X, Xperm,
+                      H, static_cast<int32_t*>(ws), stream);
+}
+
+// moe_route with the block histograms in the library's own fixed device array instead of a caller workspace, for
+// callers that cannot allocate.  Same kernels, same results; no allocation of any kind happens here.
+int moe_route_static(qg_ctx* ctx, int M, int E, int k, const float* logits, int32_t* topk_idx, float* topk_w,
+                     int32_t* expert_counts, int32_t* expert_offsets, int32_t* row_pair, int32_t* pair_row,
+                     const void* X, void* Xperm, int H, void* stream) {
+    const int rc = route_check(ctx, M, E, k, logits, topk_idx, topk_w, expert_counts, expert_offsets, row_pair, pair_row,
+                               X, Xperm, H);
+    if (rc != QG_OK) return rc;
     const long long nb = (static_cast<long long>(M) + qg::ROUTE_TOKENS_PER_BLOCK - 1) / qg::ROUTE_TOKENS_PER_BLOCK;
     if (nb * E > qg::ROUTE_STATIC_MAX_INTS) return QG_ERR_TOO_LARGE;
-    // Set-up, once per device, with that device current: the array's name is a host-side stand-in, the kernels need
-    // its device address.
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev != ctx->device || dev < 0 || dev >= qg::ROUTE_STATIC_MAX_DEVICES) {
-        cudaGetLastError();
-        return QG_ERR_CUDA;
-    }
+    // Set-up, once per device, with that device current (route_check made sure it is the context's): the array's
+    // name is a host-side stand-in, the kernels need its device address.
+    const int dev = ctx->device;
+    if (dev < 0 || dev >= qg::ROUTE_STATIC_MAX_DEVICES) return QG_ERR_CUDA;
     if (!qg::g_route_static_ptr[dev]) {
         int32_t* ptr = nullptr;
         if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), qg::g_route_static_scratch) != cudaSuccess || !ptr) {
@@ -361,37 +375,8 @@ int moe_route_static(qg_ctx* ctx, int M, int E, int k, const float* logits, int3
         }
         qg::g_route_static_ptr[dev] = ptr;
     }
-    int32_t* hist = qg::g_route_static_ptr[dev];
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (M == 0) {
-        if (cudaMemsetAsync(expert_counts, 0, sizeof(int32_t) * E, st) != cudaSuccess ||
-            cudaMemsetAsync(expert_offsets, 0, sizeof(int32_t) * (E + 1), st) != cudaSuccess) {
-            cudaGetLastError();
-            return QG_ERR_CUDA;
-        }
-        return QG_OK;
-    }
-    // one token per warp when 32 warps' rows fit in 64 KB of shared memory, else 8 warps take 4 tokens each
-    const int topk_warps = (32 * static_cast<size_t>(E + k) * sizeof(float) <= 64 * 1024) ? 32 : qg::ROUTE_WARPS;
-    const size_t sm_topk = (static_cast<size_t>(topk_warps) * (E + k) + E) * sizeof(float);
-    if (sm_topk > 48 * 1024) {
-        if (cudaFuncSetAttribute(qg::route_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(sm_topk)) != cudaSuccess) {
-            cudaGetLastError();
-            return QG_ERR_CUDA;
-        }
-    }
-    // every entry hist[b, e] that the scan and the scatter read is written by the first kernel of this call, so
-    // whatever an earlier call left in the shared array does not matter
-    const int nbi = static_cast<int>(nb);
-    qg::route_topk_kernel<<<nbi, topk_warps * 32, sm_topk, st>>>(M, E, k, logits, topk_idx, topk_w, hist);
-    qg::route_scan_kernel<<<1, 1024, 0, st>>>(nbi, E, hist, expert_counts, expert_offsets);
-    qg::route_scatter_kernel<<<nbi, qg::ROUTE_WARPS * 32, E * sizeof(int), st>>>(M, E, k, topk_idx, expert_offsets, hist,
-                                                                                row_pair, pair_row);
-    const int rc = qg::launch_ok();
-    if (rc != QG_OK) return rc;
-    if (gather) return moe_permute(ctx, M, k, H, X, row_pair, Xperm, stream);
-    return QG_OK;
+    return route_impl(ctx, M, E, k, logits, topk_idx, topk_w, expert_counts, expert_offsets, row_pair, pair_row, X, Xperm,
+                      H, qg::g_route_static_ptr[dev], stream);
 }
 
 int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
@@ -402,6 +387,7 @@ int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, con
     if (M == 0) return QG_OK;
     if (!D || !Y) return QG_ERR_NULL;
     if (!qg::aligned16(D) || !qg::aligned16(Y)) return QG_ERR_ALIGN;
+    if (const int rc = qg::check_device(ctx)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (d_kind == QG_D_F32_ACC) {
         const size_t n8 = static_cast<size_t>(M) * H / 8;

@@ -96,3 +96,36 @@ def test_dense_full_size_sampled_config1_gate_up():
     ref = orc.qgemm_dense_sample(qbits, A, Wq, Ws, rows, cols)
     util.assert_close(out[rows, cols], ref, "config 1 gate/up sampled")
     assert np.all(np.isfinite(out))
+
+
+def _sampled_on_device(qbits, A, Wq, Ws, out, per_tile, seed, tile=128):
+    """Compares `out` (device bf16 [M, N]) with the oracle on per_tile random elements of every 128 x 128 tile and on
+    the four corners; only the sampled elements leave the device."""
+    M, N = out.shape
+    rng = np.random.default_rng(seed)
+    rt, ct = np.meshgrid(np.arange((M + tile - 1) // tile), np.arange((N + tile - 1) // tile), indexing="ij")
+    rows = np.minimum(rt.reshape(-1, 1) * tile + rng.integers(0, tile, (rt.size, per_tile)), M - 1).reshape(-1)
+    cols = np.minimum(ct.reshape(-1, 1) * tile + rng.integers(0, tile, (ct.size, per_tile)), N - 1).reshape(-1)
+    rows = np.concatenate([rows, [0, M - 1, M - 1, 0]]); cols = np.concatenate([cols, [0, N - 1, 0, N - 1]])
+    got = out[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()].to(torch.float64).cpu().numpy()
+    assert bool(torch.isfinite(out.float()).all().item())
+    ref = orc.qgemm_dense_sample(qbits, A, Wq, Ws, rows, cols)
+    return util.assert_close(got, ref, f"sampled q{qbits} {M}x{N}x{A.shape[1]}")
+
+
+# Short K with several full token tiles per SM pair: the tile boundary logic (accumulator hand-over, the helpers
+# of the last epilogue) runs with fewer k-blocks per tile than the rings are deep.  2048 x 8192 runs as 192-token
+# tiles (about five per pair), 128 x 57344 as 128-token tiles (three per pair).
+SHORT_K = [(8, 2048, 8192, 256), (4, 2048, 8192, 256), (8, 2048, 8192, 512), (4, 2048, 8192, 512),
+           (8, 128, 57344, 256), (4, 128, 57344, 512), (8, 1536, 8192, 256)]
+
+
+@pytest.mark.parametrize("qbits,M,N,K", SHORT_K, ids=[f"q{c[0]}-{c[1]}x{c[2]}x{c[3]}" for c in SHORT_K])
+def test_dense_short_k_many_tiles_per_pair(qbits, M, N, K):
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=4)
+    out = run_dense(qbits, A, Wq, Ws)
+    _sampled_on_device(qbits, A, Wq, Ws, out, per_tile=8, seed=K + M)
+    # and every element of the last token tile and of a middle one, where a stale accumulator would show
+    for r0 in (M - 128, (M // 2) & ~127):
+        ref = orc.qgemm_dense(qbits, A[r0:r0 + 128], Wq[:2048], Ws[:2048])
+        util.assert_close(util.host_bf16_f64(out[r0:r0 + 128, :2048]), ref, f"rows {r0}..")

@@ -43,7 +43,8 @@ def test_dense_full_size_sampled(qbits, M, N, K):
     _sampled_dense(qbits, M, N, K, seed=0, per_tile=1 if M * N > 2 ** 24 else 2)
 
 
-@pytest.mark.parametrize("M,skewed", [(2048, False), (2048, True), (1024, False)], ids=["uniform-2048", "skewed-2048", "uniform-1024"])
+@pytest.mark.parametrize("M,skewed", [(2048, False), (2048, True), (1024, False), (4096, False), (8192, False), (8192, True)],
+                         ids=["uniform-2048", "skewed-2048", "uniform-1024", "uniform-4096", "uniform-8192", "skewed-8192"])
 def test_moe_config3_full_size_selected_experts(M, skewed):
     """Config 3 (H=2048, E=128, top-8, F=768, Q4) at the bench's token counts.  Routing and permutation are compared in
     full (bit exact); the two GEMM stages are compared on every row of a few experts (the busiest, the least busy and
@@ -68,7 +69,6 @@ def test_moe_config3_full_size_selected_experts(M, skewed):
     assert np.array_equal(r["pair_row"].cpu().numpy(), pair_row)
     Xp = orc.permute(X, row_pair, k)
     assert np.array_equal(util.host_bf16_bits(r["Xperm"]), Xp)
-    Hh_g = util.host_bf16_f64(Hh); Dw_g = util.host_bf16_f64(Dw)
     w_gpu = r["topk_w"].cpu().numpy().astype(np.float64).reshape(-1)
     experts = sorted({int(np.argmax(counts)), int(np.argmin(counts)), 5, 64})
     for e in experts:
@@ -76,9 +76,28 @@ def test_moe_config3_full_size_selected_experts(M, skewed):
         if seg.stop == seg.start:
             continue
         off1 = np.array([0, seg.stop - seg.start], np.int32)
+        Hh_e = util.host_bf16_f64(Hh[seg])
         GU = orc.grouped_gemm(qbits, orc.bf16_to_f64(Xp[seg]), off1, W1q[e:e + 1], W1s[e:e + 1])
-        util.assert_close(Hh_g[seg], orc.silu_mul(GU), f"gate/up expert {e}")
-        Dn = orc.grouped_gemm(qbits, Hh_g[seg], off1, W2q[e:e + 1], W2s[e:e + 1])
-        util.assert_close(Dw_g[seg], Dn * w_gpu[row_pair[seg]][:, None], f"down expert {e}")
-    util.assert_close(util.host_bf16_f64(y), orc.combine(Dw_g, pair_row, k), "combine")
-    assert np.all(np.isfinite(util.host_bf16_f64(y)))
+        util.assert_close(Hh_e, orc.silu_mul(GU), f"gate/up expert {e}")
+        Dn = orc.grouped_gemm(qbits, Hh_e, off1, W2q[e:e + 1], W2s[e:e + 1])
+        util.assert_close(util.host_bf16_f64(Dw[seg]), Dn * w_gpu[row_pair[seg]][:, None], f"down expert {e}")
+    assert bool(torch.isfinite(Hh.float()).all().item()) and bool(torch.isfinite(Dw.float()).all().item())
+    # combine on the GPU's own weighted rows: all tokens up to M = 2048, else the first and the last 512 tokens
+    yh = util.host_bf16_f64(y)
+    assert np.all(np.isfinite(yh))
+    toks = np.arange(M) if M <= 2048 else np.concatenate([np.arange(512), np.arange(M - 512, M)])
+    rows_needed = pair_row.reshape(M, k)[toks].reshape(-1)
+    D_sub = util.host_bf16_f64(Dw[torch.from_numpy(rows_needed.astype(np.int64)).cuda()])
+    sub_pair_row = np.arange(rows_needed.size, dtype=np.int32)            # token i of the subset owns rows i k .. i k + k - 1
+    util.assert_close(yh[toks], orc.combine(D_sub, sub_pair_row, k), "combine")
+
+
+def test_config4_gate_up_projection_sampled():
+    """Config 4's largest dense launch: M = 8192 tokens, N = 2 x 14336, K = 4096 (224 weight tiles, 32 token tiles), one
+    sampled element in every 128 x 128 output tile plus the corners."""
+    from tests.test_gpu_dense import _sampled_on_device
+    qbits, M, N, K = 8, 8192, 28672, 4096
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=0)
+    out = qg.qgemm_dense(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws))
+    qg.poll_status()
+    _sampled_on_device(qbits, A, Wq, Ws, out, per_tile=1, seed=4)

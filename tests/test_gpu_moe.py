@@ -68,8 +68,8 @@ def test_moe_stages_and_layer(name, qbits, M, H, E, F, k, skewed):
 
 
 def test_moe_config3_shape_reduced_tokens():
-    """Config 3 geometry (H=2048, E=128, k=8, F=768, Q4) at M=128: 8 rows per expert on average, some experts empty
-    in the skewed case; checked end to end on a subset of experts' rows to bound oracle time."""
+    """Config 3 geometry (H=2048, E=128, k=8, F=768, Q4) at M=128 with skewed routing: 8 rows per expert on average,
+    segments from at most 2 rows to at least 20 in one launch; every stage output against the oracle."""
     qbits, M, H, E, F, k = 4, 128, 2048, 128, 768, 8
     logits, X, W1q, W1s, W2q, W2s = synth.moe_problem(qbits, M, H, E, F, seed=0, skewed=True)
     r, Hh, Dw, y, d = gpu_layer(qbits, logits, X, W1q, W1s, W2q, W2s, k)
@@ -100,3 +100,34 @@ def test_grouped_more_tiles_per_pair_than_the_tile_table():
     qg.poll_status()
     ref = orc.grouped_gemm(qbits, orc.bf16_to_f64(A), offsets, Wq, Ws)
     util.assert_close(util.host_bf16_f64(out), ref, "grouped plain, tiles beyond the table")
+
+
+@pytest.mark.parametrize("qbits,E,rows,K,N,mode", [
+    (4, 2, 600, 256, 8192, qg.MODE_PLAIN), (8, 2, 600, 512, 8192, qg.MODE_DOWN_WEIGHTED),
+    (4, 16, 96, 256, 8192, qg.MODE_PLAIN), (8, 16, 96, 512, 8192, qg.MODE_DOWN_WEIGHTED),
+    (4, 3, 500, 256, 4096, qg.MODE_GATE_UP_SILU)],
+    ids=["q4-192tile-k256", "q8-192tile-k512-weighted", "q4-128tile-k256", "q8-128tile-k512-weighted", "q4-gateup-k256"])
+def test_grouped_short_k_many_tiles_per_pair(qbits, E, rows, K, N, mode):
+    """Grouped calls with K = 256 / 512 and several token tiles of real length per SM pair (long segments -> 192-token
+    tiles, 96-row segments -> 128-token tiles): every output row against the oracle."""
+    counts = np.full(E, rows, np.int32)
+    counts[-1] = rows - 37                                      # one ragged segment
+    offsets = np.zeros(E + 1, np.int32)
+    offsets[1:] = np.cumsum(counts)
+    R = int(offsets[-1])
+    A = synth.activations(R, K, 8, 51)
+    gen = synth.weights_q8 if qbits == 8 else synth.weights_q4
+    Wq = gen(E * N, K, 8, 52).reshape(E, N, -1)
+    Ws = synth.scales(E * N, K // 32, 127 if qbits == 8 else 7, 8, 53).reshape(E, N, K // 32)
+    rng = np.random.default_rng(3)
+    row_pair = rng.permutation(R).astype(np.int32)
+    w = rng.uniform(0.1, 1.0, R).astype(np.float32)
+    out = qg.moe_grouped_qgemm(mode, qbits, util.dev_bf16(A), util.dev(offsets), util.dev(Wq), util.dev_f16(Ws),
+                               topk_w=util.dev(w), row_pair=util.dev(row_pair), k=1)
+    qg.poll_status()
+    ref = orc.grouped_gemm(qbits, orc.bf16_to_f64(A), offsets, Wq, Ws)
+    if mode == qg.MODE_GATE_UP_SILU:
+        ref = orc.silu_mul(ref)
+    elif mode == qg.MODE_DOWN_WEIGHTED:
+        ref = ref * w[row_pair].astype(np.float64)[:, None]
+    util.assert_close(util.host_bf16_f64(out), ref, "grouped short K")

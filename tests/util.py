@@ -41,3 +41,32 @@ def assert_close(out, ref, what=""):
     assert mx <= MAX_ERR_FACTOR * rmax, f"{what}: max err {mx:.3e} > 2e-2 * {rmax:.3e}"
     assert fro <= REL_FRO, f"{what}: rel Frobenius {fro:.3e} > 5e-3"
     return mx, rmax, fro
+
+
+SENTINEL16 = 0x7B5A     # a finite bf16 pattern (about 1.1e36) no kernel output takes
+
+
+class Guarded:
+    """A tensor placed inside a larger buffer filled with a sentinel, at a 16-byte-aligned offset with a head and a
+    tail of `pad` elements.  `intact()` tells whether a kernel wrote outside the tensor."""
+
+    def __init__(self, shape, dtype, pad=4096, fill_inside=True):
+        n = int(np.prod(shape))
+        esz = torch.empty((), dtype=dtype).element_size()
+        assert (pad * esz) % 16 == 0
+        self.pad, self.n = pad, n
+        self.bits = {2: torch.int16, 4: torch.int32}[esz]
+        self.sent = SENTINEL16 if esz == 2 else 0x7B5A7B5A
+        self.buf = torch.full((n + 2 * pad,), self.sent, dtype=self.bits, device="cuda")
+        self.t = self.buf[pad:pad + n].view(dtype).view(*shape)
+        if not fill_inside:
+            self.t.zero_()
+
+    def intact(self):
+        head = self.buf[:self.pad]
+        tail = self.buf[self.pad + self.n:]
+        return bool((head == self.sent).all().item()) and bool((tail == self.sent).all().item())
+
+    def untouched_inside(self):
+        """Mask of elements of the tensor itself that still hold the sentinel."""
+        return self.buf[self.pad:self.pad + self.n].view(self.t.shape) == self.sent
