@@ -137,9 +137,18 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------ clocks
+def clocks_in_window(samples, t0, t1):
+    """Median SM clock and the throttle reasons seen between two host times (None if no sample fell inside)."""
+    inside = [(mhz, act) for ts, mhz, act in samples if t0 <= ts <= t1]
+    if not inside:
+        return None
+    return {"sm_mhz": float(np.median([m for m, _ in inside])), "samples": len(inside),
+            "reasons": sorted({r for _, act in inside for r in act})}
+
+
 class ClockSampler:
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,timestamp")
 
     def __init__(self, index):
         self.proc = None
@@ -158,7 +167,9 @@ class ClockSampler:
             out, _ = self.proc.communicate(timeout=5)
         except Exception:
             self.proc.kill(); out = ""
+        import datetime
         sm, mx, pw, reasons = [], [], [], set()
+        self.samples = []          # (epoch seconds, SM MHz, reasons active) for per-window summaries
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in out.strip().splitlines():
             f = [x.strip() for x in ln.split(",")]
@@ -168,9 +179,14 @@ class ClockSampler:
                 sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
             except ValueError:
                 continue
-            for nm, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(nm)
+            act = [nm for nm, v in zip(names, f[3:7]) if v.lower().startswith("active")]
+            reasons.update(act)
+            if len(f) >= 8:
+                try:
+                    ts = datetime.datetime.strptime(f[7], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    self.samples.append((ts, float(f[0]), act))
+                except ValueError:
+                    pass
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
         return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "power_w_max": float(max(pw)),
@@ -214,10 +230,16 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
 
     def timed_calls(calls, n_iter):
         """calls: list of (label, flops, bytes, fn(it)).  Returns {label: [total_ms, flops, bytes]} over n_iter passes."""
-        for it in range(3):
+        t_w = time.perf_counter()          # warm up for at least 60 ms: a short burst after a host-side pause would
+        it = 0                             # otherwise be timed while the SM clock is still ramping up
+        while it < 3 or time.perf_counter() - t_w < 0.06:
             for _, _, _, fn in calls:
                 fn(it)
+            it += 1
+            if it % 8 == 0:
+                torch.cuda.synchronize()
         torch.cuda.synchronize()
+        windows.append([time.time(), None])
         evs = []
         for it in range(n_iter):
             for lab, fl, nb, fn in calls:
@@ -225,13 +247,15 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
                 e0.record(stream); fn(it); e1.record(stream)
                 evs.append((lab, fl, nb, e0, e1))
         torch.cuda.synchronize()
+        windows[-1][1] = time.time()
         agg = {}
         for lab, fl, nb, e0, e1 in evs:
             d = agg.setdefault(lab, [0.0, fl, nb])
             d[0] += e0.elapsed_time(e1)
         return agg
 
-    out = {"method": "one CUDA-event pair per call on the launching stream, 3 warm-up + %d timed passes per configuration, "
+    windows = []
+    out = {"method": "one CUDA-event pair per call on the launching stream, at least 60 ms of warm-up passes then %d timed passes per configuration, "
                      "dense weights rotated through copies exceeding 2x L2, inputs drawn on the device (seed 0)" % iters,
            "peak_tflops": peak_tf, "dense": [], "moe": []}
     for name, M in SWEEP_DENSE:
@@ -306,6 +330,7 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
         row["frac_of_measured_peak"] = row["gemms_tflops"] / peak_tf
         row["frac_of_composite_bound"] = max(t_tensor, t_hbm) / (gemm_ms / n_it * 1e-3)
         out["moe"].append(row)
+    out["_windows"] = windows
     return out
 
 # ------------------------------------------------------------------------------------------ GPU arm
@@ -549,8 +574,13 @@ def run_ours(args):
     if world == 1 and not args.no_sweep:
         del inA, inL, inX, outC2, outY2
         torch.cuda.empty_cache()
+        sampler3 = ClockSampler(local)
         sweep = run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm)
         qg.poll_status()
+        sweep["clocks"] = sampler3.stop()
+        wins = sweep.pop("_windows")
+        for row, (t0, t1) in zip(sweep["dense"] + sweep["moe"], wins):
+            row["clocks"] = clocks_in_window(getattr(sampler3, "samples", []), t0 - 0.02, t1 + 0.02)
     if rank == 0:
         dense_h0, moe_h0 = dense_h, moe_h
         cpu = cpu_baseline(dense_h0, moe_h0) if world == 1 else None

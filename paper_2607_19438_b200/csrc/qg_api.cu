@@ -41,6 +41,8 @@ int qg_create(qg_ctx** out, int device) {
     ctx->sm_count = prop.multiProcessorCount;
     ctx->wait_limit = qg::DEFAULT_WAIT_LIMIT;
     ctx->skip_kb = -1;
+    const char* no_pdl = getenv("QG_NO_PDL");
+    ctx->pdl = !(no_pdl && no_pdl[0] == '1');
     if (const char* f = getenv("QG_FORCE_BT")) {   // tile-shape override for sweeps, read once
         const int v = atoi(f);
         if (v == 128 || v == 192 || v == 256) ctx->force_bt = v;

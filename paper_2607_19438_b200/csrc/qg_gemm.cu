@@ -317,6 +317,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();          // 0: issues the MMAs, 1: its peer
+    // The next kernel in the stream may be scheduled as this grid's CTAs leave their SMs.  This kernel in turn may
+    // have started before the previous one finished: whatever that kernel may have written (activations, expert
+    // offsets, routing tables) or may still read (the output buffer) is touched only after pdl_wait().  The weights
+    // are constants of the model, so in the dense case their producer and the dequantising warps start at once.
+    pdl_launch_dependents();
+    const bool grouped = (p.offsets != nullptr);
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     volatile int* abort_flag = misc + 1;
 
@@ -338,6 +344,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     }
     const int n_pw = (p.n_wt + 1) >> 1;
     if (warp == 2) {  // prefix[e] = pair tiles before expert e; prefix[E] = total
+        if (grouped) pdl_wait();
         int carry = 0;
         for (int e0 = 0; e0 < p.E; e0 += 32) {
             const int e = e0 + lane;
@@ -361,6 +368,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     __syncthreads();
     cluster_sync_all();          // both CTAs' barriers are initialised and both halves of TMEM are allocated
     tc_fence_after_sync();
+    if (grouped || warp == 0 || (warp >= 4 && warp < 8)) pdl_wait();   // dense: the other roles wait when they must
     const uint32_t tmem_base = static_cast<uint32_t>(misc[0]);
     const int total_tiles = prefix[p.E];
     const int nkb = p.K / BK;     // a multiple of 4
@@ -536,6 +544,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         uint32_t ta = static_cast<uint32_t>(g) % C::SA;                 // TMEM weight stage of own k-block i = i % SA
         bool dq_ok = true;
         auto help_tile = [&](uint32_t jt, bool release) -> bool {
+            pdl_wait();          // these warps store to the output from here on (returns at once after the first time)
             const Tile tl = tile_at(static_cast<int>(jt));
             const int wt = 2 * tl.pw + static_cast<int>(rank);
             const uint32_t a = (C::NACC == 2) ? (jt & 1u) : 0u;
@@ -778,8 +787,11 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const vo
         (static_cast<long long>((p.R + BT - 1) / BT) + (p.offsets ? p.E : 0)) * ((p.n_wt + 1) / 2);
     const long long pairs_hw = ctx->sm_count / 2;
     const int grid = 2 * static_cast<int>(max_tiles < pairs_hw ? max_tiles : pairs_hw);
-    kern<<<grid, NTHREADS, C::SMEM_BYTES, st>>>(*tm_x, *tm_w, *tm_s, p);
-    return cudaGetLastError() == cudaSuccess ? QG_OK : QG_ERR_CUDA;
+    if (launch_kernel(ctx, kern, dim3(grid), dim3(NTHREADS), C::SMEM_BYTES, st, *tm_x, *tm_w, *tm_s, p) != cudaSuccess) {
+        cudaGetLastError();
+        return QG_ERR_CUDA;
+    }
+    return QG_OK;
 }
 
 // Token tile of a dense call: the candidate with the smallest modelled time.  A wave is one pair tile per SM pair;

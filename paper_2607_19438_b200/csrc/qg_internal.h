@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "../../include/qgemm.h"
 
 namespace qg {
@@ -32,12 +34,28 @@ struct qg_ctx {
     bool attr_set[32];         // per kernel instantiation: dynamic shared-memory attribute set on this device
     qg::TmapEntry tmaps[qg::TMAP_CACHE];   // tensor maps of recent calls (weights and buffers recur every layer)
     int tmap_count, tmap_next;
+    bool pdl;                  // launch kernels with programmatic stream serialization (QG_NO_PDL=1 turns it off)
     void* d_ws;                // device workspace owned by the context (split-K partial tiles and their flags)
     size_t ws_bytes;
     long long* stats;          // profiling builds only
 };
 
 namespace qg {
+// Launches `kern`; with ctx->pdl the launch carries the programmatic-serialization attribute, so the kernel's prologue
+// may overlap the tail of the kernel before it in the stream (every kernel of this library calls pdl_wait() before it
+// reads or writes anything an earlier kernel may touch).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(const qg_ctx* ctx, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = ctx->pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 // QG_OK if the calling thread's current device is the context's, else QG_ERR_DEVICE.
 int check_device(const qg_ctx* ctx);

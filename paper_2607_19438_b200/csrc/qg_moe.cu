@@ -8,6 +8,7 @@
 #include <math.h>
 
 #include "qg_internal.h"
+#include "qg_ptx.cuh"
 
 namespace qg {
 
@@ -41,8 +42,10 @@ route_topk_kernel(int M, int E, int k, const float* __restrict__ logits, int32_t
     uint32_t* keys = reinterpret_cast<uint32_t*>(sm) + warp * (E + k);
     float* sel = reinterpret_cast<float*>(keys + E);
     int* hist = reinterpret_cast<int*>(sm + nwarps * (E + k));
+    pdl_launch_dependents();
     for (int e = threadIdx.x; e < E; e += blockDim.x) hist[e] = 0;
     __syncthreads();
+    pdl_wait();
 
     const int t0 = blockIdx.x * ROUTE_TOKENS_PER_BLOCK;
     for (int tt = warp; tt < ROUTE_TOKENS_PER_BLOCK; tt += nwarps) {
@@ -88,6 +91,8 @@ route_scan_kernel(int nb, int E, int32_t* __restrict__ block_hist, int32_t* __re
                   int32_t* __restrict__ offsets) {
     __shared__ int part[1024];
     __shared__ int tot[1024];
+    pdl_launch_dependents();
+    pdl_wait();
     const int G = 1024 / E > 0 ? 1024 / E : 1;
     const int g = threadIdx.x / E, e = threadIdx.x % E;
     const bool active = g < G;
@@ -152,6 +157,8 @@ route_scatter_kernel(int M, int E, int k, const int32_t* __restrict__ topk_idx, 
                      int32_t* __restrict__ pair_row) {
     extern __shared__ int run[];  // E running row cursors
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    pdl_wait();
     for (int e = threadIdx.x; e < E; e += blockDim.x)
         run[e] = offsets[e] + block_base[static_cast<size_t>(blockIdx.x) * E + e];
     __syncthreads();
@@ -186,6 +193,8 @@ permute_rows_kernel(int R, int k, int H8, const int4* __restrict__ X, const int3
                     int4* __restrict__ Xp) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     const int nwarps = (gridDim.x * blockDim.x) >> 5;
+    pdl_launch_dependents();
+    pdl_wait();
     for (int r = warp; r < R; r += nwarps) {
         const int t = row_pair[r] / k;
         const int4* src = X + static_cast<size_t>(t) * H8;
@@ -214,6 +223,8 @@ __global__ void __launch_bounds__(256)
 combine_kernel(int M, int k, int H8, const int4* __restrict__ D, const int32_t* __restrict__ pair_row,
                const float* __restrict__ topk_w, int4* __restrict__ Y) {
     const int t = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     for (int v = threadIdx.x; v < H8; v += blockDim.x) {
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         // Eight slots at a time: all row indices, then all rows, are in flight together; the sum stays in slot order.
@@ -244,6 +255,8 @@ combine_kernel(int M, int k, int H8, const int4* __restrict__ D, const int32_t* 
 // Y = bf16(acc) for the f32 accumulator produced by the atomic-accumulate epilogue.
 __global__ void __launch_bounds__(256)
 round_f32_kernel(size_t n8, const float4* __restrict__ acc, int4* __restrict__ Y) {
+    pdl_launch_dependents();
+    pdl_wait();
     for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n8;
          i += static_cast<size_t>(gridDim.x) * blockDim.x) {
         const float4 a = acc[2 * i], b = acc[2 * i + 1];
@@ -254,7 +267,11 @@ round_f32_kernel(size_t n8, const float4* __restrict__ acc, int4* __restrict__ Y
     }
 }
 
-static int launch_ok() { return cudaGetLastError() == cudaSuccess ? QG_OK : QG_ERR_CUDA; }
+static int launch_rc(cudaError_t e) {
+    if (e == cudaSuccess) return QG_OK;
+    cudaGetLastError();
+    return QG_ERR_CUDA;
+}
 
 // Built-in scratch of moe_route_static: per-block expert histograms for callers that cannot hand over a workspace.
 // In host code this name is only a handle; the device address is looked up once per device (see below).
@@ -286,9 +303,9 @@ int moe_permute(qg_ctx* ctx, int M, int k, int H, const void* X, const int32_t* 
     if (R == 0) return QG_OK;
     if (R > 0x7FFFFFFF) return QG_ERR_SHAPE;
     const int blocks = static_cast<int>(min(static_cast<long long>(ctx->sm_count) * 8, (R + 7) / 8));
-    qg::permute_rows_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<int>(R), k, H / 8, static_cast<const int4*>(X), row_pair, static_cast<int4*>(Xperm));
-    return qg::launch_ok();
+    return qg::launch_rc(qg::launch_kernel(ctx, qg::permute_rows_kernel, dim3(blocks), dim3(256), 0,
+                                           static_cast<cudaStream_t>(stream), static_cast<int>(R), k, H / 8,
+                                           static_cast<const int4*>(X), row_pair, static_cast<int4*>(Xperm)));
 }
 
 // Shared body of moe_route and moe_route_static: validation, then the three routing launches and the optional row
@@ -319,11 +336,16 @@ static int route_impl(qg_ctx* ctx, int M, int E, int k, const float* logits, int
     }
     // every entry hist[b, e] that the scan and the scatter read is written by the first kernel, so whatever an
     // earlier call left in the scratch does not matter
-    qg::route_topk_kernel<<<nb, topk_warps * 32, sm_topk, st>>>(M, E, k, logits, topk_idx, topk_w, hist);
-    qg::route_scan_kernel<<<1, 1024, 0, st>>>(nb, E, hist, expert_counts, expert_offsets);
-    qg::route_scatter_kernel<<<nb, qg::ROUTE_WARPS * 32, E * sizeof(int), st>>>(M, E, k, topk_idx, expert_offsets, hist,
-                                                                               row_pair, pair_row);
-    const int rc = qg::launch_ok();
+    int rc = qg::launch_rc(qg::launch_kernel(ctx, qg::route_topk_kernel, dim3(nb), dim3(topk_warps * 32), sm_topk, st, M, E, k,
+                                             logits, topk_idx, topk_w, hist));
+    if (rc == QG_OK)
+        rc = qg::launch_rc(qg::launch_kernel(ctx, qg::route_scan_kernel, dim3(1), dim3(1024), 0, st, nb, E, hist,
+                                             expert_counts, expert_offsets));
+    if (rc == QG_OK)
+        rc = qg::launch_rc(qg::launch_kernel(ctx, qg::route_scatter_kernel, dim3(nb), dim3(qg::ROUTE_WARPS * 32),
+                                             E * sizeof(int), st, M, E, k, static_cast<const int32_t*>(topk_idx),
+                                             static_cast<const int32_t*>(expert_offsets),
+                                             static_cast<const int32_t*>(hist), row_pair, pair_row));
     if (rc != QG_OK) return rc;
     if (gather) return moe_permute(ctx, M, k, H, X, row_pair, Xperm, stream);
     return QG_OK;
@@ -392,13 +414,12 @@ int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, con
     if (d_kind == QG_D_F32_ACC) {
         const size_t n8 = static_cast<size_t>(M) * H / 8;
         const int blocks = static_cast<int>(min(static_cast<size_t>(ctx->sm_count) * 8, (n8 + 255) / 256));
-        qg::round_f32_kernel<<<blocks, 256, 0, st>>>(n8, static_cast<const float4*>(D), static_cast<int4*>(Y));
-        return qg::launch_ok();
+        return qg::launch_rc(qg::launch_kernel(ctx, qg::round_f32_kernel, dim3(blocks), dim3(256), 0, st, n8,
+                                               static_cast<const float4*>(D), static_cast<int4*>(Y)));
     }
     if (!pair_row) return QG_ERR_NULL;
-    qg::combine_kernel<<<M, 256, 0, st>>>(M, k, H / 8, static_cast<const int4*>(D), pair_row, topk_w,
-                                         static_cast<int4*>(Y));
-    return qg::launch_ok();
+    return qg::launch_rc(qg::launch_kernel(ctx, qg::combine_kernel, dim3(M), dim3(256), 0, st, M, k, H / 8,
+                                           static_cast<const int4*>(D), pair_row, topk_w, static_cast<int4*>(Y)));
 }
 
 }  // extern "C"

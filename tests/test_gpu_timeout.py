@@ -29,12 +29,15 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(qbits, M, N, 
         assert qg.poll_status_code() == 0                            # the status word was cleared by the poll
     finally:
         qg.test_inject(0, -1)
-    # tensor memory was freed and the barriers of the next launch start clean: same result as before, bit for bit
+    # tensor memory was freed and the barriers of the next launch start clean: the next call is correct again.  (Two
+    # runs need not agree bit for bit: the even and the odd k-blocks of a tile are issued by two warps and accumulate
+    # in whichever order they reach the tensor cores, so the fp32 sums may differ in the last place.)
     again = qg.qgemm_dense(qbits, dA, dWq, dWs)
     assert qg.poll_status_code() == 0
-    assert torch.equal(again, good)
-    rows = slice(0, min(M, 64))
-    util.assert_close(util.host_bf16_f64(again[rows]), orc.qgemm_dense(qbits, A[rows], Wq, Ws), "after a timeout")
+    ref = orc.qgemm_dense(qbits, A, Wq, Ws)
+    util.assert_close(util.host_bf16_f64(again), ref, "after a timeout")
+    util.assert_close(util.host_bf16_f64(good), ref, "before the timeout")
+    assert float((again.float() - good.float()).abs().max()) <= 2e-2 * float(np.abs(ref).max())
 
 
 def test_the_hook_acts_on_one_launch_only():
