@@ -297,7 +297,24 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
                  counts=torch.empty(E, **i32), offsets=torch.empty(E + 1, **i32), row_pair=torch.empty(R, **i32),
                  pair_row=torch.empty(R, **i32), Xp=torch.empty((R, H), dtype=torch.bfloat16, device=dev),
                  Hh=torch.empty((R, F), dtype=torch.bfloat16, device=dev),
-                 Dw=torch.empty((R, H), dtype=torch.bfloat16, device=dev), y=torch.empty((M, H), dtype=torch.bfloat16, device=dev))
+                 Dw=torch.empty((R, H), dtype=torch.bfloat16, device=dev), y=torch.empty((M, H), dtype=torch.bfloat16, device=dev),
+                 acc=torch.zeros((M, H), dtype=torch.float32, device=dev))
+
+        def down_acc(it):
+            o["acc"].zero_()
+            chk(lib.moe_grouped_qgemm(ctx, qg.MODE_DOWN_ACCUM_F32, 4, R, E, H, F, P(o["Hh"]), P(o["offsets"]), P(W2q),
+                                      P(W2s), P(o["w"]), P(o["row_pair"]), k, P(o["acc"]), S), "down acc")
+        calls_fused = [
+            ("route", 0.0, 4.0 * M * E + 16.0 * R, lambda it: chk(lib.moe_route(
+                ctx, M, E, k, P(L), P(o["idx"]), P(o["w"]), P(o["counts"]), P(o["offsets"]), P(o["row_pair"]),
+                P(o["pair_row"]), None, None, H, P(ws), ws.numel(), S), "moe_route")),
+            ("gate_up", 2.0 * R * 2 * F * H, 0.0, lambda it: chk(lib.moe_grouped_qgemm_gather(
+                ctx, qg.MODE_GATE_UP_SILU, 4, M, R, E, 2 * F, H, P(X), P(o["row_pair"]), k, P(o["offsets"]), P(W1q),
+                P(W1s), None, P(o["Hh"]), S), "gate/up gather")),
+            ("down", 2.0 * R * F * H, 0.0, down_acc),
+            ("combine", 0.0, 6.0 * M * H, lambda it: chk(lib.moe_combine(
+                ctx, M, k, H, P(o["acc"]), qg.D_F32_ACC, None, None, P(o["y"]), S), "round")),
+        ]
         calls = [
             ("route_permute", 0.0, 4.0 * M * E + 16.0 * R + 2.0 * M * H + 2.0 * R * H, lambda it: chk(lib.moe_route(
                 ctx, M, E, k, P(L), P(o["idx"]), P(o["w"]), P(o["counts"]), P(o["offsets"]), P(o["row_pair"]),
@@ -329,6 +346,14 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
                "bound": "hbm (expert weights)" if t_hbm > t_tensor else "tensor"}
         row["frac_of_measured_peak"] = row["gemms_tflops"] / peak_tf
         row["frac_of_composite_bound"] = max(t_tensor, t_hbm) / (gemm_ms / n_it * 1e-3)
+        windows.pop()                       # one clock window per row: the one of the fused pass below
+        aggf = timed_calls(calls_fused, n_it)
+        gemm_ms_f = aggf["gate_up"][0] + aggf["down"][0]
+        row["fused"] = {"what": "route without row gather, gate/up with gathered loads, down with fp32 accumulate "
+                                "(its time includes the accumulator's zero fill), rounding",
+                        "call_us": {lab: v[0] / n_it * 1e3 for lab, v in aggf.items()},
+                        "gemms_tflops": gemm_fl / (gemm_ms_f * 1e-3) / 1e12,
+                        "layer_tok_per_s": M * n_it / (sum(v[0] for v in aggf.values()) * 1e-3)}
         out["moe"].append(row)
     out["_windows"] = windows
     return out
@@ -373,7 +398,9 @@ def run_ours(args):
              counts=torch.empty(E, **i32), offsets=torch.empty(E + 1, **i32), row_pair=torch.empty(R, **i32),
              pair_row=torch.empty(R, **i32), Xp=torch.empty((R, H), dtype=torch.bfloat16, device=dev),
              Hh=torch.empty((R, F), dtype=torch.bfloat16, device=dev),
-             Dw=torch.empty((R, H), dtype=torch.bfloat16, device=dev), y=torch.empty((M, H), dtype=torch.bfloat16, device=dev))
+             Dw=torch.empty((R, H), dtype=torch.bfloat16, device=dev), y=torch.empty((M, H), dtype=torch.bfloat16, device=dev),
+             acc=torch.zeros((M, H), dtype=torch.float32, device=dev))
+    fused = (args.moe_path == "fused")
     hC = [torch.empty((M, N), dtype=torch.bfloat16).pin_memory() for _, N, _ in DENSE_SET]
     hY = torch.empty((M, H), dtype=torch.bfloat16).pin_memory()
 
@@ -397,28 +424,47 @@ def run_ours(args):
             chk(lib.qgemm_dense(ctx, 8, M, N, K, P(A_list[i]), P(dW[i][1]), P(dW[i][2]), P(outC[i]), S), "qgemm_dense")
             if record:
                 e1.record(stream); gemm_events.append(("dense_q8_" + name, 2.0 * M * N * K, e0, e1))
-        if record:
-            r0 = torch.cuda.Event(enable_timing=True); r1 = torch.cuda.Event(enable_timing=True); r0.record(stream)
+        def ev():
+            e = torch.cuda.Event(enable_timing=True); e.record(stream); return e
+        if fused:
+            # routing tables only; the token rows are gathered by the gate/up kernel's loads, the routing-weighted
+            # sum over a token's experts is accumulated in fp32 by the down kernel's epilogue and rounded once
+            a = ev() if record else None
+            chk(lib.moe_route(ctx, M, E, k, P(L), P(o["idx"]), P(o["w"]), P(o["counts"]), P(o["offsets"]), P(o["row_pair"]),
+                              P(o["pair_row"]), None, None, H, P(ws), ws.numel(), S), "moe_route")
+            b = ev() if record else None
+            chk(lib.moe_grouped_qgemm_gather(ctx, qg.MODE_GATE_UP_SILU, 4, M, R, E, 2 * F, H, P(X), P(o["row_pair"]), k,
+                                             P(o["offsets"]), P(dW1q), P(dW1s), None, P(o["Hh"]), S), "gate/up (gather)")
+            c = ev() if record else None
+            o["acc"].zero_()
+            chk(lib.moe_grouped_qgemm(ctx, qg.MODE_DOWN_ACCUM_F32, 4, R, E, H, F, P(o["Hh"]), P(o["offsets"]), P(dW2q),
+                                      P(dW2s), P(o["w"]), P(o["row_pair"]), k, P(o["acc"]), S), "down (accumulate)")
+            d = ev() if record else None
+            chk(lib.moe_combine(ctx, M, k, H, P(o["acc"]), qg.D_F32_ACC, None, None, P(outY), S), "moe_combine (round)")
+            e = ev() if record else None
+            if record:
+                gemm_events.extend([("route", 0.0, a, b), ("moe_gate_up_q4", 2.0 * R * 2 * F * H, b, c),
+                                    ("moe_down_q4", 2.0 * R * F * H, c, d), ("combine", 0.0, d, e)])
+            return
+        a = ev() if record else None
         chk(lib.moe_route(ctx, M, E, k, P(L), P(o["idx"]), P(o["w"]), P(o["counts"]), P(o["offsets"]), P(o["row_pair"]),
                           P(o["pair_row"]), P(X), P(o["Xp"]), H, P(ws), ws.numel(), S), "moe_route")
-        if record:
-            r1.record(stream); gemm_events.append(("route_permute", 0.0, r0, r1))
-            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+        b = ev() if record else None
         chk(lib.moe_grouped_qgemm(ctx, qg.MODE_GATE_UP_SILU, 4, R, E, 2 * F, H, P(o["Xp"]), P(o["offsets"]), P(dW1q),
                                   P(dW1s), None, None, k, P(o["Hh"]), S), "moe_grouped_qgemm gate/up")
-        if record:
-            e1.record(stream); gemm_events.append(("moe_gate_up_q4", 2.0 * R * 2 * F * H, e0, e1))
-            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+        c = ev() if record else None
         chk(lib.moe_grouped_qgemm(ctx, qg.MODE_DOWN_WEIGHTED, 4, R, E, H, F, P(o["Hh"]), P(o["offsets"]), P(dW2q),
                                   P(dW2s), P(o["w"]), P(o["row_pair"]), k, P(o["Dw"]), S), "moe_grouped_qgemm down")
-        if record:
-            e1.record(stream); gemm_events.append(("moe_down_q4", 2.0 * R * F * H, e0, e1))
-            c0 = torch.cuda.Event(enable_timing=True); c1 = torch.cuda.Event(enable_timing=True); c0.record(stream)
+        d = ev() if record else None
         chk(lib.moe_combine(ctx, M, k, H, P(o["Dw"]), qg.D_BF16, P(o["pair_row"]), None, P(outY), S), "moe_combine")
+        e = ev() if record else None
         if record:
-            c1.record(stream); gemm_events.append(("combine", 0.0, c0, c1))
+            gemm_events.extend([("route", 0.0, a, b), ("moe_gate_up_q4", 2.0 * R * 2 * F * H, b, c),
+                                ("moe_down_q4", 2.0 * R * F * H, c, d), ("combine", 0.0, d, e)])
 
-    LAUNCHES_PER_STEP = 4 + 3 + 1 + 2 + 1   # dense x4, route (topk, scan, scatter), permute, grouped x2, combine
+    # dense x4, route (topk, scan, scatter), [permute,] grouped x2, combine or rounding (the fused path's zero fill of
+    # the fp32 accumulator is a memset, not counted)
+    LAUNCHES_PER_STEP = 4 + 3 + (0 if fused else 1) + 2 + 1
 
     def sync_all():
         torch.cuda.synchronize()
@@ -481,7 +527,10 @@ def run_ours(args):
     peak_tf, peak_hbm, peak_src = measured_peaks()
     # the HBM-bound calls: algorithmic bytes (route: logits in, indices/weights/permutation out; permute: X in, permuted
     # rows out; combine: weighted rows in, y out) against the measured copy bandwidth
-    hbm_bytes = {"route_permute": 4.0 * M * E + 16.0 * R + 2.0 * M * H + 2.0 * R * H, "combine": 2.0 * R * H + 2.0 * M * H}
+    if fused:   # route: logits in, tables out; "combine": zero fill and rounding of the fp32 accumulator
+        hbm_bytes = {"route": 4.0 * M * E + 16.0 * R, "combine": 4.0 * M * H + 2.0 * M * H}
+    else:
+        hbm_bytes = {"route": 4.0 * M * E + 16.0 * R + 2.0 * M * H + 2.0 * R * H, "combine": 2.0 * R * H + 2.0 * M * H}
     for lab, nbytes in hbm_bytes.items():
         gbs = nbytes / (detail[lab]["avg_us"] * 1e-6) / 1e9
         detail[lab].update({"bound": "hbm", "algorithmic_bytes": nbytes, "gbs": gbs, "frac_of_measured_hbm": gbs / peak_hbm})
@@ -511,7 +560,7 @@ def run_ours(args):
     gemm_ms = sum(v[1] for lab, v in agg.items() if v[0])
     gemm_fl = sum(v[0] for lab, v in agg.items() if v[0])
     dense_ms = dq[1] / ev_steps
-    moe_ms = sum(agg[lab][1] for lab in ("route_permute", "moe_gate_up_q4", "moe_down_q4", "combine")) / ev_steps
+    moe_ms = sum(agg[lab][1] for lab in ("route", "moe_gate_up_q4", "moe_down_q4", "combine")) / ev_steps
 
     # ---- end-to-end leg: host inputs in pinned memory, copies inside the timed region.  Steps are pipelined the way a
     # server would run them: step i's inputs are copied in on one stream while step i-1 computes and step i-2's
@@ -590,7 +639,8 @@ def run_ours(args):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"cfg1 dense Q8 layer set (QKV/O/gate-up/down, K=2048/8192) + cfg3 MoE Q4 layer "
                                    f"(H=2048,E=128,top-8,F=768), M={M} tokens per GPU",
-                       "l2": "inputs exceed L2: 403 MB of weights stream per step", "parallelism": f"replicas x{world}"},
+                       "l2": "inputs exceed L2: 403 MB of weights stream per step", "parallelism": f"replicas x{world}",
+                       "moe_path": args.moe_path},
             "tok_per_s": {"dense_q8_layer_set": world * M / (dense_ms * 1e-3), "moe_q4_layer": world * M / (moe_ms * 1e-3),
                           "definition": "tokens / time of that layer's calls; not a whole-model figure"},
             "gemm_only": {"tflops": gemm_fl / (gemm_ms * 1e-3) / 1e12, "frac_of_peak": gemm_fl / (gemm_ms * 1e-3) / 1e12 / peak_tf},
@@ -623,6 +673,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-configuration sweep block")
+    ap.add_argument("--moe-path", default="fused", choices=["fused", "staged"],
+                    help="fused: token gather in the gate/up loads + fp32 accumulate in the down epilogue; staged: "
+                         "permute, routing-weighted bf16 rows, slot-ordered combine (deterministic)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

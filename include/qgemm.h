@@ -157,6 +157,18 @@ int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int
                       const float* topk_w, const int32_t* row_pair, int k, void* Out, void* stream);
 
 /*
+ * The same grouped GEMM with the token permutation folded into its loads (Sec. 3.1 computes each expert's
+ * projection over the tokens routed to it; here they are read where they lie, so the permuted copy Xperm and its
+ * round trip through global memory never exist): row r of the input is X[row_pair[r] / k, :], X bf16 [M, K] in
+ * token order.  Everything else - segments, weights, modes, outputs in sorted-row order - is as in
+ * moe_grouped_qgemm; row_pair and k are always required.  Results are identical to
+ * moe_permute followed by moe_grouped_qgemm.
+ */
+int moe_grouped_qgemm_gather(qg_ctx* ctx, int mode, int qbits, int M, int R, int E, int N, int K, const void* X,
+                             const int32_t* row_pair, int k, const int32_t* expert_offsets, const void* Wq,
+                             const void* Wscale, const float* topk_w, void* Out, void* stream);
+
+/*
  * Combine (not described by the paper; plain definition): d_kind = QG_D_BF16:
  *   Y[t, :] = sum_{s = 0..k-1, in that order, fp32} w(t, s) * D[pair_row[t*k+s], :], with
  *   w = topk_w[t*k+s] if topk_w != NULL else 1 (rows already weighted).  D bf16 [M*k, H].

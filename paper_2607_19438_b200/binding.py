@@ -20,7 +20,7 @@ D_BF16, D_F32_ACC = 0, 1
 
 EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_route_workspace_bytes",
            "qgemm_dense",
-           "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_combine"]
+           "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_grouped_qgemm_gather", "moe_combine"]
 
 
 class QGemmError(RuntimeError):
@@ -54,6 +54,7 @@ def load():
         lib.moe_route_static.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         lib.moe_permute.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
         lib.moe_grouped_qgemm.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp]
+        lib.moe_grouped_qgemm_gather.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp]
         lib.moe_combine.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp, vp, vp]
         _lib = lib
     return _lib
@@ -188,6 +189,25 @@ def moe_grouped_qgemm(mode, qbits, Ain, offsets, Wq, Wscale, topk_w=None, row_pa
     _check(load().moe_grouped_qgemm(context(), mode, qbits, R, E, N, K, _ptr(Ain), _ptr(offsets), _ptr(Wq),
                                     _ptr(Wscale), _ptr(topk_w), _ptr(row_pair), k, _ptr(out), _stream()),
            "moe_grouped_qgemm")
+    return out
+
+
+def moe_grouped_qgemm_gather(mode, qbits, X, row_pair, k, offsets, Wq, Wscale, topk_w=None, out=None):
+    """moe_grouped_qgemm whose input row r is X[row_pair[r] // k] (X bf16 [M,K] in token order)."""
+    M, K = X.shape
+    R = row_pair.numel()
+    E, N = Wscale.shape[0], Wscale.shape[1]
+    dev = X.device
+    if out is None:
+        if mode == MODE_GATE_UP_SILU:
+            out = torch.empty((R, N // 2), dtype=torch.bfloat16, device=dev)
+        elif mode == MODE_DOWN_ACCUM_F32:
+            out = torch.zeros((M, N), dtype=torch.float32, device=dev)
+        else:
+            out = torch.empty((R, N), dtype=torch.bfloat16, device=dev)
+    _check(load().moe_grouped_qgemm_gather(context(), mode, qbits, M, R, E, N, K, _ptr(X), _ptr(row_pair), k,
+                                           _ptr(offsets), _ptr(Wq), _ptr(Wscale), _ptr(topk_w), _ptr(out), _stream()),
+           "moe_grouped_qgemm_gather")
     return out
 
 

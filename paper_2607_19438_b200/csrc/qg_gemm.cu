@@ -39,6 +39,7 @@ constexpr int MAX_E = 1024;
 struct GemmParams {
     int mode, R, N, K, E, k;
     int n_wt;                   // 128-row weight tiles per expert (64 gate + 64 up rows each in gate/up mode)
+    int gather_k;               // > 0: input row r is X[row_pair[r] / gather_k] (token gather folded into the loads)
     const int32_t* offsets;     // device expert offsets [E+1]; nullptr: one segment [0, R)
     void* out;
     const float* topk_w;
@@ -398,6 +399,17 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const Tile tl = tile_at(jt);
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const int row0 = tl.tok0 + static_cast<int>(rank) * (n_mma >> 1);   // B rows split at N / 2
+            // Gathered input: lane l fetches rows 4 l .. 4 l + 3 of this CTA's half tile from the token rows the
+            // routing table names (rows past the segment end fetch token 0: computed, never stored).
+            const int groups = n_mma >> 3;                                      // (n_mma / 2) / 4
+            int g0 = 0, g1 = 0, g2 = 0, g3 = 0;
+            if (p.gather_k > 0 && lane < groups) {
+                const int r = row0 + 4 * lane;
+                if (r < tl.tok_end) g0 = p.row_pair[r] / p.gather_k;
+                if (r + 1 < tl.tok_end) g1 = p.row_pair[r + 1] / p.gather_k;
+                if (r + 2 < tl.tok_end) g2 = p.row_pair[r + 2] / p.gather_k;
+                if (r + 3 < tl.tok_end) g3 = p.row_pair[r + 3] / p.gather_k;
+            }
             for (int kb = 0; kb < nkb; kb += 2) {
                 QG_T0();
                 // a stage is free once the MMAs that read it eight k-blocks ago are done (even and odd stages
@@ -405,7 +417,16 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 if (!wait_bar<false>(done(s), ph ^ 1u, abort_flag, p) ||
                     !wait_bar<false>(done(s + 1), ph ^ 1u, abort_flag, p)) { ok = false; break; }
                 QG_ACC(0);
-                if (lane == 0) {
+                if (p.gather_k > 0) {
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        if (jt == 0 && kb + j == p.skip_kb) continue;      // test hook: this stage never fills
+                        if (lane == 0 && rank == 0) mbar_arrive_expect_tx(full(s + j), 2u * groups * 512u);
+                        if (lane < groups)
+                            tma_gather4_pair(sbase + C::OFF_X + (s + j) * C::X_BYTES + lane * 512, &tm_x, (kb + j) * BK,
+                                             g0, g1, g2, g3, full_leader + 8u * (s + j));
+                    }
+                } else if (lane == 0) {
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
                         if (jt == 0 && kb + j == p.skip_kb) continue;      // test hook: this stage never fills
@@ -757,14 +778,15 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
 }
 
 template <int QBITS, int BT, int EPI>
-static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, const void* Wq, const void* Ws,
+static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_rows, const void* Wq, const void* Ws,
                        cudaStream_t st) {
     using C = Cfg<QBITS, BT>;
     static_assert(C::SMEM_BYTES <= 232448, "shared memory budget");
     const CUtensorMap *tm_x, *tm_w, *tm_s;       // cached in the context: the same buffers recur every layer and step
     const uint64_t wrows = static_cast<uint64_t>(p.E) * p.N;
-    int rc = get_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, p.R, BK, C::XH_ROWS,
-                         CU_TENSOR_MAP_SWIZZLE_128B);
+    // activations: a box of half a token tile, or of a single row when the rows are gathered four at a time
+    int rc = get_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, x_rows, BK,
+                         p.gather_k > 0 ? 1 : C::XH_ROWS, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc == QG_OK)
         rc = get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (QBITS == 8) ? p.K : p.K / 2, wrows,
                          C::RAW_ROW, 64, (QBITS == 8) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
@@ -813,8 +835,8 @@ static int pick_token_tile(const qg_ctx* ctx, int M, int n_wt, int K) {
     return best;
 }
 
-static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in, const void* X, const void* Wq,
-                         const void* Ws, cudaStream_t st) {
+static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in, const void* X, int x_rows,
+                         const void* Wq, const void* Ws, cudaStream_t st) {
     GemmParams p = p_in;
     if (ctx->force_bt) bt = ctx->force_bt;       // QG_FORCE_BT, read when the context was created (tile-shape sweeps)
     p.status = ctx->d_status;
@@ -827,9 +849,9 @@ static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in,
     const int epi = (p.mode == QG_MODE_GATE_UP_SILU) ? 1 : (p.mode == QG_MODE_DOWN_ACCUM_F32) ? 2 : 0;
 #define QG_LAUNCH(Q, B)                                                                 \
     do {                                                                                \
-        if (epi == 0) return launch_gemm<Q, B, 0>(ctx, p, X, Wq, Ws, st);               \
-        if (epi == 1) return launch_gemm<Q, B, 1>(ctx, p, X, Wq, Ws, st);               \
-        return launch_gemm<Q, B, 2>(ctx, p, X, Wq, Ws, st);                             \
+        if (epi == 0) return launch_gemm<Q, B, 0>(ctx, p, X, x_rows, Wq, Ws, st);       \
+        if (epi == 1) return launch_gemm<Q, B, 1>(ctx, p, X, x_rows, Wq, Ws, st);       \
+        return launch_gemm<Q, B, 2>(ctx, p, X, x_rows, Wq, Ws, st);                     \
     } while (0)
     if (qbits == QG_Q8) {
         if (bt == 256) QG_LAUNCH(8, 256);
@@ -860,12 +882,12 @@ int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, cons
     p.n_wt = (N + qg::BW - 1) / qg::BW;
     p.offsets = nullptr; p.out = Cout; p.topk_w = nullptr; p.row_pair = nullptr;
     const int bt = qg::pick_token_tile(ctx, M, p.n_wt, K);
-    return qg::dispatch_gemm(ctx, qbits, bt, p, A, Wq, Wscale, static_cast<cudaStream_t>(stream));
+    return qg::dispatch_gemm(ctx, qbits, bt, p, A, M, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 
-int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int K, const void* Ain,
-                      const int32_t* expert_offsets, const void* Wq, const void* Wscale, const float* topk_w,
-                      const int32_t* row_pair, int k, void* Out, void* stream) {
+static int grouped_impl(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int K, const void* Ain, int in_rows,
+                        int gather_k, const int32_t* expert_offsets, const void* Wq, const void* Wscale,
+                        const float* topk_w, const int32_t* row_pair, int k, void* Out, void* stream) {
     if (!ctx) return QG_ERR_NULL;
     if (R == 0) return QG_OK;     // nothing to do: empty tensors may carry null pointers
     if (!Ain || !expert_offsets || !Wq || !Wscale || !Out) return QG_ERR_NULL;
@@ -873,19 +895,37 @@ int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int
     if (mode < QG_MODE_PLAIN || mode > QG_MODE_DOWN_ACCUM_F32) return QG_ERR_SHAPE;
     if (R < 0 || E < 1 || E > qg::MAX_E || N < 8 || N % 8 || K < 256 || K % 256) return QG_ERR_SHAPE;
     if (mode == QG_MODE_GATE_UP_SILU && (N % 128)) return QG_ERR_SHAPE;  // F % 64 == 0
-    if (mode >= QG_MODE_DOWN_WEIGHTED && (!topk_w || !row_pair)) return QG_ERR_NULL;
-    if (mode == QG_MODE_DOWN_ACCUM_F32 && k < 1) return QG_ERR_SHAPE;
+    if ((mode >= QG_MODE_DOWN_WEIGHTED || gather_k > 0) && !row_pair) return QG_ERR_NULL;
+    if (mode >= QG_MODE_DOWN_WEIGHTED && !topk_w) return QG_ERR_NULL;
+    if ((mode == QG_MODE_DOWN_ACCUM_F32 || gather_k > 0) && k < 1) return QG_ERR_SHAPE;
+    if (gather_k > 0 && in_rows < 1) return QG_ERR_SHAPE;
     if (static_cast<long long>(E) * N > 0x7FFFFFFF) return QG_ERR_SHAPE;
     if (!qg::aligned16(Ain) || !qg::aligned16(Wq) || !qg::aligned16(Wscale) || !qg::aligned16(Out)) return QG_ERR_ALIGN;
     if (const int rc = qg::check_device(ctx)) return rc;
     qg::GemmParams p{};
     p.mode = mode; p.R = R; p.N = N; p.K = K; p.E = E; p.k = (k < 1) ? 1 : k;
     p.n_wt = (mode == QG_MODE_GATE_UP_SILU) ? (N / 128) : (N + qg::BW - 1) / qg::BW;
+    p.gather_k = gather_k;
     p.offsets = expert_offsets; p.out = Out; p.topk_w = topk_w; p.row_pair = row_pair;
     // expected rows per expert decide the token tile; 192 keeps two accumulators, so the short main loops of
     // expert tiles overlap their epilogues
     const int bt = (R / E > 100) ? 192 : 128;
-    return qg::dispatch_gemm(ctx, qbits, bt, p, Ain, Wq, Wscale, static_cast<cudaStream_t>(stream));
+    return qg::dispatch_gemm(ctx, qbits, bt, p, Ain, in_rows, Wq, Wscale, static_cast<cudaStream_t>(stream));
+}
+
+int moe_grouped_qgemm(qg_ctx* ctx, int mode, int qbits, int R, int E, int N, int K, const void* Ain,
+                      const int32_t* expert_offsets, const void* Wq, const void* Wscale, const float* topk_w,
+                      const int32_t* row_pair, int k, void* Out, void* stream) {
+    return grouped_impl(ctx, mode, qbits, R, E, N, K, Ain, R, 0, expert_offsets, Wq, Wscale, topk_w, row_pair, k, Out,
+                        stream);
+}
+
+int moe_grouped_qgemm_gather(qg_ctx* ctx, int mode, int qbits, int M, int R, int E, int N, int K, const void* X,
+                             const int32_t* row_pair, int k, const int32_t* expert_offsets, const void* Wq,
+                             const void* Wscale, const float* topk_w, void* Out, void* stream) {
+    if (M < 1 && R > 0) return QG_ERR_SHAPE;
+    return grouped_impl(ctx, mode, qbits, R, E, N, K, X, M, k, expert_offsets, Wq, Wscale, topk_w, row_pair, k, Out,
+                        stream);
 }
 
 }  // extern "C"

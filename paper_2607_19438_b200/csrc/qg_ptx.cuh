@@ -113,6 +113,17 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap,
         : "memory");
 }
 
+// Row gather for a CTA pair: four rows y0..y3 of a 2-D tensor (tensor map with a box of one row), columns x .., land
+// as four consecutive rows at dst; completion bytes on `bar_cluster` (own CTA or the peer).  No multicast.
+__device__ __forceinline__ void tma_gather4_pair(uint32_t dst, const void* tmap, int x, int y0, int y1, int y2, int y3,
+                                                 uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3), "r"(bar_cluster)
+        : "memory");
+}
+
 // ---------------------------------------------------------------- tcgen05 / TMEM
 // CTA-pair (cta_group::2) forms: allocation is issued by the same warp of both CTAs; the MMA is issued by one
 // thread of the even CTA and uses both CTAs' operands; commit signals the barrier at the same offset in both.

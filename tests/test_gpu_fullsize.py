@@ -90,6 +90,24 @@ def test_moe_config3_full_size_selected_experts(M, skewed):
     D_sub = util.host_bf16_f64(Dw[torch.from_numpy(rows_needed.astype(np.int64)).cuda()])
     sub_pair_row = np.arange(rows_needed.size, dtype=np.int32)            # token i of the subset owns rows i k .. i k + k - 1
     util.assert_close(yh[toks], orc.combine(D_sub, sub_pair_row, k), "combine")
+    # the fused flavour the benchmark times: rows gathered by the gate/up kernel's loads, fp32 accumulate in the down
+    # epilogue, one rounding.  Gate/up again on the selected experts' rows; the layer output against the staged one,
+    # whose stages were checked above (both carry their own rounding: twice the single-result tolerance).
+    Hh_f = qg.moe_grouped_qgemm_gather(qg.MODE_GATE_UP_SILU, qbits, d["X"], r["row_pair"], k, r["offsets"], d["W1q"], d["W1s"])
+    acc = qg.moe_grouped_qgemm(qg.MODE_DOWN_ACCUM_F32, qbits, Hh_f, r["offsets"], d["W2q"], d["W2s"],
+                               topk_w=r["topk_w"].view(-1), row_pair=r["row_pair"], k=k, M=M)
+    y_f = qg.moe_combine(acc, None, k, d_kind=qg.D_F32_ACC)
+    qg.poll_status()
+    for e in experts:
+        seg = slice(int(offsets[e]), int(offsets[e + 1]))
+        if seg.stop == seg.start:
+            continue
+        off1 = np.array([0, seg.stop - seg.start], np.int32)
+        GU = orc.grouped_gemm(qbits, orc.bf16_to_f64(Xp[seg]), off1, W1q[e:e + 1], W1s[e:e + 1])
+        util.assert_close(util.host_bf16_f64(Hh_f[seg]), orc.silu_mul(GU), f"gathered gate/up expert {e}")
+    yf = util.host_bf16_f64(y_f)
+    mx, rmax, fro = util.errors(yf, yh)
+    assert np.all(np.isfinite(yf)) and mx <= 2 * util.MAX_ERR_FACTOR * rmax and fro <= 2 * util.REL_FRO, (mx, rmax, fro)
 
 
 def test_config4_gate_up_projection_sampled():

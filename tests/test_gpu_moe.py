@@ -131,3 +131,34 @@ def test_grouped_short_k_many_tiles_per_pair(qbits, E, rows, K, N, mode):
     elif mode == qg.MODE_DOWN_WEIGHTED:
         ref = ref * w[row_pair].astype(np.float64)[:, None]
     util.assert_close(util.host_bf16_f64(out), ref, "grouped short K")
+
+
+GATHER = [("small-q4", 4, 96, 256, 8, 256, 2, False), ("ragged-q8", 8, 333, 512, 5, 256, 3, False),
+          ("skewed-q4", 4, 512, 512, 32, 256, 8, True), ("long-q4", 4, 700, 256, 2, 256, 1, False),
+          ("cfg3-128", 4, 128, 2048, 128, 768, 8, True)]
+
+
+@pytest.mark.parametrize("name,qbits,M,H,E,F,k,skewed", GATHER, ids=[c[0] for c in GATHER])
+def test_gather_in_load_equals_permute_then_gemm(name, qbits, M, H, E, F, k, skewed):
+    """moe_grouped_qgemm_gather reads the token rows through the routing table instead of from a permuted copy: its
+    gate/up output must match the oracle, and the whole layer built on it (no Xperm, accumulate epilogue, rounding)
+    must match the unrounded fp64 layer."""
+    logits, X, W1q, W1s, W2q, W2s = synth.moe_problem(qbits, M, H, E, F, seed=2, skewed=skewed)
+    dX, dW1q, dW1s, dW2q, dW2s = util.dev_bf16(X), util.dev(W1q), util.dev_f16(W1s), util.dev(W2q), util.dev_f16(W2s)
+    r = qg.moe_route(util.dev(logits), k)                                   # no row gather here
+    Hh = qg.moe_grouped_qgemm_gather(qg.MODE_GATE_UP_SILU, qbits, dX, r["row_pair"], k, r["offsets"], dW1q, dW1s)
+    Gp = qg.moe_grouped_qgemm_gather(qg.MODE_PLAIN, qbits, dX, r["row_pair"], k, r["offsets"], dW1q, dW1s)
+    acc = qg.moe_grouped_qgemm(qg.MODE_DOWN_ACCUM_F32, qbits, Hh, r["offsets"], dW2q, dW2s, topk_w=r["topk_w"].view(-1),
+                               row_pair=r["row_pair"], k=k, M=M)
+    y = qg.moe_combine(acc, None, k, d_kind=qg.D_F32_ACC)
+    qg.poll_status()
+    o = orc.moe_layer(qbits, logits, X, W1q, W1s, W2q, W2s, k)
+    assert np.array_equal(r["row_pair"].cpu().numpy(), o["row_pair"])
+    util.assert_close(util.host_bf16_f64(Gp), o["GU"], "gathered plain")
+    util.assert_close(util.host_bf16_f64(Hh), o["Hh"], "gathered gate/up+silu")
+    util.assert_close(util.host_bf16_f64(y), o["y"], "layer (gather + accumulate)")
+    # and the two ways of feeding the kernel agree to the last bit on a stage with one k-block order per tile
+    Xp = qg.moe_permute(dX, r["row_pair"], k)
+    Hh2 = qg.moe_grouped_qgemm(qg.MODE_GATE_UP_SILU, qbits, Xp, r["offsets"], dW1q, dW1s)
+    qg.poll_status()
+    util.assert_close(util.host_bf16_f64(Hh2), o["Hh"], "permute + gemm")
