@@ -230,9 +230,13 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
 
     def timed_calls(calls, n_iter):
         """calls: list of (label, flops, bytes, fn(it)).  Returns {label: [total_ms, flops, bytes]} over n_iter passes."""
-        t_w = time.perf_counter()          # warm up for at least 60 ms: a short burst after a host-side pause would
-        it = 0                             # otherwise be timed while the SM clock is still ramping up
-        while it < 3 or time.perf_counter() - t_w < 0.06:
+        # burst regime, like the headline region: a pause lets the board's power average settle, then at least 15 ms
+        # of warm-up passes bring the SM clock back up before the short timed region
+        torch.cuda.synchronize()
+        time.sleep(0.3)
+        t_w = time.perf_counter()
+        it = 0
+        while it < 3 or time.perf_counter() - t_w < 0.015:
             for _, _, _, fn in calls:
                 fn(it)
             it += 1
@@ -281,6 +285,34 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
         row["frac_of_measured_peak"] = row["set_tflops"] / peak_tf
         out["dense"].append(row)
         del W, A, Cs
+        torch.cuda.empty_cache()
+
+    # small batches (decode side): weight streaming, against the measured HBM copy bandwidth
+    out["small_m"] = []
+    for name in ("cfg1_q8", "cfg2_q4"):
+        qbits, layers = LAYER_SETS[name]
+        wbytes = sum(N * K * (1.0625 if qbits == 8 else 0.5625) for _, N, K in layers)
+        ncopy = max(2, int(2 * L2_BYTES // wbytes) + 1)
+        W = [[weights(qbits, N, K) for _, N, K in layers] for _ in range(ncopy)]
+        for M in (1, 4, 16):
+            A = {K: torch.randn((M, K), device=dev, generator=g).to(torch.bfloat16) for K in {K for _, _, K in layers}}
+            Cs = [torch.empty((M, N), dtype=torch.bfloat16, device=dev) for _, N, _ in layers]
+            for api, label in ((lib.qgemm_small_m, "qgemm_small_m"), (lib.qgemm_dense, "qgemm_dense")):
+                calls = []
+                for i, (lab, N, K) in enumerate(layers):
+                    def fn(it, i=i, N=N, K=K, api=api):
+                        q, sc = W[it % ncopy][i]
+                        chk(api(ctx, qbits, M, N, K, P(A[K]), P(q), P(sc), P(Cs[i]), S), label)
+                    calls.append((lab, 2.0 * M * N * K, N * K * (1.0625 if qbits == 8 else 0.5625) + 2.0 * M * (N + K), fn))
+                agg = timed_calls(calls, iters)
+                tot_ms = sum(v[0] for v in agg.values()); tot_b = sum(v[2] for v in agg.values()) * iters
+                out["small_m"].append({"set": name, "M": M, "call": label,
+                                       "gemm_us": {lab: v[0] / iters * 1e3 for lab, v in agg.items()},
+                                       "gemm_gbs": {lab: v[2] * iters / (v[0] * 1e-3) / 1e9 for lab, v in agg.items()},
+                                       "set_gbs": tot_b / (tot_ms * 1e-3) / 1e9,
+                                       "frac_of_measured_hbm": tot_b / (tot_ms * 1e-3) / 1e9 / peak_hbm,
+                                       "tok_per_s": M * iters / (tot_ms * 1e-3)})
+        del W
         torch.cuda.empty_cache()
 
     H, E, k, F = MOE["H"], MOE["E"], MOE["k"], MOE["F"]
@@ -628,7 +660,7 @@ def run_ours(args):
         qg.poll_status()
         sweep["clocks"] = sampler3.stop()
         wins = sweep.pop("_windows")
-        for row, (t0, t1) in zip(sweep["dense"] + sweep["moe"], wins):
+        for row, (t0, t1) in zip(sweep["dense"] + sweep["small_m"] + sweep["moe"], wins):
             row["clocks"] = clocks_in_window(getattr(sampler3, "samples", []), t0 - 0.02, t1 + 0.02)
     if rank == 0:
         dense_h0, moe_h0 = dense_h, moe_h
@@ -666,6 +698,34 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_case(args):
+    """One small case, a few passes, no timing: a target for profiler captures (one kernel, few launches)."""
+    import ctypes as C
+    import torch
+    from paper_2607_19438_b200 import binding as qg
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    lib, ctx = qg.load(), qg.context(0)
+    g = torch.Generator(device=dev); g.manual_seed(0)
+    H, F, k = MOE["H"], MOE["F"], MOE["k"]
+    E, M = 16, 256
+    R = M * k
+    W1q = torch.randint(0, 256, (E, 2 * F, H // 2), dtype=torch.uint8, device=dev, generator=g)
+    W2q = torch.randint(0, 256, (E, H, F // 2), dtype=torch.uint8, device=dev, generator=g)
+    W1s = (torch.randn((E, 2 * F, H // 32), device=dev, generator=g).abs() * (0.02 / 7)).to(torch.float16)
+    W2s = (torch.randn((E, H, F // 32), device=dev, generator=g).abs() * (0.02 / 7)).to(torch.float16)
+    L = torch.randn((M, E), device=dev, generator=g)
+    X = torch.randn((M, H), device=dev, generator=g).to(torch.bfloat16)
+    for _ in range(3):
+        r = qg.moe_route(L, k, X=X)
+        Hh = qg.moe_grouped_qgemm(qg.MODE_GATE_UP_SILU, 4, r["Xperm"], r["offsets"], W1q, W1s)
+        Dw = qg.moe_grouped_qgemm(qg.MODE_DOWN_WEIGHTED, 4, Hh, r["offsets"], W2q, W2s, topk_w=r["topk_w"].view(-1),
+                                  row_pair=r["row_pair"], k=k)
+        qg.moe_combine(Dw, r["pair_row"], k)
+    qg.poll_status()
+    print(json.dumps({"case": args.case, "E": E, "M": M, "rows_per_expert": R / E, "passes": 3}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -673,11 +733,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-configuration sweep block")
-    ap.add_argument("--moe-path", default="fused", choices=["fused", "staged"],
-                    help="fused: token gather in the gate/up loads + fp32 accumulate in the down epilogue; staged: "
-                         "permute, routing-weighted bf16 rows, slot-ordered combine (deterministic)")
+    ap.add_argument("--moe-path", default="staged", choices=["fused", "staged"],
+                    help="staged: permute, routing-weighted bf16 rows, slot-ordered combine (deterministic, faster on "
+                         "B200); fused: token gather in the gate/up loads + fp32 accumulate in the down epilogue")
+    ap.add_argument("--case", default=None, choices=["moe_small"],
+                    help="run one small case a few times and exit (for profiler captures): moe_small = the cfg-3 MoE "
+                         "layer shape with 16 experts and 256 tokens (128 rows per expert)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

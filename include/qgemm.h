@@ -14,7 +14,7 @@
  *     (a cudaStream_t passed as void*; NULL = the legacy default stream);
  *   - the context's device must be the calling thread's current device (else QG_ERR_DEVICE); a
  *     context and its calls belong to one host thread and one stream at a time (it caches tensor
- *     maps and owns the split-K scratch of qgemm_dense);
+ *     maps and owns the K-slice scratch of qgemm_small_m);
  *   - return value: QG_OK (0) or a negative QG_ERR_* code; an error is detected before anything is
  *     launched, so the outputs are untouched; nothing aborts, traps or throws;
  *   - there is no fallback path: a shape the kernels do not accept is an error (the paper's
@@ -70,7 +70,7 @@ enum {
 enum { QG_D_BF16 = 0, QG_D_F32_ACC = 1 };
 
 /* Create / destroy a context for `device`.  Only these two allocate device memory (the status word and the
- * split-K scratch of qgemm_dense, about 20 MB); qg_create leaves the caller's current device as it was. */
+ * scratch of qgemm_small_m, 32 MB); qg_create leaves the caller's current device as it was. */
 int qg_create(qg_ctx** out, int device);
 int qg_destroy(qg_ctx* ctx);
 const char* qg_strerror(int code);
@@ -96,6 +96,25 @@ int qg_test_inject(qg_ctx* ctx, unsigned wait_limit_polls, int skip_kblock);
  */
 int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq,
                 const void* Wscale, void* C, void* stream);
+
+/*
+ * Dense feed-forward gate/up projection with the gating fused (Sec. 3.1 applies SiLU on the accumulators of the MoE
+ * gate/up projection; this is the same epilogue for a dense layer): Wq holds 2F rows, rows 0..F-1 the gate and
+ * F..2F-1 the up projection (F % 64 == 0);  Out[m, f] = silu(G[m, f]) * U[m, f], bf16 [M, F].
+ */
+int qgemm_dense_gate_up_silu(qg_ctx* ctx, int qbits, int M, int F, int K, const void* A, const void* Wq,
+                             const void* Wscale, void* Out, void* stream);
+
+/*
+ * The same product for 1 <= M <= 16 tokens (else QG_ERR_SHAPE): the decode-side and small verification-batch
+ * regime that Sec. 2.3 describes as bound by memory bandwidth and Sec. 5.2 names as future work for the tensor
+ * path.  Every weight byte is used once, so this kernel streams the packed weights at HBM speed and reduces its
+ * K slices in a fixed order (results do not depend on scheduling).  Same formats, constraints and numerics
+ * (weights rounded once to bf16, fp32 accumulate) as qgemm_dense; uses the context's scratch, so calls on one
+ * context must not overlap on the GPU.
+ */
+int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq,
+                  const void* Wscale, void* C, void* stream);
 
 /*
  * Routing (Sec. 3.1 only presupposes that tokens have been assigned to experts; defined here): for every token the k

@@ -19,7 +19,7 @@ MODE_PLAIN, MODE_GATE_UP_SILU, MODE_DOWN_WEIGHTED, MODE_DOWN_ACCUM_F32 = 0, 1, 2
 D_BF16, D_F32_ACC = 0, 1
 
 EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_route_workspace_bytes",
-           "qgemm_dense",
+           "qgemm_dense", "qgemm_small_m", "qgemm_dense_gate_up_silu",
            "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_grouped_qgemm_gather", "moe_combine"]
 
 
@@ -50,6 +50,8 @@ def load():
         lib.qg_test_inject.argtypes = [C.c_void_p, C.c_uint, C.c_int]
         vp, ci = C.c_void_p, C.c_int
         lib.qgemm_dense.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
+        lib.qgemm_small_m.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
+        lib.qgemm_dense_gate_up_silu.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
         lib.moe_route.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp, C.c_size_t, vp]
         lib.moe_route_static.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         lib.moe_permute.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
@@ -121,6 +123,28 @@ def qgemm_dense(qbits, A, Wq, Wscale, out=None):
         out = torch.empty((M, N), dtype=torch.bfloat16, device=A.device)
     _check(load().qgemm_dense(context(), qbits, M, N, K, _ptr(A), _ptr(Wq), _ptr(Wscale), _ptr(out), _stream()),
            "qgemm_dense")
+    return out
+
+
+def qgemm_small_m(qbits, A, Wq, Wscale, out=None):
+    """qgemm_dense for 1..16 tokens: the weight-streaming kernel."""
+    M, K = A.shape
+    N = Wq.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=A.device)
+    _check(load().qgemm_small_m(context(), qbits, M, N, K, _ptr(A), _ptr(Wq), _ptr(Wscale), _ptr(out), _stream()),
+           "qgemm_small_m")
+    return out
+
+
+def qgemm_dense_gate_up_silu(qbits, A, Wq, Wscale, out=None):
+    """A bf16 [M,K]; Wq [2F,K(/2)] (gate rows then up rows) -> silu(gate) * up, bf16 [M,F]."""
+    M, K = A.shape
+    F = Wq.shape[0] // 2
+    if out is None:
+        out = torch.empty((M, F), dtype=torch.bfloat16, device=A.device)
+    _check(load().qgemm_dense_gate_up_silu(context(), qbits, M, F, K, _ptr(A), _ptr(Wq), _ptr(Wscale), _ptr(out),
+                                           _stream()), "qgemm_dense_gate_up_silu")
     return out
 
 

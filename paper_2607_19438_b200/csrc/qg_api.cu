@@ -56,8 +56,14 @@ int qg_create(qg_ctx** out, int device) {
         return QG_ERR_CUDA;
     }
     ctx->encode_tiled = reinterpret_cast<decltype(ctx->encode_tiled)>(fn);
-    if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) {
+    ctx->gemv_partial_bytes = static_cast<size_t>(32) << 20;
+    ctx->gemv_ticket_count = 4096;
+    if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess ||
+        cudaMalloc(&ctx->gemv_partial, ctx->gemv_partial_bytes) != cudaSuccess ||
+        cudaMalloc(&ctx->gemv_tickets, sizeof(int) * ctx->gemv_ticket_count) != cudaSuccess ||
+        cudaMemset(ctx->gemv_tickets, 0, sizeof(int) * ctx->gemv_ticket_count) != cudaSuccess) {
         cudaGetLastError();
+        cudaFree(ctx->d_status); cudaFree(ctx->gemv_partial); cudaFree(ctx->gemv_tickets);
         delete ctx;
         return QG_ERR_CUDA;
     }
@@ -68,7 +74,8 @@ int qg_create(qg_ctx** out, int device) {
 int qg_destroy(qg_ctx* ctx) {
     if (!ctx) return QG_ERR_NULL;
     cudaFree(ctx->d_status);
-    if (ctx->d_ws) cudaFree(ctx->d_ws);
+    cudaFree(ctx->gemv_partial);
+    cudaFree(ctx->gemv_tickets);
     delete ctx;
     return QG_OK;
 }

@@ -28,6 +28,7 @@
 #include "qg_internal.h"
 #include "qg_ptx.cuh"
 #include "qg_profile.cuh"
+#include "qg_dequant.cuh"
 
 namespace qg {
 
@@ -133,56 +134,6 @@ __device__ __forceinline__ bool spin_wait_bar(uint32_t bar, uint32_t parity, vol
     for (int it = 0; it < 64; ++it)
         if (mbar_test_wait_cluster(bar, parity)) return true;
     return wait_bar<true>(bar, parity, abort_flag, p);
-}
-
-__device__ __forceinline__ uint32_t bf16x2(float lo, float hi) {
-    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&b);
-}
-
-// Dequantisation arithmetic.  A code byte c (0..255) dropped into byte 1 of 0x43000000 reads as the float
-// 128 + c / 256, so q * s = fma(f, 256 s, -(32768 + 256 z) s) for the code's zero point z (128 for the sign-flipped
-// int8 byte, 8 for a nibble): both constants and the result are exact in fp32, one rounding (to bf16) follows.
-// Per weight: one byte permute builds f from a code byte and the magic word, half a packed two-float fused
-// multiply-add (fma.rn.f32x2, each lane IEEE-exact as fmaf) converts, half a packed conversion rounds to bf16x2.
-__device__ __forceinline__ uint32_t fma2_bf16x2(uint32_t a0, uint32_t a1, uint64_t m, uint64_t c) {
-    uint32_t r;     // bf16(a0 * m.lo + c.lo) | bf16(a1 * m.hi + c.hi) << 16
-    asm("{\n\t.reg .b64 t;\n\t.reg .b32 lo, hi;\n\t"
-        "mov.b64 t, {%1, %2};\n\t"
-        "fma.rn.f32x2 t, t, %3, %4;\n\t"
-        "mov.b64 {lo, hi}, t;\n\t"
-        "cvt.rn.bf16x2.f32 %0, hi, lo;\n\t}"
-        : "=r"(r) : "r"(a0), "r"(a1), "l"(m), "l"(c));
-    return r;
-}
-__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
-    return static_cast<uint64_t>(__float_as_uint(lo)) | (static_cast<uint64_t>(__float_as_uint(hi)) << 32);
-}
-template <int BYTE>
-__device__ __forceinline__ uint32_t code_byte_to_float(uint32_t x, uint32_t magic) {   // bits of 128 + byte BYTE of x / 256
-    return __byte_perm(x, magic, 0x7404 + (BYTE << 4));
-}
-
-// 4 int8 codes (one word) -> 4 bf16 = q * scale.  m2 = {256 s, 256 s}, c2 = {-32896 s, -32896 s}.
-__device__ __forceinline__ void dq8_word(uint32_t x, uint64_t m2, uint64_t c2, uint32_t magic, uint32_t& o0, uint32_t& o1) {
-    x ^= 0x80808080u;                            // byte = q + 128
-    o0 = fma2_bf16x2(code_byte_to_float<0>(x, magic), code_byte_to_float<1>(x, magic), m2, c2);
-    o1 = fma2_bf16x2(code_byte_to_float<2>(x, magic), code_byte_to_float<3>(x, magic), m2, c2);
-}
-
-// 8 4-bit codes (one word, nibble i = weight i, code u = q + 8) -> 8 bf16.  The nibbles are first spread into
-// the bytes of two words in k order (mask the even and the odd nibbles, interleave their bytes), then converted like
-// the 8-bit codes.  Both permutes of a packed multiply-add read the same word: with operands from two different
-// words the compiler needs a register move per weight to form the pair (measured with the opcode counters).
-// m2 = {256 s, 256 s}, c2 = {-32776 s, -32776 s}.
-__device__ __forceinline__ void dq4_word(uint32_t x, uint64_t m2, uint64_t c2, uint32_t magic, uint32_t* o) {
-    const uint32_t xe = x & 0x0F0F0F0Fu, xo = (x >> 4) & 0x0F0F0F0Fu;
-    const uint32_t w03 = __byte_perm(xe, xo, 0x5140);        // codes 0, 1, 2, 3
-    const uint32_t w47 = __byte_perm(xe, xo, 0x7362);        // codes 4, 5, 6, 7
-    o[0] = fma2_bf16x2(code_byte_to_float<0>(w03, magic), code_byte_to_float<1>(w03, magic), m2, c2);
-    o[1] = fma2_bf16x2(code_byte_to_float<2>(w03, magic), code_byte_to_float<3>(w03, magic), m2, c2);
-    o[2] = fma2_bf16x2(code_byte_to_float<0>(w47, magic), code_byte_to_float<1>(w47, magic), m2, c2);
-    o[3] = fma2_bf16x2(code_byte_to_float<2>(w47, magic), code_byte_to_float<3>(w47, magic), m2, c2);
 }
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
@@ -882,6 +833,24 @@ int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, cons
     p.n_wt = (N + qg::BW - 1) / qg::BW;
     p.offsets = nullptr; p.out = Cout; p.topk_w = nullptr; p.row_pair = nullptr;
     const int bt = qg::pick_token_tile(ctx, M, p.n_wt, K);
+    return qg::dispatch_gemm(ctx, qbits, bt, p, A, M, Wq, Wscale, static_cast<cudaStream_t>(stream));
+}
+
+int qgemm_dense_gate_up_silu(qg_ctx* ctx, int qbits, int M, int F, int K, const void* A, const void* Wq,
+                             const void* Wscale, void* Out, void* stream) {
+    if (!ctx) return QG_ERR_NULL;
+    if (qbits != QG_Q8 && qbits != QG_Q4) return QG_ERR_SHAPE;
+    if (M < 0 || F < 64 || F % 64 || K < 256 || K % 256) return QG_ERR_SHAPE;
+    if (M == 0) return QG_OK;
+    if (!A || !Wq || !Wscale || !Out) return QG_ERR_NULL;
+    if (!qg::aligned16(A) || !qg::aligned16(Wq) || !qg::aligned16(Wscale) || !qg::aligned16(Out)) return QG_ERR_ALIGN;
+    if (const int rc = qg::check_device(ctx)) return rc;
+    qg::GemmParams p{};      // one segment [0, M), the gate/up epilogue of the grouped kernel
+    p.mode = QG_MODE_GATE_UP_SILU; p.R = M; p.N = 2 * F; p.K = K; p.E = 1; p.k = 1;
+    p.n_wt = (2 * F) / 128;
+    p.offsets = nullptr; p.out = Out; p.topk_w = nullptr; p.row_pair = nullptr;
+    // this epilogue always overlaps the next tile (two accumulators), so the 256-token tile is not a candidate
+    const int bt = (M > 128) ? 192 : 128;
     return qg::dispatch_gemm(ctx, qbits, bt, p, A, M, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 

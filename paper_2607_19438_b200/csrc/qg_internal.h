@@ -35,8 +35,10 @@ struct qg_ctx {
     qg::TmapEntry tmaps[qg::TMAP_CACHE];   // tensor maps of recent calls (weights and buffers recur every layer)
     int tmap_count, tmap_next;
     bool pdl;                  // launch kernels with programmatic stream serialization (QG_NO_PDL=1 turns it off)
-    void* d_ws;                // device workspace owned by the context (split-K partial tiles and their flags)
-    size_t ws_bytes;
+    float* gemv_partial;       // K-slice partial sums of qgemm_small_m, [slices][16][N] fp32
+    size_t gemv_partial_bytes;
+    int* gemv_tickets;         // one arrival counter per 64-row tile, zero between launches
+    int gemv_ticket_count;
     long long* stats;          // profiling builds only
 };
 

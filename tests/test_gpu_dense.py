@@ -129,3 +129,14 @@ def test_dense_short_k_many_tiles_per_pair(qbits, M, N, K):
     for r0 in (M - 128, (M // 2) & ~127):
         ref = orc.qgemm_dense(qbits, A[r0:r0 + 128], Wq[:2048], Ws[:2048])
         util.assert_close(util.host_bf16_f64(out[r0:r0 + 128, :2048]), ref, f"rows {r0}..")
+
+
+@pytest.mark.parametrize("qbits,M,F,K", [(8, 300, 256, 512), (4, 1000, 1024, 768), (8, 64, 64, 256), (4, 2048, 2048, 1024)],
+                         ids=["q8-300", "q4-1000", "q8-64", "q4-2048"])
+def test_dense_gate_up_with_fused_silu(qbits, M, F, K):
+    A, Wq, Ws = synth.dense_problem(qbits, M, 2 * F, K, seed=9)
+    g = util.Guarded((M, F), torch.bfloat16)
+    qg.qgemm_dense_gate_up_silu(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws), out=g.t)
+    qg.poll_status()
+    assert g.intact() and not bool(g.untouched_inside().any().item())
+    util.assert_close(util.host_bf16_f64(g.t), orc.silu_mul(orc.qgemm_dense(qbits, A, Wq, Ws)), "dense gate/up + silu")

@@ -1,0 +1,74 @@
+"""GPU parity of qgemm_small_m (1..16 tokens, the weight-streaming kernel) against the fp64 oracle, and agreement
+with qgemm_dense, which multiplies the same once-rounded bf16 weights."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2607_19438_b200 import binding as qg, synth
+from tests import util
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    (8, 1, 2048, 2048), (4, 1, 2048, 2048), (8, 16, 2048, 2048), (4, 16, 3072, 3072),
+    (8, 5, 200, 256),          # N not a multiple of the 64-row tile, a single K slice
+    (4, 3, 136, 768), (8, 7, 2560, 2048), (4, 16, 72, 4096), (8, 2, 2048, 8192), (4, 9, 1536, 2304),
+]
+
+
+@pytest.mark.parametrize("qbits,M,N,K", SHAPES, ids=[f"q{s[0]}-{s[1]}x{s[2]}x{s[3]}" for s in SHAPES])
+def test_small_m_parity_and_guards(qbits, M, N, K):
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=6)
+    g = util.Guarded((M, N), torch.bfloat16)
+    dA, dWq, dWs = util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws)
+    qg.qgemm_small_m(qbits, dA, dWq, dWs, out=g.t)
+    qg.poll_status()
+    assert g.intact() and not bool(g.untouched_inside().any().item())
+    ref = orc.qgemm_dense(qbits, A, Wq, Ws)
+    mx, rmax, fro = util.assert_close(util.host_bf16_f64(g.t), ref, f"small-M q{qbits} {M}x{N}x{K}")
+    assert fro > 1e-4
+    # fixed-order reduction over the K slices: a second run gives the same bits
+    again = qg.qgemm_small_m(qbits, dA, dWq, dWs)
+    qg.poll_status()
+    assert torch.equal(again, g.t)
+
+
+@pytest.mark.parametrize("qbits", [8, 4])
+def test_small_m_integer_exact_is_bit_exact(qbits):
+    M, N, K = 11, 264, 512
+    rng = np.random.default_rng(17)
+    A = synth.f32_to_bf16_bits(rng.integers(-1, 2, (M, K)).astype(np.float32))
+    if qbits == 8:
+        Wq = rng.integers(-3, 4, (N, K)).astype(np.int8)
+        Wq[0, :] = 0; Wq[0, 5] = -128; Wq[1, :] = 0; Wq[1, 511] = 127
+    else:
+        Wq = rng.integers(0, 256, (N, K // 2)).astype(np.uint8)
+        Wq[:, 16:] = 0x88
+    Ws = (2.0 ** rng.integers(-3, 2, (N, K // 32))).astype(np.float16).view(np.uint16)
+    out = qg.qgemm_small_m(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws))
+    qg.poll_status()
+    ref = orc.qgemm_dense(qbits, A, Wq, Ws)
+    assert np.array_equal(ref, ref.astype(np.float32).astype(np.float64))
+    assert np.array_equal(util.host_bf16_bits(out), orc.f64_to_bf16(ref))
+
+
+def test_small_m_extreme_scales_and_argument_checks():
+    qbits, M, N, K = 8, 4, 128, 512
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=2)
+    Ws = Ws.copy(); Wq = Wq.copy()
+    Wq[::3, ::5] = -128
+    s = Ws.view(np.float16)
+    s[0::4, :] = -s[0::4, :]
+    s[1::4, 0] = 0.0
+    Ws[2::4, :] = np.arange(1, K // 32 + 1, dtype=np.uint16)      # subnormal scales
+    out = qg.qgemm_small_m(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws))
+    qg.poll_status()
+    ref = orc.qgemm_dense(qbits, A, Wq, Ws)
+    util.assert_close(util.host_bf16_f64(out), ref, "extreme")
+    assert np.any(util.host_bf16_f64(out)[:, 2::4] != 0.0), "subnormal scales were flushed to zero"
+    A17 = torch.zeros((17, K), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(qg.QGemmError) as e:
+        qg.qgemm_small_m(qbits, A17, util.dev(Wq), util.dev_f16(Ws))
+    assert e.value.code == -2
+    assert qg.qgemm_small_m(qbits, A17[:0], util.dev(Wq), util.dev_f16(Ws)).shape == (0, N)
