@@ -14,7 +14,7 @@
  *     (a cudaStream_t passed as void*; NULL = the legacy default stream);
  *   - the context's device must be the calling thread's current device (else QG_ERR_DEVICE); a
  *     context and its calls belong to one host thread and one stream at a time (it caches tensor
- *     maps and owns the K-slice scratch of qgemm_small_m);
+ *     maps and owns the partial-sum scratch of qgemm_small_m and qgemm_dense);
  *   - return value: QG_OK (0) or a negative QG_ERR_* code; an error is detected before anything is
  *     launched, so the outputs are untouched; nothing aborts, traps or throws;
  *   - there is no fallback path: a shape the kernels do not accept is an error (the paper's
@@ -70,7 +70,7 @@ enum {
 enum { QG_D_BF16 = 0, QG_D_F32_ACC = 1 };
 
 /* Create / destroy a context for `device`.  Only these two allocate device memory (the status word and the
- * scratch of qgemm_small_m, 32 MB); qg_create leaves the caller's current device as it was. */
+ * scratch of qgemm_small_m and of stream-K qgemm_dense calls, about 52 MB); qg_create leaves the caller's current device as it was. */
 int qg_create(qg_ctx** out, int device);
 int qg_destroy(qg_ctx* ctx);
 const char* qg_strerror(int code);
@@ -78,6 +78,18 @@ const char* qg_strerror(int code);
 int qg_poll_status(qg_ctx* ctx, void* stream);
 /* Bytes of scratch moe_route needs for M tokens, E experts, top-k (per-block expert histograms). */
 size_t qg_route_workspace_bytes(int M, int E, int k);
+
+/*
+ * Launch configuration of qgemm_dense (host only, nothing is launched): the token tile (128, 192 or 256) and whether
+ * the call runs as stream-K, i.e. with the k-blocks of all output tiles dealt out evenly over the SM pairs and the
+ * tiles that are cut in the middle summed through the context's scratch in a fixed order.  The library chooses
+ * both per call from (M, N, K) with a cost model; qg_set_schedule overrides the choice for sweeps and tests:
+ * token_tile 0 = model, else 128 / 192 / 256 (also applies to the grouped calls); streamk_mode -1 = model, 0 = never,
+ * 1 = whenever the tile count is not a multiple of the SM-pair count.  The environment variables QG_FORCE_BT and
+ * QG_STREAMK set the same two values when the context is created.
+ */
+int qg_plan_dense(qg_ctx* ctx, int M, int N, int K, int* token_tile, int* streamk);
+int qg_set_schedule(qg_ctx* ctx, int token_tile, int streamk_mode);
 
 /*
  * Testing hook (no counterpart in the paper): the GEMM kernels' device-side waits give up after

@@ -18,7 +18,7 @@ QG_Q8, QG_Q4 = 8, 4
 MODE_PLAIN, MODE_GATE_UP_SILU, MODE_DOWN_WEIGHTED, MODE_DOWN_ACCUM_F32 = 0, 1, 2, 3
 D_BF16, D_F32_ACC = 0, 1
 
-EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_route_workspace_bytes",
+EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_plan_dense", "qg_set_schedule", "qg_route_workspace_bytes",
            "qgemm_dense", "qgemm_small_m", "qgemm_dense_gate_up_silu",
            "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_grouped_qgemm_gather", "moe_combine"]
 
@@ -48,6 +48,8 @@ def load():
         lib.qg_destroy.argtypes = [C.c_void_p]
         lib.qg_poll_status.argtypes = [C.c_void_p, C.c_void_p]
         lib.qg_test_inject.argtypes = [C.c_void_p, C.c_uint, C.c_int]
+        lib.qg_plan_dense.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        lib.qg_set_schedule.argtypes = [C.c_void_p, C.c_int, C.c_int]
         vp, ci = C.c_void_p, C.c_int
         lib.qgemm_dense.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
         lib.qgemm_small_m.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
@@ -109,6 +111,18 @@ def test_inject(wait_limit_polls: int = 0, skip_kblock: int = -1):
     """Testing hook: bounded-wait limit in polls (0 = default) and the k-block whose activation load the next GEMM
     launch leaves out (-1 = none)."""
     _check(load().qg_test_inject(context(), wait_limit_polls, skip_kblock), "qg_test_inject")
+
+
+def plan_dense(M, N, K):
+    """(token tile, stream-K flag) qgemm_dense would use for this shape."""
+    bt, sk = C.c_int(0), C.c_int(0)
+    _check(load().qg_plan_dense(context(), M, N, K, C.byref(bt), C.byref(sk)), "qg_plan_dense")
+    return bt.value, bool(sk.value)
+
+
+def set_schedule(token_tile: int = 0, streamk_mode: int = -1):
+    """Overrides the launch configuration (0 / -1 = the library's cost model); for sweeps and tests."""
+    _check(load().qg_set_schedule(context(), token_tile, streamk_mode), "qg_set_schedule")
 
 
 def route_workspace_bytes(M, E, k) -> int:

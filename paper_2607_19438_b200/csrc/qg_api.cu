@@ -56,14 +56,20 @@ int qg_create(qg_ctx** out, int device) {
         return QG_ERR_CUDA;
     }
     ctx->encode_tiled = reinterpret_cast<decltype(ctx->encode_tiled)>(fn);
+    ctx->streamk_mode = -1;
+    if (const char* f = getenv("QG_STREAMK")) ctx->streamk_mode = (f[0] == '0') ? 0 : (f[0] == '1') ? 1 : -1;
     ctx->gemv_partial_bytes = static_cast<size_t>(32) << 20;
     ctx->gemv_ticket_count = 4096;
     if (cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess ||
+        cudaMalloc(&ctx->sk_partial, static_cast<size_t>(ctx->sm_count) * 256 * 128 * sizeof(float)) != cudaSuccess ||
+        cudaMalloc(&ctx->sk_flags, sizeof(int) * 2 * ctx->sm_count) != cudaSuccess ||
+        cudaMemset(ctx->sk_flags, 0, sizeof(int) * 2 * ctx->sm_count) != cudaSuccess ||
         cudaMalloc(&ctx->gemv_partial, ctx->gemv_partial_bytes) != cudaSuccess ||
         cudaMalloc(&ctx->gemv_tickets, sizeof(int) * ctx->gemv_ticket_count) != cudaSuccess ||
         cudaMemset(ctx->gemv_tickets, 0, sizeof(int) * ctx->gemv_ticket_count) != cudaSuccess) {
         cudaGetLastError();
         cudaFree(ctx->d_status); cudaFree(ctx->gemv_partial); cudaFree(ctx->gemv_tickets);
+        cudaFree(ctx->sk_partial); cudaFree(ctx->sk_flags);
         delete ctx;
         return QG_ERR_CUDA;
     }
@@ -76,6 +82,8 @@ int qg_destroy(qg_ctx* ctx) {
     cudaFree(ctx->d_status);
     cudaFree(ctx->gemv_partial);
     cudaFree(ctx->gemv_tickets);
+    cudaFree(ctx->sk_partial);
+    cudaFree(ctx->sk_flags);
     delete ctx;
     return QG_OK;
 }
@@ -86,8 +94,23 @@ int qg_poll_status(qg_ctx* ctx, void* stream) {
     int host = 0;
     if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return QG_ERR_CUDA; }
     if (cudaMemcpy(&host, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return QG_ERR_CUDA; }
-    if (host != 0) cudaMemset(ctx->d_status, 0, sizeof(int));
+    if (host != 0) {
+        // a kernel gave up: clear the status word and the cross-CTA counters it may have left half-way, so that the
+        // next launch starts clean
+        cudaMemset(ctx->d_status, 0, sizeof(int));
+        cudaMemset(ctx->sk_flags, 0, sizeof(int) * 2 * ctx->sm_count);
+        cudaMemset(ctx->gemv_tickets, 0, sizeof(int) * ctx->gemv_ticket_count);
+    }
     return host;
+}
+
+int qg_set_schedule(qg_ctx* ctx, int token_tile, int streamk_mode) {
+    if (!ctx) return QG_ERR_NULL;
+    if (token_tile != 0 && token_tile != 128 && token_tile != 192 && token_tile != 256) return QG_ERR_SHAPE;
+    if (streamk_mode < -1 || streamk_mode > 1) return QG_ERR_SHAPE;
+    ctx->force_bt = token_tile;
+    ctx->streamk_mode = streamk_mode;
+    return QG_OK;
 }
 
 int qg_test_inject(qg_ctx* ctx, unsigned wait_limit_polls, int skip_kblock) {

@@ -45,6 +45,10 @@ struct GemmParams {
     void* out;
     const float* topk_w;
     const int32_t* row_pair;
+    int streamk;                // dense plain calls only: the k-blocks of all tiles are dealt out evenly over the CTA
+                                // pairs; tiles cut in the middle are summed through sk_partial
+    float* sk_partial;          // [CTAs][BT * 128] fp32: the partial accumulator of each CTA's unfinished first tile
+    int* sk_flags;              // [CTAs][2]: 16-token blocks of the partial written / consumed; zero between launches
     int* status;
     uint32_t wait_limit;        // polls per bounded wait (an unsatisfied poll lasts about 4 us)
     int skip_kb;                // test hook: k-block of the first tile whose activation load is left out (-1: none)
@@ -95,6 +99,14 @@ struct Cfg {
 
 struct __align__(16) Tile {
     int e, pw, tok0, tok_end;   // expert, pair weight tile (weight tiles 2 pw and 2 pw + 1), token range
+};
+
+// The part of a tile one CTA pair computes: k-blocks [kb0, kb1), the first of which has ring index i0 in this pair's
+// sequence.  nsrc: 0 the whole tile; -1 a part that does not start at k = 0 (its fp32 partial goes to this CTA's slot
+// of sk_partial); n > 0 the part that starts at k = 0 but stops early: the n following pairs hold the rest, their
+// partials are added in pair order before the tile is rounded and stored.
+struct __align__(16) Piece {
+    int kb0, kb1, i0, nsrc;
 };
 
 __device__ __forceinline__ Tile decode_tile(int t, const int* prefix, const GemmParams& p, int BT) {
@@ -160,13 +172,41 @@ __device__ __forceinline__ float lds_scale(uint32_t addr) {
 // loads are in flight while the current one is stored.  Called by the four epilogue warps and, for a
 // single-accumulator tile, by the sixteen dequantising warps, which would otherwise idle at the tile boundary.
 __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int tok_end, int n_base, uint32_t taddr,
-                                            int n_epi, int pid, int npart, __nv_bfloat16* st, int lane) {
+                                            int n_epi, int pid, int npart, __nv_bfloat16* st, int lane, int nsrc,
+                                            int quarter, int slot_floats, volatile int* abort_flag) {
     // The loop is issue-bound (five warps of a scheduler drain together), so everything that does not depend on the
     // block is computed once: the lane's two shared-memory read addresses, its global pointer and its token limit.
     const int nblk = n_epi >> 4;
     int b = pid;
     if (b >= nblk) return;
     const bool weighted = (p.mode == QG_MODE_DOWN_WEIGHTED);
+    // Stream-K parts of a tile.  A part that does not start at k = 0 leaves its raw fp32 fragments in this CTA's slot
+    // (register r of 16-token block b and lane quarter q at ((b 4 + q) 16 + r) 32 + lane: 128-byte rows) and counts its
+    // blocks in the slot's first flag.  The part that starts at k = 0 waits until every block of each of the nsrc
+    // following pairs' slots is there, adds them in pair order and goes on as for a whole tile; the second flag
+    // counts what has been read, and whoever reads last clears both for the next launch.
+    const int mine = (nblk - pid + npart - 1) / npart;          // blocks this warp drains
+    const int slot = static_cast<int>(blockIdx.x);
+    if (nsrc > 0) {
+        for (int c = 1; c <= nsrc; ++c) {
+            const int* f = p.sk_flags + 2 * (slot + 2 * c);
+            bool there = false;
+            for (uint32_t it = 0; it < p.wait_limit * 16u && !there; ++it) {
+                int v;
+                asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
+                there = (v >= nblk * 4);
+                if (!there) {
+                    if ((it & 1023u) == 1023u && *abort_flag) break;
+                    __nanosleep(200);
+                }
+            }
+            if (!there) {        // give up: the launch reports a timeout, the host clears the flags
+                *abort_flag = 1;
+                atomicCAS(p.status, 0, QG_ERR_TIMEOUT);
+                return;
+            }
+        }
+    }
     uint32_t v0[8], v1[8];                       // TMEM lanes 0-15 / 16-31 of this warp's quarter
     tmem_ld_16x256_x2(taddr + 16 * b, v0);
     tmem_ld_16x256_x2(taddr + (16u << 16) + 16 * b, v1);
@@ -194,6 +234,32 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
     const int left_step = 16 * npart;
     while (b < nblk) {
         tmem_ld_wait();
+        if (nsrc != 0) {
+            const size_t at = (static_cast<size_t>(b * 4 + quarter) * 16) * 32 + lane;
+            if (nsrc < 0) {
+                float* dst = p.sk_partial + static_cast<size_t>(slot) * slot_floats + at;
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    dst[r * 32] = __uint_as_float(v0[r]);
+                    dst[(8 + r) * 32] = __uint_as_float(v1[r]);
+                }
+                const int bn = b + npart;
+                if (bn < nblk) {
+                    tmem_ld_16x256_x2(taddr + 16 * bn, v0);
+                    tmem_ld_16x256_x2(taddr + (16u << 16) + 16 * bn, v1);
+                }
+                b = bn;
+                continue;
+            }
+            for (int c = 1; c <= nsrc; ++c) {
+                const float* src = p.sk_partial + static_cast<size_t>(slot + 2 * c) * slot_floats + at;
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    v0[r] = __float_as_uint(__uint_as_float(v0[r]) + __ldcg(src + r * 32));
+                    v1[r] = __float_as_uint(__uint_as_float(v1[r]) + __ldcg(src + (8 + r) * 32));
+                }
+            }
+        }
         uint32_t pk[8];
         if (weighted) {
             const int j = b >> 1;                // tokens 16 b .. 16 b + 15 live in register j, lanes 16 (b & 1) ..
@@ -234,6 +300,19 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
         g += g_step;
         left -= left_step;
         b = bn;
+    }
+    if (nsrc < 0) {
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) atomicAdd(p.sk_flags + 2 * slot, mine);
+    } else if (nsrc > 0) {
+        __syncwarp();
+        if (lane == 0) {
+            for (int c = 1; c <= nsrc; ++c) {
+                int* f = p.sk_flags + 2 * (slot + 2 * c);
+                if (atomicAdd(f + 1, mine) + mine == nblk * 4) { f[1] = 0; __threadfence(); f[0] = 0; }
+            }
+        }
     }
 }
 
@@ -326,13 +405,54 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     const int nkb = p.K / BK;     // a multiple of 4
     // The pair's j-th tile is tile pair + j n_pairs.  Decoding one costs a binary search and two global loads, far
     // too much for the control warps to repeat at every tile boundary, so the first TAB_N are decoded once, here.
-    const int my_tiles = (total_tiles > pair) ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
     Tile* tab = reinterpret_cast<Tile*>(sgen + C::OFF_TAB);
-    for (int j = threadIdx.x; j < min(my_tiles, C::TAB_N); j += NTHREADS)
-        tab[j] = decode_tile(pair + j * n_pairs, prefix, p, BT);
+    // stream-K (dense only, so the prefix array needs two entries and the piece table takes the rest of its space)
+    Piece* ptab = reinterpret_cast<Piece*>(sgen + C::OFF_PREFIX + 16);
+    const int nk4 = nkb >> 2;
+    int my_tiles;
+    uint32_t own_kb4;            // this pair's k-blocks / 4
+    if (p.streamk) {
+        // Units of four k-blocks, U = tiles * nk4 in all; pair q owns units [U q / P, U (q + 1) / P).  Piece j of this
+        // pair lies in tile t_first + j (the host keeps the number of pieces within the table).
+        const long long U = static_cast<long long>(total_tiles) * nk4;
+        const long long u0 = U * pair / n_pairs, u1 = U * (pair + 1) / n_pairs;
+        const int t_first = static_cast<int>(u0 / nk4);
+        my_tiles = (u1 > u0) ? static_cast<int>((u1 - 1) / nk4) - t_first + 1 : 0;
+        own_kb4 = static_cast<uint32_t>(u1 - u0);
+        for (int j = threadIdx.x; j < my_tiles; j += NTHREADS) {
+            const int t = t_first + j;
+            const long long tb = static_cast<long long>(t) * nk4;
+            const long long a = (u0 > tb) ? u0 : tb, b = (u1 < tb + nk4) ? u1 : tb + nk4;
+            Piece pc;
+            pc.kb0 = static_cast<int>(a - tb) * 4;
+            pc.kb1 = static_cast<int>(b - tb) * 4;
+            pc.i0 = static_cast<int>(a - u0) * 4;
+            pc.nsrc = 0;
+            if (pc.kb0 > 0) {
+                pc.nsrc = -1;
+            } else if (pc.kb1 < nkb) {
+                int q = pair + 1;                                   // owner of the tile's last unit
+                while (q + 1 < n_pairs && U * (q + 1) / n_pairs <= tb + nk4 - 1) ++q;
+                pc.nsrc = q - pair;
+            }
+            ptab[j] = pc;
+            tab[j] = decode_tile(t, prefix, p, BT);
+        }
+    } else {
+        my_tiles = (total_tiles > pair) ? (total_tiles - pair + n_pairs - 1) / n_pairs : 0;
+        own_kb4 = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(nk4);
+        for (int j = threadIdx.x; j < min(my_tiles, C::TAB_N); j += NTHREADS)
+            tab[j] = decode_tile(pair + j * n_pairs, prefix, p, BT);
+    }
     __syncthreads();
     auto tile_at = [&](int j) -> Tile {
         return (j < C::TAB_N) ? tab[j] : decode_tile(pair + j * n_pairs, prefix, p, BT);
+    };
+    auto piece_at = [&](int j) -> Piece {
+        if (p.streamk) return ptab[j];
+        Piece pc;
+        pc.kb0 = 0; pc.kb1 = nkb; pc.i0 = j * nkb; pc.nsrc = 0;
+        return pc;
     };
     constexpr bool gate_up = (EPI == 1);
 
@@ -348,6 +468,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         QG_DECL();
         for (int jt = 0; jt < my_tiles && ok; ++jt) {
             const Tile tl = tile_at(jt);
+            const Piece pc = piece_at(jt);
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const int row0 = tl.tok0 + static_cast<int>(rank) * (n_mma >> 1);   // B rows split at N / 2
             // Gathered input: lane l fetches rows 4 l .. 4 l + 3 of this CTA's half tile from the token rows the
@@ -361,7 +482,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 if (r + 2 < tl.tok_end) g2 = p.row_pair[r + 2] / p.gather_k;
                 if (r + 3 < tl.tok_end) g3 = p.row_pair[r + 3] / p.gather_k;
             }
-            for (int kb = 0; kb < nkb; kb += 2) {
+            for (int kb = pc.kb0; kb < pc.kb1; kb += 2) {
                 QG_T0();
                 // a stage is free once the MMAs that read it eight k-blocks ago are done (even and odd stages
                 // belong to different MMA warps, so both are checked)
@@ -400,10 +521,11 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         QG_DECL();
         for (int jt = 0; jt < my_tiles && ok; ++jt) {
             const Tile tl = tile_at(jt);
+            const Piece pc = piece_at(jt);
             const int wt = 2 * tl.pw + static_cast<int>(rank);
             const int row_a = tl.e * p.N + wt * (gate_up ? 64 : 128);
             const int row_b = row_a + (gate_up ? (p.N / 2) : 64);
-            for (int kb = 0; kb < nkb; kb += 4) {
+            for (int kb = pc.kb0; kb < pc.kb1; kb += 4) {
                 QG_T0();
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
@@ -436,9 +558,11 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         // ------------------------------------------------ MMA issuers (even CTA of the pair only)
         // One warp needs about 500-560 cycles to issue the four TMEM-operand MMAs, the commit and the wait of a
         // k-block, more than the 256-512 cycles the tensor cores need for it, and two warps issue concurrently at
-        // full speed; so warps 1 and 3 take the even and the odd k-blocks.  MMAs of different threads are ordered
-        // only through completion, so the odd warp starts a tile after the "done" of the tile's first k-block (which
-        // overwrites the accumulator); within a tile the order of the accumulating k-blocks does not matter.
+        // full speed; so warps 1 and 3 take alternate pairs of k-blocks (0, 1 | 2, 3 | 4, 5 ...).  MMAs of different
+        // threads are ordered only through completion, so the second warp starts a tile after the "done" of the
+        // tile's first k-block (which overwrites the accumulator); by then it has usually just finished the last
+        // pair of the previous tile, while the first warp has already issued two k-blocks of the new one.  Within
+        // a tile the order of the accumulating k-blocks does not matter.
         if (rank == 0) {
             const uint32_t w = (warp == 3) ? 1u : 0u;
             bool ok = true;
@@ -448,11 +572,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             uint32_t j = 0;
             for (; static_cast<int>(j) < my_tiles && ok; ++j) {
                 const Tile tl = tile_at(static_cast<int>(j));
+                const Piece pc = piece_at(static_cast<int>(j));
                 const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
                 const uint32_t idesc = umma_idesc_bf16(2 * BW, n_mma);
                 const uint32_t a = (C::NACC == 2) ? (j & 1u) : 0u;
                 const uint32_t aph = (C::NACC == 2) ? ((j >> 1) & 1u) : (j & 1u);
-                const uint32_t i0 = j * static_cast<uint32_t>(nkb);          // first k-block of the tile (ring index)
+                const uint32_t i0 = static_cast<uint32_t>(pc.i0);             // first k-block of the piece (ring index)
                 QG_T0();
                 if (w == 0) {
                     if (!spin_wait_bar(acc_empty(a), aph ^ 1u, abort_flag, p)) { ok = false; break; }
@@ -461,26 +586,30 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 }
                 QG_ACC(2);
                 const uint32_t d_tmem = tmem_base + a * BT;
-                uint32_t i = i0 + w;
-                uint32_t ta = i % C::SA;                                     // TMEM weight stage of k-block i
+                // this warp's k-blocks of the piece: kb0 + 2 w + {0, 1}, then every fourth pair
+                int kb = pc.kb0 + 2 * static_cast<int>(w);
+                uint32_t i = i0 + 2u * w;
                 bool ready = mbar_test_wait_cluster(full(i & 7u), (i >> 3) & 1u);
-                for (int kb = static_cast<int>(w); kb < nkb; kb += 2, i += 2) {
+                while (kb < pc.kb1) {
                     const uint32_t st = i & 7u;
+                    const uint32_t ta = i % C::SA;                               // TMEM weight stage of k-block i
                     QG_T0();
                     if (!ready && !spin_wait_bar(full(st), (i >> 3) & 1u, abort_flag, p)) { ok = false; break; }
                     QG_ACC(3);
                     tc_fence_after_sync();
                     // start the wait for this warp's next k-block before issuing, so its latency is hidden
-                    ready = (kb + 2 < nkb) && mbar_test_wait_cluster(full((i + 2) & 7u), ((i + 2) >> 3) & 1u);
+                    const int step = (kb & 1) ? 3 : 1;
+                    const uint32_t in = i + static_cast<uint32_t>(step);
+                    ready = (kb + step < pc.kb1) && mbar_test_wait_cluster(full(in & 7u), (in >> 3) & 1u);
                     if (lane == 0) {
                         umma_kblock_ts_pair(d_tmem, tmem_base + C::A_COL0 + ta * C::A_COLS,
-                                            b_lo0 + st * (C::X_BYTES >> 4), b_hi, idesc, kb != 0 ? 1u : 0u);
+                                            b_lo0 + st * (C::X_BYTES >> 4), b_hi, idesc, kb != pc.kb0 ? 1u : 0u);
                         umma_commit_pair(done(st));
                     }
                     __syncwarp();
                     QG_ACC(10);
-                    ta += 2;
-                    if (ta >= C::SA) ta -= C::SA;
+                    kb += step;
+                    i = in;
                 }
                 if (ok && lane == 0) umma_commit_pair(acc_full(a));
                 __syncwarp();
@@ -501,13 +630,17 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         const uint32_t raw_row = row * C::RAW_ROW;
         const uint32_t a_taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + C::A_COL0;
         const uint32_t full_leader = map_to_cta(full(0), 0);
-        const uint32_t n_own = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(nkb >> 2);
+        const uint32_t n_own = own_kb4;
         constexpr uint32_t magic = 0x43000000u;
         QG_DECL();
         // Helping with the epilogue.  Before this warp waits for the MMAs of own k-block n - 2 (to reuse their TMEM
         // stage) it must have released every accumulator of an earlier tile, otherwise a single-accumulator pipeline
         // would wait for itself; at that point it has filled the ring for the next tile and would idle anyway.
-        const uint32_t per_tile = static_cast<uint32_t>(nkb >> 2);     // own k-blocks per tile
+        auto per_tile = [&](uint32_t t) -> uint32_t {                  // own k-blocks of the pair's t-th tile (piece)
+            if (!p.streamk) return static_cast<uint32_t>(nk4);
+            const Piece pc = ptab[t];
+            return static_cast<uint32_t>(pc.kb1 - pc.kb0) >> 2;
+        };
         uint32_t helped = 0;                                           // tiles whose accumulator this warp released
         uint32_t t2 = 0, in2 = 0;                                      // tile of own k-block n - 2, position in it
         const uint32_t acc_empty_leader = map_to_cta(acc_empty(0), 0);
@@ -528,7 +661,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             if (plain_ep && wt < p.n_wt) {
                 const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
                 drain_plain(p, tl.tok0, tl.tok_end, wt * BW + q * 32,
-                            tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BT, n_mma, 1 + g, 5, my_st, lane);
+                            tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BT, n_mma, 1 + g, 5, my_st, lane,
+                            piece_at(static_cast<int>(jt)).nsrc, q, BT * 128, abort_flag);
             }
             tc_fence_before_sync();
             __syncwarp();
@@ -545,7 +679,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             if (C::HELP && n >= 2) {
                 while (dq_ok && helped < t2) dq_ok = help_tile(helped++, true);
                 if (!dq_ok) break;
-                if (++in2 == per_tile) { in2 = 0; ++t2; }
+                if (++in2 == per_tile(t2)) { in2 = 0; ++t2; }
             }
             QG_T0();
             // the scales of this group of four k-blocks arrive with the first of them (stage 0 or 4)
@@ -647,7 +781,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 // shared with the dequantising warps (participants 1..4 of this lane quarter) when they help
                 drain_plain(p, tl.tok0, tl.tok_end, wt * BW + qd * 32, taddr, n_epi, 0,
                             (C::HELP || static_cast<int>(j) == my_tiles - 1) ? 5 : 1,
-                            stg16 + (16 + qd) * 512, lane);
+                            stg16 + (16 + qd) * 512, lane, piece_at(static_cast<int>(j)).nsrc, qd, BT * 128, abort_flag);
             } else {
                 for (int c = 0; c < n_epi; c += 32) {
                     uint32_t v[32];
@@ -756,8 +890,9 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_ro
         ctx->attr_set[inst] = true;
     }
     // Upper bound on the number of pair tiles (the exact count lives on the device for grouped calls).
-    const long long max_tiles =
+    long long max_tiles =
         (static_cast<long long>((p.R + BT - 1) / BT) + (p.offsets ? p.E : 0)) * ((p.n_wt + 1) / 2);
+    if (p.streamk) max_tiles *= p.K / (4 * BK);      // units of four k-blocks: every pair gets at least one
     const long long pairs_hw = ctx->sm_count / 2;
     const int grid = 2 * static_cast<int>(max_tiles < pairs_hw ? max_tiles : pairs_hw);
     if (launch_kernel(ctx, kern, dim3(grid), dim3(NTHREADS), C::SMEM_BYTES, st, *tm_x, *tm_w, *tm_s, p) != cudaSuccess) {
@@ -767,21 +902,36 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_ro
     return QG_OK;
 }
 
-// Token tile of a dense call: the candidate with the smallest modelled time.  A wave is one pair tile per SM pair;
-// a tile costs nkb k-blocks of about `period` cycles (measured: issue- and latency-bound, nearly independent of
-// the tile width) plus, for the single-accumulator 256-wide tile, an epilogue that is not overlapped.
-static int pick_token_tile(const qg_ctx* ctx, int M, int n_wt, int K) {
-    if (M <= 128) return 128;
+// Token tile and schedule of a dense call: the candidate with the smallest modelled time.  Data-parallel: a wave is
+// one pair tile per SM pair; a tile costs nkb k-blocks of about `period` cycles (measured: issue- and latency-bound,
+// nearly independent of the tile width) plus, for the single-accumulator 256-wide tile, an epilogue that is not
+// overlapped.  Stream-K: every pair gets the same share of all k-blocks, pays the exposed epilogue once per tile it
+// touches and a fixed amount for writing and reading the partial tiles.
+struct DensePlan {
+    int bt, streamk;
+};
+static DensePlan plan_dense(const qg_ctx* ctx, int M, int n_wt, int K) {
     const int cand[3] = {128, 192, 256};
-    const double period[3] = {625.0, 665.0, 720.0}, epilogue[3] = {0.0, 0.0, 6000.0};
+    const double period[3] = {625.0, 665.0, 720.0}, epilogue[3] = {0.0, 0.0, 6000.0}, last_epi[3] = {2500.0, 3000.0, 0.0};
     const long long pairs = ctx->sm_count / 2, n_pw = (n_wt + 1) / 2;
-    int best = 256;
+    const int nk4 = K / (4 * BK);
+    DensePlan best{256, 0};
     double best_cost = 1e300;
     for (int c = 0; c < 3; ++c) {
+        if (M <= 128 && cand[c] > 128) break;
         const long long tiles = n_pw * ((M + cand[c] - 1) / cand[c]);
         const long long waves = (tiles + pairs - 1) / pairs;
-        const double cost = static_cast<double>(waves) * ((K / BK) * period[c] + epilogue[c]);
-        if (cost < best_cost * 0.999) { best_cost = cost; best = cand[c]; }
+        const double dp = static_cast<double>(waves) * ((K / BK) * period[c] + epilogue[c]) + last_epi[c];
+        if (ctx->streamk_mode != 1 || tiles % pairs == 0)
+            if (dp < best_cost * 0.999) { best_cost = dp; best = DensePlan{cand[c], 0}; }
+        if (ctx->streamk_mode == 0 || tiles % pairs == 0) continue;
+        const long long units = tiles * nk4;
+        const long long P = units < pairs ? units : pairs;
+        const long long share = (units + P - 1) / P;                        // units of the busiest pair
+        const double pieces = static_cast<double>(share) / nk4 + 1.5;       // tiles it touches, on average
+        if (share / nk4 + 2 > 120) continue;                                // the piece table has 128 entries
+        const double sk = share * 4.0 * period[c] + pieces * epilogue[c] + last_epi[c] + 5000.0;
+        if (sk < best_cost * 0.97) { best_cost = sk; best = DensePlan{cand[c], 1}; }
     }
     return best;
 }
@@ -819,6 +969,15 @@ static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in,
 
 extern "C" {
 
+int qg_plan_dense(qg_ctx* ctx, int M, int N, int K, int* token_tile, int* streamk) {
+    if (!ctx) return QG_ERR_NULL;
+    if (M < 1 || N < 8 || N % 8 || K < 256 || K % 256) return QG_ERR_SHAPE;
+    const qg::DensePlan plan = qg::plan_dense(ctx, M, (N + qg::BW - 1) / qg::BW, K);
+    if (token_tile) *token_tile = ctx->force_bt ? ctx->force_bt : plan.bt;
+    if (streamk) *streamk = (ctx->force_bt == 0 || ctx->streamk_mode == 1) ? plan.streamk : 0;
+    return QG_OK;
+}
+
 int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq, const void* Wscale,
                 void* Cout, void* stream) {
     if (!ctx) return QG_ERR_NULL;
@@ -832,8 +991,10 @@ int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, cons
     p.mode = QG_MODE_PLAIN; p.R = M; p.N = N; p.K = K; p.E = 1; p.k = 1;
     p.n_wt = (N + qg::BW - 1) / qg::BW;
     p.offsets = nullptr; p.out = Cout; p.topk_w = nullptr; p.row_pair = nullptr;
-    const int bt = qg::pick_token_tile(ctx, M, p.n_wt, K);
-    return qg::dispatch_gemm(ctx, qbits, bt, p, A, M, Wq, Wscale, static_cast<cudaStream_t>(stream));
+    const qg::DensePlan plan = qg::plan_dense(ctx, M, p.n_wt, K);
+    p.streamk = (ctx->force_bt == 0 || ctx->streamk_mode == 1) ? plan.streamk : 0;
+    p.sk_partial = ctx->sk_partial; p.sk_flags = ctx->sk_flags;
+    return qg::dispatch_gemm(ctx, qbits, plan.bt, p, A, M, Wq, Wscale, static_cast<cudaStream_t>(stream));
 }
 
 int qgemm_dense_gate_up_silu(qg_ctx* ctx, int qbits, int M, int F, int K, const void* A, const void* Wq,

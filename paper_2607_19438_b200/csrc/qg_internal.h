@@ -35,6 +35,9 @@ struct qg_ctx {
     qg::TmapEntry tmaps[qg::TMAP_CACHE];   // tensor maps of recent calls (weights and buffers recur every layer)
     int tmap_count, tmap_next;
     bool pdl;                  // launch kernels with programmatic stream serialization (QG_NO_PDL=1 turns it off)
+    float* sk_partial;         // stream-K: one fp32 partial tile (256 tokens x 128 rows) per CTA
+    int* sk_flags;             // stream-K: two counters per CTA, zero between launches
+    int streamk_mode;          // QG_STREAMK at creation: -1 heuristic (default), 0 never, 1 whenever legal
     float* gemv_partial;       // K-slice partial sums of qgemm_small_m, [slices][16][N] fp32
     size_t gemv_partial_bytes;
     int* gemv_tickets;         // one arrival counter per 64-row tile, zero between launches
