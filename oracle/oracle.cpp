@@ -22,6 +22,9 @@
 //   expert GEMM the dense definition applied per expert segment   (Sec. 3.1 "MoE expert GEMM")
 //   gate/up     H = silu(G) * U with silu(g) = g / (1 + exp(-g))  (Sec. 3.1 "Fused MoE gate/up")
 //   combine     y[t] = sum over slots s (ascending) of w[t][s] * D[row of (t, s)]
+//   attention   O[i, h] = sum_j softmax_j(scale * q[i, h] . k[j, g(h)]) v[j, g(h)], j <= i if causal,
+//               g(h) = h / (Hq / Hkv)                           (Sec. 3.1 "Prefill attention": the
+//               paper only requires the tensor path to equal the plain softmax(Q K^T) V)
 //
 // Pins (tests run without a GPU): hand-computed products, exhaustive code tables, closed forms of
 // silu and softmax, a full stable sort as brute-force routing, an independent fp64 library matmul,
@@ -244,6 +247,45 @@ void orc_combine(int64_t M, int k, int64_t H, const double* D, const int32_t* pa
             }
             y[t * H + c] = acc;
         }
+}
+
+// Scaled-dot-product attention for one sequence, plain definition.  Q [S, Hq, d], K and V [S, Hkv, d] as bf16 bits with
+// row strides ldq / ldk / ldv (elements); rows of a sample of query positions only (qpos, nq entries) so that long
+// sequences can be checked on a subset.  out fp64 [nq, Hq, d].  The softmax subtracts the row maximum (same value in
+// exact arithmetic) so that exp never overflows.
+void orc_attention(int64_t S, int Hq, int Hkv, int d, const uint16_t* Q, int64_t ldq, const uint16_t* K, int64_t ldk,
+                   const uint16_t* V, int64_t ldv, double scale, int causal, int64_t nq, const int64_t* qpos,
+                   double* out) {
+    const int group = Hq / Hkv;
+#pragma omp parallel for schedule(dynamic) collapse(2)
+    for (int64_t qi = 0; qi < nq; ++qi) {
+        for (int h = 0; h < Hq; ++h) {
+            const int64_t i = qpos[qi];
+            const int g = h / group;
+            const int64_t last = causal ? i : S - 1;                 // keys 0 .. last take part
+            std::vector<double> sc(static_cast<size_t>(last + 1));
+            double mx = -INFINITY;
+            for (int64_t j = 0; j <= last; ++j) {
+                double dot = 0.0;
+                for (int c = 0; c < d; ++c)
+                    dot += bf16_to_f64(Q[i * ldq + static_cast<int64_t>(h) * d + c]) *
+                           bf16_to_f64(K[j * ldk + static_cast<int64_t>(g) * d + c]);
+                sc[j] = dot * scale;
+                if (sc[j] > mx) mx = sc[j];
+            }
+            double den = 0.0;
+            for (int64_t j = 0; j <= last; ++j) {
+                sc[j] = std::exp(sc[j] - mx);
+                den += sc[j];
+            }
+            double* o = out + (qi * Hq + h) * static_cast<int64_t>(d);
+            for (int c = 0; c < d; ++c) o[c] = 0.0;
+            for (int64_t j = 0; j <= last; ++j) {
+                const double pj = sc[j] / den;
+                for (int c = 0; c < d; ++c) o[c] += pj * bf16_to_f64(V[j * ldv + static_cast<int64_t>(g) * d + c]);
+            }
+        }
+    }
 }
 
 int orc_num_threads(void) {

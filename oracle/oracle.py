@@ -181,3 +181,21 @@ def moe_layer(qbits, logits, X, W1q, W1s, W2q, W2s, k):
     y = combine(Dn, pair_row, k, w)
     return dict(idx=idx, w=w, w32=w32, counts=counts, offsets=offsets, row_pair=row_pair, pair_row=pair_row,
                 Xp=Xp, GU=GU, Hh=Hh, Dn=Dn, y=y)
+
+
+def attention(Q, K, V, Hq, Hkv, d, causal=True, scale=None, qpos=None):
+    """Q bf16 bits [S, Hq*d], K / V bf16 bits [S, Hkv*d] (any row stride: pass 2-D views of a wider array) -> fp64
+    [nq, Hq*d] for the query positions qpos (all if None).  softmax(scale * Q K^T) V per head, keys j <= i if causal,
+    query head h uses key/value head h // (Hq // Hkv); scale defaults to 1 / sqrt(d)."""
+    Q, K, V = (np.asarray(x) for x in (Q, K, V))
+    assert Q.dtype == np.uint16 and K.dtype == np.uint16 and V.dtype == np.uint16
+    S = Q.shape[0]
+    for x in (Q, K, V):
+        assert x.strides[1] == 2, "rows must be contiguous"
+    qpos = np.arange(S, dtype=np.int64) if qpos is None else _c(qpos, np.int64)
+    out = np.empty((qpos.size, Hq * d), np.float64)
+    scale = 1.0 / np.sqrt(d) if scale is None else float(scale)
+    lib().orc_attention(C.c_int64(S), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), _p(Q), C.c_int64(Q.strides[0] // 2), _p(K),
+                        C.c_int64(K.strides[0] // 2), _p(V), C.c_int64(V.strides[0] // 2), C.c_double(scale),
+                        C.c_int(1 if causal else 0), C.c_int64(qpos.size), _p(qpos), _p(out))
+    return out

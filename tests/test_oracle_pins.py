@@ -290,3 +290,67 @@ def test_one_hot_logits_select_one_expert():
     Hh = orc.silu_mul(GU)
     y = Hh @ _np_dequant(4, W2q[e], W2s[e]).T
     assert np.allclose(r["y"][t], y[0], rtol=1e-12, atol=1e-16)
+
+
+# ---------------------------------------------------------------------------------------------- attention
+def _bf16(x):
+    return synth.f32_to_bf16_bits(np.asarray(x, np.float32))
+
+
+def test_attention_closed_forms():
+    """Pins that need no other implementation.  Zero queries give uniform weights, so a causal row i is the mean of
+    V[0..i] and a full row the mean of all V; a query aligned with exactly one key by a huge margin returns that
+    key's value; row 0 of a causal problem is V[0]."""
+    S, Hq, Hkv, d = 7, 2, 1, 8
+    rng = np.random.default_rng(0)
+    V = _bf16(rng.standard_normal((S, Hkv * d)))
+    K = _bf16(rng.standard_normal((S, Hkv * d)))
+    Q0 = _bf16(np.zeros((S, Hq * d)))
+    Vf = orc.bf16_to_f64(V)
+    out = orc.attention(Q0, K, V, Hq, Hkv, d, causal=True)
+    for i in range(S):
+        want = Vf[:i + 1].mean(axis=0)
+        assert np.allclose(out[i, :d], want, atol=1e-12) and np.allclose(out[i, d:], want, atol=1e-12)
+    full = orc.attention(Q0, K, V, Hq, Hkv, d, causal=False)
+    assert np.allclose(full, np.tile(Vf.mean(axis=0), (S, Hq)), atol=1e-12)
+    # one-hot keys, query = 64 * e_j: score gap of 64 * scale * 1 = 22.6, weights of the others below 2e-10
+    Ke = _bf16(np.eye(S, d)); Qe = _bf16(np.tile(64.0 * np.eye(S, d)[::-1], (1, Hq)))   # query i looks for key S-1-i
+    pick = orc.attention(Qe, Ke, V, Hq, Hkv, d, causal=False)
+    assert np.allclose(pick[:, :d], Vf[::-1], atol=1e-8)
+    assert np.array_equal(orc.attention(Qe, Ke, V, Hq, Hkv, d, causal=True)[0, :d], Vf[0])
+
+
+def test_attention_hand_case():
+    """S = 2, d = 2, one head, scale 1: scores [[q0.k0], [q1.k0, q1.k1]] = [[1], [0, ln 3]] -> weights [1], [1/4, 3/4];
+    values v0 = (4, 0), v1 = (0, 8)  ->  O = [(4, 0), (1, 6)]."""
+    ln3 = np.log(3.0)
+    Q = np.array([[1.0, 0.0], [0.0, 1.0]], np.float32)
+    K = np.array([[1.0, 0.0], [0.0, ln3]], np.float32)
+    V = np.array([[4.0, 0.0], [0.0, 8.0]], np.float32)
+    out = orc.attention(_bf16(Q), _bf16(K), _bf16(V), 1, 1, 2, causal=True, scale=1.0)
+    k11 = float(orc.bf16_to_f64(_bf16(K))[1, 1])                 # ln 3 rounded to bf16
+    w1 = np.exp(k11) / (1.0 + np.exp(k11))
+    assert np.allclose(out[0], [4.0, 0.0], atol=1e-15)
+    assert np.allclose(out[1], [4.0 * (1 - w1), 8.0 * w1], atol=1e-13)
+    assert abs(out[1, 1] - 6.0) < 0.02                            # 3/4 * 8 up to the rounding of ln 3
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_attention_against_library_softmax_and_matmul(causal):
+    """torch fp64 matmul + softmax as an independent routine, grouped-query heads expanded explicitly, inputs taken as
+    strided views of one wide [S, (Hq + 2 Hkv) d] buffer (the layout a fused QKV projection leaves behind)."""
+    S, Hq, Hkv, d = 37, 6, 2, 16
+    rng = np.random.default_rng(1)
+    qkv = _bf16(rng.standard_normal((S, (Hq + 2 * Hkv) * d)))
+    Q, K, V = qkv[:, :Hq * d], qkv[:, Hq * d:(Hq + Hkv) * d], qkv[:, (Hq + Hkv) * d:]
+    out = orc.attention(Q, K, V, Hq, Hkv, d, causal=causal)
+    f = lambda x, h: torch.from_numpy(orc.bf16_to_f64(np.ascontiguousarray(x))).view(S, h, d).permute(1, 0, 2)
+    q, k, v = f(Q, Hq), f(K, Hkv).repeat_interleave(Hq // Hkv, 0), f(V, Hkv).repeat_interleave(Hq // Hkv, 0)
+    sc = q @ k.transpose(1, 2) / np.sqrt(d)
+    if causal:
+        sc = sc.masked_fill(torch.triu(torch.ones(S, S, dtype=torch.bool), 1), float("-inf"))
+    want = (torch.softmax(sc, -1) @ v).permute(1, 0, 2).reshape(S, Hq * d).numpy()
+    assert np.allclose(out, want, atol=1e-12)
+    # a sample of query rows equals the same rows of the full result
+    qpos = np.array([0, 5, S - 1])
+    assert np.array_equal(orc.attention(Q, K, V, Hq, Hkv, d, causal=causal, qpos=qpos), out[qpos])
