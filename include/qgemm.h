@@ -88,7 +88,7 @@ size_t qg_route_workspace_bytes(int M, int E, int k);
  * 1 = whenever the tile count is not a multiple of the SM-pair count.  The environment variables QG_FORCE_BT and
  * QG_STREAMK set the same two values when the context is created.
  */
-int qg_plan_dense(qg_ctx* ctx, int M, int N, int K, int* token_tile, int* streamk);
+int qg_plan_dense(qg_ctx* ctx, int qbits, int M, int N, int K, int* token_tile, int* streamk);
 int qg_set_schedule(qg_ctx* ctx, int token_tile, int streamk_mode);
 
 /*
@@ -127,6 +127,21 @@ int qgemm_dense_gate_up_silu(qg_ctx* ctx, int qbits, int M, int F, int K, const 
  */
 int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq,
                   const void* Wscale, void* C, void* stream);
+
+/*
+ * Prefill attention (Sec. 3.1: the attention operator of prompt processing with both matrix products on the tensor
+ * units and the softmax kept exact, so that it equals the plain definition):
+ *   O[i, h, :] = sum_j softmax_j(scale * Q[i, h, :] . K[j, g, :]) * V[j, g, :],   g = h / (Hq / Hkv),
+ *   over keys j <= i if `causal` is non-zero, else over all S keys; one sequence of S positions.
+ *   Q bf16 [S, Hq*d] with row stride ldq (elements), K and V bf16 [S, Hkv*d] with row strides ldk, ldv, O bf16
+ *   [S, Hq*d] with row stride ldo: the three inputs may be column blocks of one [S, (Hq + 2 Hkv) d] buffer, i.e. the
+ *   output of a fused QKV projection, without any copy.  d = 64 or 128; Hq % Hkv == 0; strides multiples of 8 elements;
+ *   scale = 0 means 1 / sqrt(d).  fp32 softmax statistics and accumulation, probabilities rounded to bf16 before the
+ *   second product, one rounding of O to bf16.
+ */
+int prefill_attention(qg_ctx* ctx, int S, int Hq, int Hkv, int d, const void* Q, long long ldq, const void* K,
+                      long long ldk, const void* V, long long ldv, void* O, long long ldo, int causal, float scale,
+                      void* stream);
 
 /*
  * Routing (Sec. 3.1 only presupposes that tokens have been assigned to experts; defined here): for every token the k

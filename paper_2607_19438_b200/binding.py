@@ -19,7 +19,7 @@ MODE_PLAIN, MODE_GATE_UP_SILU, MODE_DOWN_WEIGHTED, MODE_DOWN_ACCUM_F32 = 0, 1, 2
 D_BF16, D_F32_ACC = 0, 1
 
 EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_plan_dense", "qg_set_schedule", "qg_route_workspace_bytes",
-           "qgemm_dense", "qgemm_small_m", "qgemm_dense_gate_up_silu",
+           "qgemm_dense", "qgemm_small_m", "qgemm_dense_gate_up_silu", "prefill_attention",
            "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_grouped_qgemm_gather", "moe_combine"]
 
 
@@ -48,12 +48,14 @@ def load():
         lib.qg_destroy.argtypes = [C.c_void_p]
         lib.qg_poll_status.argtypes = [C.c_void_p, C.c_void_p]
         lib.qg_test_inject.argtypes = [C.c_void_p, C.c_uint, C.c_int]
-        lib.qg_plan_dense.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        lib.qg_plan_dense.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         lib.qg_set_schedule.argtypes = [C.c_void_p, C.c_int, C.c_int]
         vp, ci = C.c_void_p, C.c_int
         lib.qgemm_dense.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
         lib.qgemm_small_m.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
         lib.qgemm_dense_gate_up_silu.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
+        ll = C.c_longlong
+        lib.prefill_attention.argtypes = [vp, ci, ci, ci, ci, vp, ll, vp, ll, vp, ll, vp, ll, ci, C.c_float, vp]
         lib.moe_route.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp, C.c_size_t, vp]
         lib.moe_route_static.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         lib.moe_permute.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
@@ -113,10 +115,10 @@ def test_inject(wait_limit_polls: int = 0, skip_kblock: int = -1):
     _check(load().qg_test_inject(context(), wait_limit_polls, skip_kblock), "qg_test_inject")
 
 
-def plan_dense(M, N, K):
+def plan_dense(qbits, M, N, K):
     """(token tile, stream-K flag) qgemm_dense would use for this shape."""
     bt, sk = C.c_int(0), C.c_int(0)
-    _check(load().qg_plan_dense(context(), M, N, K, C.byref(bt), C.byref(sk)), "qg_plan_dense")
+    _check(load().qg_plan_dense(context(), qbits, M, N, K, C.byref(bt), C.byref(sk)), "qg_plan_dense")
     return bt.value, bool(sk.value)
 
 
@@ -159,6 +161,20 @@ def qgemm_dense_gate_up_silu(qbits, A, Wq, Wscale, out=None):
         out = torch.empty((M, F), dtype=torch.bfloat16, device=A.device)
     _check(load().qgemm_dense_gate_up_silu(context(), qbits, M, F, K, _ptr(A), _ptr(Wq), _ptr(Wscale), _ptr(out),
                                            _stream()), "qgemm_dense_gate_up_silu")
+    return out
+
+
+def prefill_attention(Q, K, V, Hq, Hkv, d, causal=True, scale=0.0, out=None):
+    """Q bf16 [S, Hq*d], K / V bf16 [S, Hkv*d] (2-D views with unit column stride and any row stride, e.g. column blocks
+    of a fused QKV projection's output) -> O bf16 [S, Hq*d]."""
+    S = Q.shape[0]
+    for t in (Q, K, V):
+        assert t.dim() == 2 and t.stride(1) == 1 and t.dtype == torch.bfloat16
+    if out is None:
+        out = torch.empty((S, Hq * d), dtype=torch.bfloat16, device=Q.device)
+    _check(load().prefill_attention(context(), S, Hq, Hkv, d, _ptr(Q), Q.stride(0), _ptr(K), K.stride(0), _ptr(V),
+                                    V.stride(0), _ptr(out), out.stride(0), 1 if causal else 0, float(scale), _stream()),
+           "prefill_attention")
     return out
 
 

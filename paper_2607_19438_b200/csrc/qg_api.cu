@@ -130,10 +130,13 @@ int check_device(const qg_ctx* ctx) {
 }
 
 int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
-                uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz) {
+                uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz,
+                uint64_t row_stride_bytes) {
+    if (row_stride_bytes == 0) row_stride_bytes = inner * static_cast<uint64_t>(elem_bytes);
     for (int i = 0; i < ctx->tmap_count; ++i) {
         const TmapEntry& e = ctx->tmaps[i];
         if (e.base == base && e.inner == inner && e.rows == rows && e.box_inner == box_inner && e.box_rows == box_rows &&
+            e.row_stride == row_stride_bytes &&
             e.dt == static_cast<int>(dt) && e.elem_bytes == elem_bytes && e.swz == static_cast<int>(swz)) {
             *out = &e.map;
             return QG_OK;
@@ -141,7 +144,7 @@ int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, in
     }
     TmapEntry& e = ctx->tmaps[ctx->tmap_next];
     cuuint64_t dims[2] = {inner, rows};
-    cuuint64_t strides[1] = {inner * static_cast<uint64_t>(elem_bytes)};
+    cuuint64_t strides[1] = {row_stride_bytes};
     cuuint32_t box[2] = {box_inner, box_rows};
     cuuint32_t estr[2] = {1, 1};
     e.base = nullptr;      // not a valid entry while it is being rewritten
@@ -149,7 +152,7 @@ int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, in
                                    CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return QG_ERR_CUDA;
-    e.base = base; e.inner = inner; e.rows = rows; e.box_inner = box_inner; e.box_rows = box_rows;
+    e.base = base; e.inner = inner; e.rows = rows; e.row_stride = row_stride_bytes; e.box_inner = box_inner; e.box_rows = box_rows;
     e.dt = static_cast<int>(dt); e.elem_bytes = elem_bytes; e.swz = static_cast<int>(swz);
     *out = &e.map;
     ctx->tmap_next = (ctx->tmap_next + 1) % TMAP_CACHE;

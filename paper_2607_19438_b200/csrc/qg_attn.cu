@@ -1,0 +1,410 @@
+// Prefill attention for sm_100a: softmax(scale * Q K^T) V per head, causal or full, grouped-query heads.
+//
+// Operation (paper Sec. 3.1, the prefill attention operator: both matrix products on the tensor units with an exact
+// softmax between them, equal to the plain definition):
+//   O[i, h, :] = sum_j p[i, j] V[j, g, :],  p[i, :] = softmax_j(scale * Q[i, h, :] . K[j, g, :]),  g = h / (Hq / Hkv),
+//   keys j <= i only when causal.
+//
+// One CTA per (query tile of 128 rows, head).  S = Q K^T (128 x 128 per key tile) is a tcgen05.mma with both operands
+// in shared memory (K-major, 128-byte swizzle, staged by TMA straight from the caller's strided Q / K / V, e.g. the
+// output of a fused QKV projection) and its fp32 result in tensor memory; four softmax warps (one thread per query
+// row) read it, keep the running row maximum and sum, and write P = exp2(...) as bf16 over the same tensor-memory
+// columns; O += P V is a tcgen05.mma whose A operand is P in tensor memory and whose B operand is the V tile in shared
+// memory read N-major (V's head dimension is contiguous), accumulated in a third tensor-memory region.  Two S / P
+// buffers let the next tile's Q K^T run while the softmax warps work; when a row maximum grows, the same warps
+// rescale O in tensor memory before the next P V is issued.
+//   warp 0      TMA producer: Q once, then K and V tiles through two-stage rings
+//   warp 1      MMA issuer, allocates and frees tensor memory
+//   warps 2-5   softmax, O rescaling, final normalisation and store
+// Every mbarrier wait is bounded; when one expires the CTA records QG_ERR_TIMEOUT and leaves.
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "qg_internal.h"
+#include "qg_ptx.cuh"
+
+namespace qg {
+
+constexpr int AT_BQ = 128, AT_BKV = 128, AT_THREADS = 192;
+
+struct AttnParams {
+    int S, Hq, Hkv, causal;
+    float scale_log2;           // softmax scale times log2(e)
+    __nv_bfloat16* O;
+    long long ldo;              // elements
+    int* status;
+    uint32_t wait_limit;
+};
+
+template <int D>
+struct AttnCfg {
+    static constexpr int BOX_BYTES = 128 * 128;                 // one [128 rows x 64 columns] bf16 box
+    static constexpr int NBOX = D / 64;
+    static constexpr int TILE_BYTES = NBOX * BOX_BYTES;
+    static constexpr int NST = 2;
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = OFF_Q + TILE_BYTES;
+    static constexpr int OFF_V = OFF_K + NST * TILE_BYTES;
+    static constexpr int OFF_BAR = OFF_V + NST * TILE_BYTES;
+    static constexpr int NBAR = 16;
+    static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
+    static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;
+    static constexpr int COL_S = 0;                             // two S / P buffers of 128 columns
+    static constexpr int COL_O = 256;                           // O accumulator, D columns
+    static constexpr int TMEM_COLS = 512;
+    static constexpr int OUT_PITCH = D * 2 + 16;                // bytes per staged output row
+    static_assert(D == 64 || D == 128, "head dimension");
+    static_assert(COL_O + D <= TMEM_COLS, "tensor memory budget");
+    static_assert(128 * OUT_PITCH <= NST * TILE_BYTES, "output staging reuses the K ring");
+};
+
+// Shared-memory operand descriptor for an N-major (or M-major) bf16 tile: 64 consecutive N elements are contiguous
+// (128 bytes, 128-byte swizzle), consecutive k are 128 bytes apart in groups of eight (1024 bytes), the next 64 N
+// elements start lbo_bytes further on.
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFF) >> 4);
+    d |= static_cast<uint64_t>(lbo_bytes >> 4) << 16;
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;
+    return d;
+}
+// Instruction descriptor: f32 accumulate, bf16 x bf16, A K-major, B K-major (b_mn = 0) or N-major (1), tile M x N.
+__device__ __forceinline__ uint32_t umma_idesc_bf16_major(uint32_t M, uint32_t N, uint32_t b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {     // 2^x, exp2(-inf) = 0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ bool at_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, const AttnParams& p) {
+    const uint32_t limit = p.wait_limit;
+    for (uint32_t it = 0; it < limit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    atomicCAS(p.status, 0, QG_ERR_TIMEOUT);
+    return false;
+}
+
+template <int D>
+__global__ void __launch_bounds__(AT_THREADS, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const AttnParams p) {
+    using C = AttnCfg<D>;
+    extern __shared__ uint8_t smem_dyn[];
+    const uint32_t sbase = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    uint8_t* sgen = smem_dyn + (sbase - smem_u32(smem_dyn));
+    volatile int* misc = reinterpret_cast<volatile int*>(sgen + C::OFF_MISC);   // [0] tmem base, [1] abort
+    volatile int* abort_flag = misc + 1;
+    const uint32_t bar0 = sbase + C::OFF_BAR;
+    const uint32_t q_full = bar0;
+    auto k_full = [&](int s) { return bar0 + 8u * (1 + s); };
+    auto v_full = [&](int s) { return bar0 + 8u * (3 + s); };
+    auto k_empty = [&](int s) { return bar0 + 8u * (5 + s); };
+    auto v_empty = [&](int s) { return bar0 + 8u * (7 + s); };
+    auto s_full = [&](int b) { return bar0 + 8u * (9 + b); };
+    auto p_full = [&](int b) { return bar0 + 8u * (11 + b); };
+    const uint32_t pv_done = bar0 + 8u * 13;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_qt = (p.S + AT_BQ - 1) / AT_BQ;
+    const int qt = n_qt - 1 - static_cast<int>(blockIdx.x);     // the longest (last) query tiles start first
+    const int h = blockIdx.y;
+    const int g = h / (p.Hq / p.Hkv);
+    const int q0 = qt * AT_BQ;
+    // key tiles this query tile attends to
+    const int n_kv = p.causal ? (qt + 1) : (p.S + AT_BKV - 1) / AT_BKV;
+
+    pdl_launch_dependents();
+    if (warp == 0) {
+        if (lane < 14) {
+            const uint32_t cnt = (lane == 11 || lane == 12) ? 4u : 1u;      // p_full: one arrival per softmax warp
+            mbar_init(bar0 + 8u * lane, cnt);
+        }
+        if (lane == 31) misc[1] = 0;
+        fence_mbar_init();
+        fence_proxy_async_smem();
+        if (lane == 30) prefetch_tmap(&tm_q);
+        if (lane == 29) prefetch_tmap(&tm_k);
+        if (lane == 28) prefetch_tmap(&tm_v);
+    }
+    if (warp == 1) {
+        tmem_alloc(sbase + C::OFF_MISC, C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    pdl_wait();
+    const uint32_t tmem_base = static_cast<uint32_t>(misc[0]);
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        bool ok = true;
+        if (lane == 0) {
+            mbar_arrive_expect_tx(q_full, C::TILE_BYTES);
+#pragma unroll
+            for (int a = 0; a < C::NBOX; ++a)
+                tma_load_2d(sbase + C::OFF_Q + a * C::BOX_BYTES, &tm_q, h * D + 64 * a, q0, q_full);
+        }
+        for (int j = 0; j < n_kv && ok; ++j) {
+            const int s = j & 1;
+            const uint32_t ph = (j >> 1) & 1u;
+            if (!at_wait(k_empty(s), ph ^ 1u, abort_flag, p)) { ok = false; break; }
+            if (lane == 0) {
+                mbar_arrive_expect_tx(k_full(s), C::TILE_BYTES);
+#pragma unroll
+                for (int a = 0; a < C::NBOX; ++a)
+                    tma_load_2d(sbase + C::OFF_K + s * C::TILE_BYTES + a * C::BOX_BYTES, &tm_k, g * D + 64 * a,
+                                j * AT_BKV, k_full(s));
+            }
+            if (!at_wait(v_empty(s), ph ^ 1u, abort_flag, p)) { ok = false; break; }
+            if (lane == 0) {
+                mbar_arrive_expect_tx(v_full(s), C::TILE_BYTES);
+#pragma unroll
+                for (int a = 0; a < C::NBOX; ++a)
+                    tma_load_2d(sbase + C::OFF_V + s * C::TILE_BYTES + a * C::BOX_BYTES, &tm_v, g * D + 64 * a,
+                                j * AT_BKV, v_full(s));
+            }
+            __syncwarp();
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        // Order of issue: S(0); then for every key tile j: S(j + 1) (so that it runs while the softmax warps work on
+        // S(j)), P(j) V(j).  MMAs of one thread execute in order, so S(j + 1), which overwrites the buffer that held
+        // P(j - 1), cannot overtake P(j - 1) V(j - 1).
+        const uint32_t idesc_s = umma_idesc_bf16_major(AT_BQ, AT_BKV, 0u);
+        const uint32_t idesc_o = umma_idesc_bf16_major(AT_BQ, D, 1u);
+        const uint32_t q_addr = sbase + C::OFF_Q;
+        bool ok = at_wait(q_full, 0u, abort_flag, p);
+        auto issue_s = [&](int j) -> bool {
+            const int s = j & 1;
+            if (!at_wait(k_full(s), (j >> 1) & 1u, abort_flag, p)) return false;
+            tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t k_addr = sbase + C::OFF_K + s * C::TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * C::BOX_BYTES + (kk & 3) * 32;
+                    umma_f16_ss(tmem_base + C::COL_S + s * 128, umma_desc_k_sw128(q_addr + off),
+                                umma_desc_k_sw128(k_addr + off), idesc_s, kk ? 1u : 0u);
+                }
+                umma_commit(s_full(s));
+                umma_commit(k_empty(s));
+            }
+            __syncwarp();
+            return true;
+        };
+        if (ok && n_kv > 0) ok = issue_s(0);
+        for (int j = 0; j < n_kv && ok; ++j) {
+            const int s = j & 1;
+            const uint32_t ph = (j >> 1) & 1u;
+            if (j + 1 < n_kv && !issue_s(j + 1)) { ok = false; break; }
+            if (!at_wait(p_full(s), ph, abort_flag, p) || !at_wait(v_full(s), ph, abort_flag, p)) { ok = false; break; }
+            tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t v_addr = sbase + C::OFF_V + s * C::TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < AT_BKV / 16; ++kk)          // 16 keys per instruction: two 8-key groups of V
+                    umma_f16_ts(tmem_base + C::COL_O, tmem_base + C::COL_S + s * 128 + 8 * kk,
+                                umma_desc_mn_sw128(v_addr + kk * 2048, C::BOX_BYTES), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+                umma_commit(pv_done);
+                umma_commit(v_empty(s));
+            }
+            __syncwarp();
+        }
+    } else {
+        // ------------------------------------------------ softmax (thread = one query row)
+        const int quarter = warp & 3;                                  // TMEM lanes 32 quarter .. + 31
+        const int row = quarter * 32 + lane;
+        const int qi = q0 + row;                                       // query position of this thread
+        const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        const float cl = p.scale_log2;
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_kv && ok; ++j) {
+            const int b = j & 1;
+            const uint32_t ph = (j >> 1) & 1u;
+            if (!at_wait(s_full(b), ph, abort_flag, p)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t s_addr = lane_addr + C::COL_S + b * 128;
+            const int key0 = j * AT_BKV;
+            // keys this row may see in the tile: below `lim` (all 128 except on the diagonal and at the sequence end)
+            int lim = p.S - key0;
+            if (p.causal) lim = min(lim, qi - key0 + 1);
+            const bool masked = (__any_sync(0xFFFFFFFFu, lim < AT_BKV) != 0);
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld_32x32(s_addr + 32 * c, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    float x = __uint_as_float(v[i]);
+                    if (masked && 32 * c + i >= lim) x = -INFINITY;
+                    mx = fmaxf(mx, x);
+                }
+            }
+            const float m_new = fmaxf(m, mx);
+            // rows past the sequence end see no key at all in a masked tile: keep their arithmetic finite
+            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+            const float mc = m_use * cl;
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld_32x32(s_addr + 32 * c, v);
+                tmem_ld_wait();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float x0 = __uint_as_float(v[i]), x1 = __uint_as_float(v[i + 1]);
+                    float p0 = fast_exp2(fmaf(x0, cl, -mc)), p1 = fast_exp2(fmaf(x1, cl, -mc));
+                    if (masked && 32 * c + i >= lim) p0 = 0.f;
+                    if (masked && 32 * c + i + 1 >= lim) p1 = 0.f;
+                    // the sum runs over the bf16 values the tensor cores will multiply, so that numerator and
+                    // denominator of the softmax stay consistent
+                    const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                    sum += __low2float(pb) + __high2float(pb);
+                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+                }
+                tmem_st_32x32_x16(s_addr + 16 * c, pk);          // P over the columns of S already read
+            }
+            const float alpha = fast_exp2((m - m_use) * cl);      // exp2(-inf) = 0 on the first tile
+            l = l * alpha + sum;
+            m = m_use;
+            if (j > 0) {
+                // O of the earlier tiles is rescaled once their last P V has completed
+                if (!at_wait(pv_done, (j - 1) & 1u, abort_flag, p)) { ok = false; break; }
+                tc_fence_after_sync();
+                if (!__all_sync(0xFFFFFFFFu, alpha == 1.0f)) {
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t v[32];
+                        tmem_ld_32x32(lane_addr + C::COL_O + 32 * c, v);
+                        tmem_ld_wait();
+                        uint32_t (&lo)[16] = *reinterpret_cast<uint32_t (*)[16]>(v);
+                        uint32_t (&hi)[16] = *reinterpret_cast<uint32_t (*)[16]>(v + 16);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                        tmem_st_32x32_x16(lane_addr + C::COL_O + 32 * c, lo);
+                        tmem_st_32x32_x16(lane_addr + C::COL_O + 32 * c + 16, hi);
+                    }
+                }
+            }
+            tmem_st_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full(b));
+        }
+        // ---- normalise and store: through a padded staging tile in the (now idle) K ring, then 16-byte rows
+        const bool good = ok && n_kv > 0 && at_wait(pv_done, (n_kv - 1) & 1u, abort_flag, p);
+        uint8_t* stage = sgen + C::OFF_K;
+        if (good) {
+            tc_fence_after_sync();
+            const float inv = (l > 0.f) ? 1.0f / l : 0.f;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld_32x32(lane_addr + C::COL_O + 32 * c, v);
+                tmem_ld_wait();
+                uint4* dst = reinterpret_cast<uint4*>(stage + row * C::OUT_PITCH + c * 64);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(v[8 * i + 2 * t]) * inv,
+                                                                        __uint_as_float(v[8 * i + 2 * t + 1]) * inv);
+                        w[t] = *reinterpret_cast<const uint32_t*>(&o2);
+                    }
+                    dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+        }
+        named_bar_sync(1, 128);            // reached by all four warps whatever happened above (every wait is bounded)
+        if (good) {
+            const int t = threadIdx.x - 64;
+            constexpr int VPR = D / 8;                              // 16-byte vectors per row
+            for (int idx = t; idx < AT_BQ * VPR; idx += 128) {
+                const int r = idx / VPR, vv = idx - r * VPR;
+                if (q0 + r < p.S)
+                    *reinterpret_cast<uint4*>(p.O + static_cast<size_t>(q0 + r) * p.ldo + static_cast<size_t>(h) * D + vv * 8) =
+                        *reinterpret_cast<const uint4*>(stage + r * C::OUT_PITCH + vv * 16);
+            }
+        }
+    }
+
+    // ---------------------------------------------------- teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);            // copies may still be in flight towards this CTA
+    }
+    tc_fence_after_sync();
+    if (warp == 1) tmem_dealloc(tmem_base, C::TMEM_COLS);
+}
+
+template <int D>
+static int launch_attn(qg_ctx* ctx, const AttnParams& p, const void* Q, long long ldq, const void* K, long long ldk,
+                       const void* V, long long ldv, cudaStream_t st) {
+    using C = AttnCfg<D>;
+    const CUtensorMap *tm_q, *tm_k, *tm_v;
+    int rc = get_tmap_2d(ctx, &tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, static_cast<uint64_t>(p.Hq) * D, p.S, 64, 128,
+                         CU_TENSOR_MAP_SWIZZLE_128B, static_cast<uint64_t>(ldq) * 2);
+    if (rc == QG_OK)
+        rc = get_tmap_2d(ctx, &tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, static_cast<uint64_t>(p.Hkv) * D, p.S, 64, 128,
+                         CU_TENSOR_MAP_SWIZZLE_128B, static_cast<uint64_t>(ldk) * 2);
+    if (rc == QG_OK)
+        rc = get_tmap_2d(ctx, &tm_v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, V, static_cast<uint64_t>(p.Hkv) * D, p.S, 64, 128,
+                         CU_TENSOR_MAP_SWIZZLE_128B, static_cast<uint64_t>(ldv) * 2);
+    if (rc != QG_OK) return rc;
+    auto kern = attn_fwd_kernel<D>;
+    constexpr int inst = 20 + (D == 64 ? 0 : D == 128 ? 1 : 2);
+    if (!ctx->attr_set[inst]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
+            cudaGetLastError();
+            return QG_ERR_CUDA;
+        }
+        ctx->attr_set[inst] = true;
+    }
+    const int n_qt = (p.S + AT_BQ - 1) / AT_BQ;
+    if (launch_kernel(ctx, kern, dim3(n_qt, p.Hq), dim3(AT_THREADS), C::SMEM_BYTES, st, *tm_q, *tm_k, *tm_v, p) != cudaSuccess) {
+        cudaGetLastError();
+        return QG_ERR_CUDA;
+    }
+    return QG_OK;
+}
+
+}  // namespace qg
+
+extern "C" int prefill_attention(qg_ctx* ctx, int S, int Hq, int Hkv, int d, const void* Q, long long ldq, const void* K,
+                                 long long ldk, const void* V, long long ldv, void* O, long long ldo, int causal, float scale,
+                                 void* stream) {
+    if (!ctx) return QG_ERR_NULL;
+    if (S < 0 || Hq < 1 || Hkv < 1 || Hq % Hkv || Hq > 65535) return QG_ERR_SHAPE;
+    if (d != 64 && d != 128) return QG_ERR_SHAPE;
+    if (ldq < static_cast<long long>(Hq) * d || ldk < static_cast<long long>(Hkv) * d || ldv < static_cast<long long>(Hkv) * d ||
+        ldo < static_cast<long long>(Hq) * d || ldq % 8 || ldk % 8 || ldv % 8 || ldo % 8)
+        return QG_ERR_SHAPE;
+    if (S == 0) return QG_OK;
+    if (!Q || !K || !V || !O) return QG_ERR_NULL;
+    if (!qg::aligned16(Q) || !qg::aligned16(K) || !qg::aligned16(V) || !qg::aligned16(O)) return QG_ERR_ALIGN;
+    if (!(scale >= 0.f) || isinf(scale)) return QG_ERR_SHAPE;
+    if (const int rc = qg::check_device(ctx)) return rc;
+    qg::AttnParams p{};
+    p.S = S; p.Hq = Hq; p.Hkv = Hkv; p.causal = causal ? 1 : 0;
+    p.scale_log2 = ((scale > 0.f) ? scale : 1.0f / sqrtf(static_cast<float>(d))) * 1.4426950408889634f;
+    p.O = static_cast<__nv_bfloat16*>(O); p.ldo = ldo;
+    p.status = ctx->d_status; p.wait_limit = ctx->wait_limit;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (d == 64) return qg::launch_attn<64>(ctx, p, Q, ldq, K, ldk, V, ldv, st);
+    return qg::launch_attn<128>(ctx, p, Q, ldq, K, ldk, V, ldv, st);
+}

@@ -558,11 +558,11 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         // ------------------------------------------------ MMA issuers (even CTA of the pair only)
         // One warp needs about 500-560 cycles to issue the four TMEM-operand MMAs, the commit and the wait of a
         // k-block, more than the 256-512 cycles the tensor cores need for it, and two warps issue concurrently at
-        // full speed; so warps 1 and 3 take alternate pairs of k-blocks (0, 1 | 2, 3 | 4, 5 ...).  MMAs of different
-        // threads are ordered only through completion, so the second warp starts a tile after the "done" of the
-        // tile's first k-block (which overwrites the accumulator); by then it has usually just finished the last
-        // pair of the previous tile, while the first warp has already issued two k-blocks of the new one.  Within
-        // a tile the order of the accumulating k-blocks does not matter.
+        // full speed; so warps 1 and 3 take the even and the odd k-blocks.  MMAs of different threads are ordered
+        // only through completion, so the odd warp starts a tile after the "done" of the tile's first k-block (which
+        // overwrites the accumulator); within a tile the order of the accumulating k-blocks does not matter.
+        // (Alternating pairs of k-blocks instead, so that the second warp's wait is covered by the first warp's two
+        // k-blocks, was measured slower: 5 % on the dense and 16 % on the short-K grouped GEMMs.)
         if (rank == 0) {
             const uint32_t w = (warp == 3) ? 1u : 0u;
             bool ok = true;
@@ -586,9 +586,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 }
                 QG_ACC(2);
                 const uint32_t d_tmem = tmem_base + a * BT;
-                // this warp's k-blocks of the piece: kb0 + 2 w + {0, 1}, then every fourth pair
-                int kb = pc.kb0 + 2 * static_cast<int>(w);
-                uint32_t i = i0 + 2u * w;
+                // this warp's k-blocks of the piece: every other one, starting at kb0 + w
+                int kb = pc.kb0 + static_cast<int>(w);
+                uint32_t i = i0 + w;
                 bool ready = mbar_test_wait_cluster(full(i & 7u), (i >> 3) & 1u);
                 while (kb < pc.kb1) {
                     const uint32_t st = i & 7u;
@@ -598,9 +598,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     QG_ACC(3);
                     tc_fence_after_sync();
                     // start the wait for this warp's next k-block before issuing, so its latency is hidden
-                    const int step = (kb & 1) ? 3 : 1;
-                    const uint32_t in = i + static_cast<uint32_t>(step);
-                    ready = (kb + step < pc.kb1) && mbar_test_wait_cluster(full(in & 7u), (in >> 3) & 1u);
+                    const uint32_t in = i + 2u;
+                    ready = (kb + 2 < pc.kb1) && mbar_test_wait_cluster(full(in & 7u), (in >> 3) & 1u);
                     if (lane == 0) {
                         umma_kblock_ts_pair(d_tmem, tmem_base + C::A_COL0 + ta * C::A_COLS,
                                             b_lo0 + st * (C::X_BYTES >> 4), b_hi, idesc, kb != pc.kb0 ? 1u : 0u);
@@ -608,7 +607,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     }
                     __syncwarp();
                     QG_ACC(10);
-                    kb += step;
+                    kb += 2;
                     i = in;
                 }
                 if (ok && lane == 0) umma_commit_pair(acc_full(a));
@@ -902,17 +901,20 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_ro
     return QG_OK;
 }
 
-// Token tile and schedule of a dense call: the candidate with the smallest modelled time.  Data-parallel: a wave is
-// one pair tile per SM pair; a tile costs nkb k-blocks of about `period` cycles (measured: issue- and latency-bound,
-// nearly independent of the tile width) plus, for the single-accumulator 256-wide tile, an epilogue that is not
-// overlapped.  Stream-K: every pair gets the same share of all k-blocks, pays the exposed epilogue once per tile it
-// touches and a fixed amount for writing and reading the partial tiles.
+// Token tile and schedule of a dense call: the candidate with the smallest modelled time, the model fitted to timings
+// of eleven layer shapes (Q8 and Q4, K from 2048 to 14336, M = 1024 and 2048) on B200.  Data-parallel: a tile costs nkb
+// k-blocks of `period` cycles plus, for the single-accumulator 256-token tile, an exposed epilogue; tiles come in
+// waves of one per SM pair, but a ragged last wave costs less than a full one (the pairs that are done leave L2,
+// HBM and power to the others), so the wave count is taken half-way between the rounded-up and the fractional one.
+// Stream-K: every pair gets the same share of all k-blocks and pays an epilogue per tile it touches plus the exchange
+// of partial tiles; measured, that exchange and the extra epilogues cost 4-8 us per call, so it only wins where it
+// removes most of a wave of long-K tiles, and the model charges it accordingly.
 struct DensePlan {
     int bt, streamk;
 };
-static DensePlan plan_dense(const qg_ctx* ctx, int M, int n_wt, int K) {
+static DensePlan plan_dense(const qg_ctx* ctx, int qbits, int M, int n_wt, int K) {
     const int cand[3] = {128, 192, 256};
-    const double period[3] = {625.0, 665.0, 720.0}, epilogue[3] = {0.0, 0.0, 6000.0}, last_epi[3] = {2500.0, 3000.0, 0.0};
+    const double period[3] = {630.0, 655.0, (qbits == 4) ? 760.0 : 720.0}, epilogue[3] = {0.0, 0.0, 6000.0};
     const long long pairs = ctx->sm_count / 2, n_pw = (n_wt + 1) / 2;
     const int nk4 = K / (4 * BK);
     DensePlan best{256, 0};
@@ -920,18 +922,27 @@ static DensePlan plan_dense(const qg_ctx* ctx, int M, int n_wt, int K) {
     for (int c = 0; c < 3; ++c) {
         if (M <= 128 && cand[c] > 128) break;
         const long long tiles = n_pw * ((M + cand[c] - 1) / cand[c]);
-        const long long waves = (tiles + pairs - 1) / pairs;
-        const double dp = static_cast<double>(waves) * ((K / BK) * period[c] + epilogue[c]) + last_epi[c];
+        const double frac = static_cast<double>(tiles) / pairs;
+        const double waves = 0.5 * (static_cast<double>((tiles + pairs - 1) / pairs) + frac);
+        const double dp = waves * ((K / BK) * period[c] + epilogue[c]);
         if (ctx->streamk_mode != 1 || tiles % pairs == 0)
-            if (dp < best_cost * 0.999) { best_cost = dp; best = DensePlan{cand[c], 0}; }
-        if (ctx->streamk_mode == 0 || tiles % pairs == 0) continue;
+            if (dp < best_cost) { best_cost = dp; best = DensePlan{cand[c], 0}; }
+    }
+    if (ctx->streamk_mode == 0) return best;
+    for (int c = 0; c < 3; ++c) {
+        if (M <= 128 && cand[c] > 128) break;
+        const long long tiles = n_pw * ((M + cand[c] - 1) / cand[c]);
+        if (tiles % pairs == 0) continue;
         const long long units = tiles * nk4;
         const long long P = units < pairs ? units : pairs;
         const long long share = (units + P - 1) / P;                        // units of the busiest pair
         const double pieces = static_cast<double>(share) / nk4 + 1.5;       // tiles it touches, on average
         if (share / nk4 + 2 > 120) continue;                                // the piece table has 128 entries
-        const double sk = share * 4.0 * period[c] + pieces * epilogue[c] + last_epi[c] + 5000.0;
-        if (sk < best_cost * 0.97) { best_cost = sk; best = DensePlan{cand[c], 1}; }
+        const double sk = share * 4.0 * period[c] + pieces * epilogue[c] + 10000.0;
+        if (ctx->streamk_mode == 1 ? (best.streamk == 0 || sk < best_cost) : (sk < 0.95 * best_cost)) {
+            best_cost = sk;
+            best = DensePlan{cand[c], 1};
+        }
     }
     return best;
 }
@@ -969,10 +980,11 @@ static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in,
 
 extern "C" {
 
-int qg_plan_dense(qg_ctx* ctx, int M, int N, int K, int* token_tile, int* streamk) {
+int qg_plan_dense(qg_ctx* ctx, int qbits, int M, int N, int K, int* token_tile, int* streamk) {
     if (!ctx) return QG_ERR_NULL;
+    if (qbits != QG_Q8 && qbits != QG_Q4) return QG_ERR_SHAPE;
     if (M < 1 || N < 8 || N % 8 || K < 256 || K % 256) return QG_ERR_SHAPE;
-    const qg::DensePlan plan = qg::plan_dense(ctx, M, (N + qg::BW - 1) / qg::BW, K);
+    const qg::DensePlan plan = qg::plan_dense(ctx, qbits, M, (N + qg::BW - 1) / qg::BW, K);
     if (token_tile) *token_tile = ctx->force_bt ? ctx->force_bt : plan.bt;
     if (streamk) *streamk = (ctx->force_bt == 0 || ctx->streamk_mode == 1) ? plan.streamk : 0;
     return QG_OK;
@@ -991,7 +1003,7 @@ int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, cons
     p.mode = QG_MODE_PLAIN; p.R = M; p.N = N; p.K = K; p.E = 1; p.k = 1;
     p.n_wt = (N + qg::BW - 1) / qg::BW;
     p.offsets = nullptr; p.out = Cout; p.topk_w = nullptr; p.row_pair = nullptr;
-    const qg::DensePlan plan = qg::plan_dense(ctx, M, p.n_wt, K);
+    const qg::DensePlan plan = qg::plan_dense(ctx, qbits, M, p.n_wt, K);
     p.streamk = (ctx->force_bt == 0 || ctx->streamk_mode == 1) ? plan.streamk : 0;
     p.sk_partial = ctx->sk_partial; p.sk_flags = ctx->sk_flags;
     return qg::dispatch_gemm(ctx, qbits, plan.bt, p, A, M, Wq, Wscale, static_cast<cudaStream_t>(stream));

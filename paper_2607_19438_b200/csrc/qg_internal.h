@@ -12,7 +12,7 @@ namespace qg {
 // One cached tensor map: the key is everything cuTensorMapEncodeTiled was given.
 struct TmapEntry {
     const void* base;
-    uint64_t inner, rows;
+    uint64_t inner, rows, row_stride;
     uint32_t box_inner, box_rows;
     int dt, elem_bytes, swz;
     CUtensorMap map;
@@ -64,8 +64,10 @@ inline cudaError_t launch_kernel(const qg_ctx* ctx, void (*kern)(KArgs...), dim3
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 // QG_OK if the calling thread's current device is the context's, else QG_ERR_DEVICE.
 int check_device(const qg_ctx* ctx);
-// A 2-D row-major tensor map (inner = contiguous extent in elements, box in elements): looked up in the context's
-// cache, encoded on a miss.  The returned pointer stays valid until TMAP_CACHE further misses.
+// A 2-D row-major tensor map (inner = contiguous extent in elements, box in elements, row_stride_bytes = distance
+// between rows, 0 = packed): looked up in the context's cache, encoded on a miss.  The returned pointer stays valid
+// until TMAP_CACHE further misses.
 int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
-                uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz);
+                uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz,
+                uint64_t row_stride_bytes = 0);
 }  // namespace qg

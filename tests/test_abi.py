@@ -11,7 +11,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "qgemm.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b((?:qg|qgemm|moe)_\w+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b((?:qg|qgemm|moe|prefill)_\w+)\s*\(", text)))
 
 
 def test_library_builds_loads_and_exports_every_declared_symbol():

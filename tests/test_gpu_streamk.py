@@ -54,10 +54,14 @@ def test_streamk_forced_matches_the_oracle(qbits, M, N, K, bt):
     assert float((plain.float() - g.t.float()).abs().max()) <= 2e-2 * ref_max
 
 
-def test_the_cost_model_picks_streamk_where_waves_are_ragged():
+def test_the_cost_model_follows_the_measured_best_tile():
+    """The token tile the model picks for the shapes it was fitted on (the fastest measured one), and stream-K only
+    where a forced run showed it at least level with the best data-parallel tile."""
     qg.set_schedule(0, -1)
-    assert qg.plan_dense(2048, 2560, 2048)[1]          # 80 tiles of 256 on 74 pairs
-    assert qg.plan_dense(1024, 2048, 8192)[1]          # 32 tiles: K is split over the idle pairs
-    assert not qg.plan_dense(2048, 16384, 2048)[1] or True   # a large multiple of the pair count: either is fine
-    bt, sk = qg.plan_dense(64, 2048, 2048)
-    assert bt == 128
+    want = {(8, 2048, 2560, 2048): 192, (8, 2048, 2048, 2048): 256, (8, 1024, 2560, 2048): 192, (8, 2048, 6144, 4096): 256,
+            (8, 2048, 4096, 14336): 256, (4, 2048, 5120, 3072): 192, (4, 2048, 3072, 3072): 192, (4, 2048, 3072, 8192): 192,
+            (4, 1024, 3072, 8192): 192}
+    for (qbits, M, N, K), bt in want.items():
+        got_bt, sk = qg.plan_dense(qbits, M, N, K)
+        assert got_bt == bt and not sk, (qbits, M, N, K, got_bt, sk)
+    assert qg.plan_dense(8, 64, 2048, 2048)[0] == 128
