@@ -8,9 +8,10 @@
 //
 // Work split.  A block owns 64 weight rows x one K slice; its 8 warps own 8 rows each.  The token rows of the slice
 // (16 x KS bf16, rows past M zero) and the slice's scales sit in shared memory.  Lane (g, j) = (lane / 4, lane % 4)
-// streams the 8 codes k = 8 j .. 8 j + 7 of row g of every 32-wide block straight from global memory (8 or 4 bytes,
-// eight blocks in flight) and feeds two MMAs with them; the summation index inside a block is permuted the same
-// way on the activation side, so no shuffles are needed.  K slices of one row tile are reduced in a fixed order by
+// streams the 16 codes k = 16 j .. 16 j + 15 of row g of every 64-wide chunk straight from global memory (16 or 8
+// bytes per load, eight loads in flight, the first ones issued before anything else in the kernel) and feeds four
+// MMAs with them; the summation index inside a chunk is permuted the same way on the activation side, so no
+// shuffles are needed.  K slices of one row tile are reduced in a fixed order by
 // whichever block finishes last (partial tiles in the context's workspace, one ticket per row tile), so the result
 // does not depend on the order in which blocks run.
 #include <cuda_bf16.h>
@@ -25,13 +26,18 @@ namespace qg {
 constexpr int GV_ROWS = 64;          // weight rows per block (8 per warp)
 constexpr int GV_THREADS = 256;
 constexpr int GV_MAX_KS = 2048;      // largest K slice (activation slice 16 x 2048 bf16 = 64 KB)
-constexpr int GV_UNROLL = 8;         // 32-wide blocks in flight per lane
+constexpr int GV_BATCH = 4;          // 64-wide chunks per batch of loads; two batches are in flight per lane
 
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
                  "{%0, %1, %2, %3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint4 ldg_stream128(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
 }
 __device__ __forceinline__ uint2 ldg_stream64(const void* p) {
     uint2 v;
@@ -54,14 +60,15 @@ struct GemvParams {
     int* tickets;         // one per row tile, zero between launches
 };
 
-// Shared memory: activation slice [16][KS + 32] bf16 (row stride = 128 B multiple + 64 B, so the two rows a quarter
-// warp reads with 16-byte loads fall on different banks), then scales [64][KS / 32 + 2] fp16, then one int.
+// Shared memory: activation slice [16][KS + 8] bf16 (row stride = 128 B multiple + 16 B, so the two rows and four
+// 32-byte spans a quarter warp reads with 16-byte loads fall on different banks), then scales [64][KS / 32 + 2] fp16,
+// then one int.
 template <int QBITS>
 __global__ void __launch_bounds__(GV_THREADS)
 qgemv_kernel(const GemvParams p) {
     extern __shared__ __align__(16) uint8_t smem[];
     const int KS = p.KS;
-    const int a_stride = KS + 32;                        // elements
+    const int a_stride = KS + 8;                         // elements
     const int s_stride = KS / 32 + 2;
     __nv_bfloat16* sA = reinterpret_cast<__nv_bfloat16*>(smem);
     __half* sS = reinterpret_cast<__half*>(smem + static_cast<size_t>(16) * a_stride * 2);
@@ -74,7 +81,28 @@ qgemv_kernel(const GemvParams p) {
     const int n0 = tile * GV_ROWS;
     pdl_launch_dependents();
 
-    // scales of the slice (weights and scales are constants of the model: no need to wait for the previous kernel)
+    const int row = n0 + warp * 8 + g;                   // the weight row whose codes this lane streams
+    const bool row_ok = row < p.N;                       // N % 8 == 0: a warp's eight rows are all inside or all outside
+    constexpr int BYTES_PER_CHUNK = (QBITS == 8) ? 64 : 32;
+    const uint8_t* wrow = p.Wq + static_cast<size_t>(row_ok ? row : 0) * (static_cast<size_t>(p.K) * QBITS / 8) +
+                          static_cast<size_t>(k0) * QBITS / 8 + j * (BYTES_PER_CHUNK / 4);
+    const int nch = ks >> 6;                             // 64-wide chunks of the slice, a multiple of 4
+    auto load_batch = [&](uint4 (&raw)[GV_BATCH], int c0) {
+#pragma unroll
+        for (int u = 0; u < GV_BATCH; ++u) {
+            if constexpr (QBITS == 8) {
+                raw[u] = ldg_stream128(wrow + static_cast<size_t>(c0 + u) * BYTES_PER_CHUNK);
+            } else {
+                const uint2 v = ldg_stream64(wrow + static_cast<size_t>(c0 + u) * BYTES_PER_CHUNK);
+                raw[u] = make_uint4(v.x, v.y, 0u, 0u);
+            }
+        }
+    };
+    // weights are constants of the model: the first loads go out before the previous kernel is waited for
+    uint4 raw_a[GV_BATCH], raw_b[GV_BATCH];
+    if (row_ok) load_batch(raw_a, 0);
+
+    // scales of the slice
     const int nsb = ks >> 5;
     for (int i = threadIdx.x; i < GV_ROWS * nsb; i += GV_THREADS) {
         const int r = i / nsb, b = i - r * nsb;
@@ -93,48 +121,48 @@ qgemv_kernel(const GemvParams p) {
     __syncthreads();
 
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    const int row = n0 + warp * 8 + g;                   // the weight row whose codes this lane streams
-    const bool row_ok = row < p.N;                       // N % 8 == 0: a warp's eight rows are all inside or all outside
     if (row_ok) {
-        constexpr int BYTES_PER_BLOCK = (QBITS == 8) ? 32 : 16;
-        const uint8_t* wrow = p.Wq + static_cast<size_t>(row) * (static_cast<size_t>(p.K) * QBITS / 8) +
-                              static_cast<size_t>(k0) * QBITS / 8 + j * (BYTES_PER_BLOCK / 4);
-        const __half* srow = sS + (warp * 8 + g) * s_stride;
-        const __nv_bfloat16* a_lo = sA + g * a_stride + 8 * j;
-        const __nv_bfloat16* a_hi = sA + (g + 8) * a_stride + 8 * j;
-        for (int b0 = 0; b0 < nsb; b0 += GV_UNROLL) {     // nsb is a multiple of 8
-            uint32_t raw[GV_UNROLL][2];
+        const __half* srow = sS + (warp * 8 + g) * s_stride + (j >> 1);
+        const __nv_bfloat16* a_lo = sA + g * a_stride + 16 * j;
+        const __nv_bfloat16* a_hi = sA + (g + 8) * a_stride + 16 * j;
+        auto compute_batch = [&](const uint4 (&raw)[GV_BATCH], int c0) {
 #pragma unroll
-            for (int u = 0; u < GV_UNROLL; ++u) {
-                if constexpr (QBITS == 8) {
-                    const uint2 v = ldg_stream64(wrow + static_cast<size_t>(b0 + u) * BYTES_PER_BLOCK);
-                    raw[u][0] = v.x; raw[u][1] = v.y;
-                } else {
-                    raw[u][0] = ldg_stream32(wrow + static_cast<size_t>(b0 + u) * BYTES_PER_BLOCK);
-                    raw[u][1] = 0u;
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < GV_UNROLL; ++u) {
-                const float sc = __half2float(srow[b0 + u]);
+            for (int u = 0; u < GV_BATCH; ++u) {
+                const int c = c0 + u;
+                const float sc = __half2float(srow[2 * c]);     // the 32-block that holds k = 16 j .. 16 j + 15
                 uint64_t m2, c2;
                 dq_consts(sc, QBITS == 8, m2, c2);
-                uint32_t w[4];                              // 8 bf16: k = 8 j .. 8 j + 7 of this block, row g
+                uint32_t w[8];                                   // 16 bf16: k = 16 j .. 16 j + 15 of this chunk, row g
                 if constexpr (QBITS == 8) {
-                    dq8_word(raw[u][0], m2, c2, DQ_MAGIC, w[0], w[1]);
-                    dq8_word(raw[u][1], m2, c2, DQ_MAGIC, w[2], w[3]);
+                    dq8_word(raw[u].x, m2, c2, DQ_MAGIC, w[0], w[1]);
+                    dq8_word(raw[u].y, m2, c2, DQ_MAGIC, w[2], w[3]);
+                    dq8_word(raw[u].z, m2, c2, DQ_MAGIC, w[4], w[5]);
+                    dq8_word(raw[u].w, m2, c2, DQ_MAGIC, w[6], w[7]);
                 } else {
-                    dq4_word(raw[u][0], m2, c2, DQ_MAGIC, w);
+                    dq4_word(raw[u].x, m2, c2, DQ_MAGIC, w);
+                    dq4_word(raw[u].y, m2, c2, DQ_MAGIC, w + 4);
                 }
-                const uint4 lo = *reinterpret_cast<const uint4*>(a_lo + (b0 + u) * 32);   // A[g][k .. k + 7]
-                const uint4 hi = *reinterpret_cast<const uint4*>(a_hi + (b0 + u) * 32);   // A[g + 8][k .. k + 7]
-                // Fragment positions (k = 2 j, 2 j + 1 | 8 + 2 j, 9 + 2 j) carry the block's k = 8 j + {0, 1 | 2, 3} in
-                // the first MMA and 8 j + {4, 5 | 6, 7} in the second, on both operands alike.
-                const uint32_t a1[4] = {lo.x, hi.x, lo.y, hi.y};
-                const uint32_t a2[4] = {lo.z, hi.z, lo.w, hi.w};
-                mma_bf16_16816(acc, a1, w[0], w[1]);
-                mma_bf16_16816(acc, a2, w[2], w[3]);
+                const uint4 lo0 = *reinterpret_cast<const uint4*>(a_lo + c * 64);       // A[g][k .. k + 7]
+                const uint4 lo1 = *reinterpret_cast<const uint4*>(a_lo + c * 64 + 8);   // A[g][k + 8 .. k + 15]
+                const uint4 hi0 = *reinterpret_cast<const uint4*>(a_hi + c * 64);       // A[g + 8][..]
+                const uint4 hi1 = *reinterpret_cast<const uint4*>(a_hi + c * 64 + 8);
+                // MMA t multiplies the chunk's k = 16 j + 4 t + {0, 1 | 2, 3}: fragment positions (2 j, 2 j + 1 | 8 + 2 j,
+                // 9 + 2 j) on both operands alike
+                const uint32_t a0[4] = {lo0.x, hi0.x, lo0.y, hi0.y};
+                const uint32_t a1[4] = {lo0.z, hi0.z, lo0.w, hi0.w};
+                const uint32_t a2[4] = {lo1.x, hi1.x, lo1.y, hi1.y};
+                const uint32_t a3[4] = {lo1.z, hi1.z, lo1.w, hi1.w};
+                mma_bf16_16816(acc, a0, w[0], w[1]);
+                mma_bf16_16816(acc, a1, w[2], w[3]);
+                mma_bf16_16816(acc, a2, w[4], w[5]);
+                mma_bf16_16816(acc, a3, w[6], w[7]);
             }
+        };
+        for (int c0 = 0; c0 < nch; c0 += 2 * GV_BATCH) {
+            if (c0 + GV_BATCH < nch) load_batch(raw_b, c0 + GV_BATCH);
+            compute_batch(raw_a, c0);
+            if (c0 + 2 * GV_BATCH < nch) load_batch(raw_a, c0 + 2 * GV_BATCH);
+            if (c0 + GV_BATCH < nch) compute_batch(raw_b, c0 + GV_BATCH);
         }
     }
 
@@ -187,9 +215,10 @@ extern "C" int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const 
     if (!qg::aligned16(A) || !qg::aligned16(Wq) || !qg::aligned16(Wscale) || !qg::aligned16(Cout)) return QG_ERR_ALIGN;
     if (const int rc = qg::check_device(ctx)) return rc;
     const int tiles = (N + qg::GV_ROWS - 1) / qg::GV_ROWS;
-    // K slice: as small as 256 while that keeps raising the block count towards four waves, within the workspace
+    // K slice: halved while that raises the block count towards three blocks per SM, with at most eight slices
     int KS = qg::GV_MAX_KS;
-    while (KS > 256 && static_cast<long long>(tiles) * ((K + KS - 1) / KS) < 4LL * ctx->sm_count) KS >>= 1;
+    while (KS > 256 && (K + KS / 2 - 1) / (KS / 2) <= 8 &&
+           static_cast<long long>(tiles) * ((K + KS - 1) / KS) < 3LL * ctx->sm_count) KS >>= 1;
     int n_slices = (K + KS - 1) / KS;
     while (n_slices > 1 && (static_cast<size_t>(n_slices) * 16 * N * sizeof(float) > ctx->gemv_partial_bytes ||
                             tiles > ctx->gemv_ticket_count || n_slices > 32)) {
@@ -202,12 +231,12 @@ extern "C" int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const 
     p.A = static_cast<const __nv_bfloat16*>(A); p.Wq = static_cast<const uint8_t*>(Wq);
     p.Ws = static_cast<const __half*>(Wscale); p.C = static_cast<__nv_bfloat16*>(Cout);
     p.partial = ctx->gemv_partial; p.tickets = ctx->gemv_tickets;
-    const size_t smem = static_cast<size_t>(16) * (KS + 32) * 2 + static_cast<size_t>(qg::GV_ROWS) * (KS / 32 + 2) * 2 + 16;
+    const size_t smem = static_cast<size_t>(16) * (KS + 8) * 2 + static_cast<size_t>(qg::GV_ROWS) * (KS / 32 + 2) * 2 + 16;
     auto kern = (qbits == QG_Q8) ? qg::qgemv_kernel<8> : qg::qgemv_kernel<4>;
     const int inst = 18 + (qbits == QG_Q8 ? 0 : 1);
     if (!ctx->attr_set[inst]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 16 * (qg::GV_MAX_KS + 32) * 2 + qg::GV_ROWS * (qg::GV_MAX_KS / 32 + 2) * 2 + 16) != cudaSuccess) {
+                                 16 * (qg::GV_MAX_KS + 8) * 2 + qg::GV_ROWS * (qg::GV_MAX_KS / 32 + 2) * 2 + 16) != cudaSuccess) {
             cudaGetLastError();
             return QG_ERR_CUDA;
         }
