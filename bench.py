@@ -214,7 +214,6 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
     import ctypes as C
     P = lambda t: C.c_void_p(t.data_ptr())
     S = C.c_void_p(stream.cuda_stream)
-    S_ = S
     g = torch.Generator(device=dev); g.manual_seed(0)
 
     def chk(rc, what):
@@ -318,21 +317,21 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
 
     # prefill attention (causal, grouped-query heads), reading Q, K, V as column blocks of one fused-QKV buffer
     out["attention"] = []
-    for name, Hq, Hkv, d, S in (("cfg2 heads", 24, 8, 128, 2048), ("cfg4 heads", 32, 8, 128, 2048), ("cfg4 heads", 32, 8, 128, 8192)):
-        qkv = torch.randn((S, (Hq + 2 * Hkv) * d), device=dev, generator=g).to(torch.bfloat16)
+    for name, Hq, Hkv, d, Sq in (("cfg2 heads", 24, 8, 128, 2048), ("cfg4 heads", 32, 8, 128, 2048), ("cfg4 heads", 32, 8, 128, 8192)):
+        qkv = torch.randn((Sq, (Hq + 2 * Hkv) * d), device=dev, generator=g).to(torch.bfloat16)
         Q, K, V = qkv[:, :Hq * d], qkv[:, Hq * d:(Hq + Hkv) * d], qkv[:, (Hq + Hkv) * d:]
-        O = torch.empty((S, Hq * d), dtype=torch.bfloat16, device=dev)
-        fl = 4.0 * S * S * Hq * d / 2 + 2.0 * S * 128 * Hq * d     # causal: the lower triangle in 128-wide tiles incl. the diagonal
+        O = torch.empty((Sq, Hq * d), dtype=torch.bfloat16, device=dev)
+        fl = 4.0 * Sq * Sq * Hq * d / 2 + 2.0 * Sq * 128 * Hq * d     # causal: the lower triangle in 128-wide tiles incl. the diagonal
         calls = [("attention", fl, 0.0, lambda it: chk(lib.prefill_attention(
-            ctx, S, Hq, Hkv, d, P(Q), qkv.stride(0), P(K), qkv.stride(0), P(V), qkv.stride(0), P(O), O.stride(0), 1,
-            C.c_float(0.0), S_), "prefill_attention"))]
-        n_it = iters if S <= 2048 else max(5, iters // 2)
+            ctx, Sq, Hq, Hkv, d, P(Q), qkv.stride(0), P(K), qkv.stride(0), P(V), qkv.stride(0), P(O), O.stride(0), 1,
+            C.c_float(0.0), S), "prefill_attention"))]
+        n_it = iters if Sq <= 2048 else max(5, iters // 2)
         agg = timed_calls(calls, n_it)
         ms = agg["attention"][0] / n_it
-        out["attention"].append({"shape": name, "S": S, "Hq": Hq, "Hkv": Hkv, "d": d, "causal": True, "us": ms * 1e3,
+        out["attention"].append({"shape": name, "S": Sq, "Hq": Hq, "Hkv": Hkv, "d": d, "causal": True, "us": ms * 1e3,
                                  "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_measured_peak": fl / (ms * 1e-3) / 1e12 / peak_tf,
                                  "flops": "4 S^2 Hq d / 2 plus the diagonal tiles' upper halves that are computed and masked",
-                                 "tok_per_s": S / (ms * 1e-3)})
+                                 "tok_per_s": Sq / (ms * 1e-3)})
 
     H, E, k, F = MOE["H"], MOE["E"], MOE["k"], MOE["F"]
     W1q, W1s = weights(4, E * 2 * F, H); W2q, W2s = weights(4, E * H, F)

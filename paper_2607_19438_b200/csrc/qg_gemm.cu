@@ -171,9 +171,11 @@ __device__ __forceinline__ float lds_scale(uint32_t addr) {
 // every thread moves two 16-byte pieces to global memory (64 contiguous bytes per token).  The next block's TMEM
 // loads are in flight while the current one is stored.  Called by the four epilogue warps and, for a
 // single-accumulator tile, by the sixteen dequantising warps, which would otherwise idle at the tile boundary.
+template <bool SK>
 __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int tok_end, int n_base, uint32_t taddr,
-                                            int n_epi, int pid, int npart, __nv_bfloat16* st, int lane, int nsrc,
+                                            int n_epi, int pid, int npart, __nv_bfloat16* st, int lane, int nsrc_in,
                                             int quarter, int slot_floats, volatile int* abort_flag) {
+    const int nsrc = SK ? nsrc_in : 0;       // without stream-K all of the partial-tile handling below compiles away
     // The loop is issue-bound (five warps of a scheduler drain together), so everything that does not depend on the
     // block is computed once: the lane's two shared-memory read addresses, its global pointer and its token limit.
     const int nblk = n_epi >> 4;
@@ -185,9 +187,9 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
     // blocks in the slot's first flag.  The part that starts at k = 0 waits until every block of each of the nsrc
     // following pairs' slots is there, adds them in pair order and goes on as for a whole tile; the second flag
     // counts what has been read, and whoever reads last clears both for the next launch.
-    const int mine = (nblk - pid + npart - 1) / npart;          // blocks this warp drains
+    const int mine = SK ? (nblk - pid + npart - 1) / npart : 0;     // blocks this warp drains
     const int slot = static_cast<int>(blockIdx.x);
-    if (nsrc > 0) {
+    if (SK && nsrc > 0) {
         for (int c = 1; c <= nsrc; ++c) {
             const int* f = p.sk_flags + 2 * (slot + 2 * c);
             bool there = false;
@@ -234,7 +236,7 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
     const int left_step = 16 * npart;
     while (b < nblk) {
         tmem_ld_wait();
-        if (nsrc != 0) {
+        if (SK && nsrc != 0) {
             const size_t at = (static_cast<size_t>(b * 4 + quarter) * 16) * 32 + lane;
             if (nsrc < 0) {
                 float* dst = p.sk_partial + static_cast<size_t>(slot) * slot_floats + at;
@@ -301,11 +303,11 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
         left -= left_step;
         b = bn;
     }
-    if (nsrc < 0) {
+    if (SK && nsrc < 0) {
         __threadfence();
         __syncwarp();
         if (lane == 0) atomicAdd(p.sk_flags + 2 * slot, mine);
-    } else if (nsrc > 0) {
+    } else if (SK && nsrc > 0) {
         __syncwarp();
         if (lane == 0) {
             for (int c = 1; c <= nsrc; ++c) {
@@ -318,7 +320,7 @@ __device__ __forceinline__ void drain_plain(const GemmParams& p, int tok0, int t
 
 // EPI: 0 plain / routing-weighted bf16 store, 1 gate/up + SiLU, 2 weighted fp32 atomic accumulate (compiled apart so
 // that each instantiation carries one epilogue only).
-template <int QBITS, int BT, int EPI>
+template <int QBITS, int BT, int EPI, bool SK>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
              const __grid_constant__ CUtensorMap tm_s, const GemmParams p) {
@@ -411,7 +413,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     const int nk4 = nkb >> 2;
     int my_tiles;
     uint32_t own_kb4;            // this pair's k-blocks / 4
-    if (p.streamk) {
+    if constexpr (SK) {
         // Units of four k-blocks, U = tiles * nk4 in all; pair q owns units [U q / P, U (q + 1) / P).  Piece j of this
         // pair lies in tile t_first + j (the host keeps the number of pieces within the table).
         const long long U = static_cast<long long>(total_tiles) * nk4;
@@ -449,7 +451,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         return (j < C::TAB_N) ? tab[j] : decode_tile(pair + j * n_pairs, prefix, p, BT);
     };
     auto piece_at = [&](int j) -> Piece {
-        if (p.streamk) return ptab[j];
+        if constexpr (SK) return ptab[j];
         Piece pc;
         pc.kb0 = 0; pc.kb1 = nkb; pc.i0 = j * nkb; pc.nsrc = 0;
         return pc;
@@ -636,7 +638,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         // stage) it must have released every accumulator of an earlier tile, otherwise a single-accumulator pipeline
         // would wait for itself; at that point it has filled the ring for the next tile and would idle anyway.
         auto per_tile = [&](uint32_t t) -> uint32_t {                  // own k-blocks of the pair's t-th tile (piece)
-            if (!p.streamk) return static_cast<uint32_t>(nk4);
+            if constexpr (!SK) return static_cast<uint32_t>(nk4);
             const Piece pc = ptab[t];
             return static_cast<uint32_t>(pc.kb1 - pc.kb0) >> 2;
         };
@@ -659,7 +661,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             tc_fence_after_sync();
             if (plain_ep && wt < p.n_wt) {
                 const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
-                drain_plain(p, tl.tok0, tl.tok_end, wt * BW + q * 32,
+                drain_plain<SK>(p, tl.tok0, tl.tok_end, wt * BW + q * 32,
                             tmem_base + (static_cast<uint32_t>(q * 32) << 16) + a * BT, n_mma, 1 + g, 5, my_st, lane,
                             piece_at(static_cast<int>(jt)).nsrc, q, BT * 128, abort_flag);
             }
@@ -778,7 +780,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const int n_epi = (wt < p.n_wt) ? n_mma : 0;
             if constexpr (EPI == 0) {
                 // shared with the dequantising warps (participants 1..4 of this lane quarter) when they help
-                drain_plain(p, tl.tok0, tl.tok_end, wt * BW + qd * 32, taddr, n_epi, 0,
+                drain_plain<SK>(p, tl.tok0, tl.tok_end, wt * BW + qd * 32, taddr, n_epi, 0,
                             (C::HELP || static_cast<int>(j) == my_tiles - 1) ? 5 : 1,
                             stg16 + (16 + qd) * 512, lane, piece_at(static_cast<int>(j)).nsrc, qd, BT * 128, abort_flag);
             } else {
@@ -861,7 +863,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     if (warp == 3) tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
 }
 
-template <int QBITS, int BT, int EPI>
+template <int QBITS, int BT, int EPI, bool SK>
 static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_rows, const void* Wq, const void* Ws,
                        cudaStream_t st) {
     using C = Cfg<QBITS, BT>;
@@ -878,9 +880,10 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_ro
         rc = get_tmap_2d(ctx, &tm_s, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, Ws, p.K / 32, wrows, 8, 64,
                          CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc != QG_OK) return rc;
-    auto kern = qgemm_kernel<QBITS, BT, EPI>;
+    auto kern = qgemm_kernel<QBITS, BT, EPI, SK>;
     // the shared-memory attribute belongs to the function on one device: set once per context and instantiation
-    constexpr int inst = ((QBITS == 4) ? 9 : 0) + ((BT == 128) ? 0 : (BT == 192) ? 3 : 6) + EPI;
+    constexpr int inst = SK ? 24 + ((QBITS == 4) ? 3 : 0) + ((BT == 128) ? 0 : (BT == 192) ? 1 : 2)
+                            : ((QBITS == 4) ? 9 : 0) + ((BT == 128) ? 0 : (BT == 192) ? 3 : 6) + EPI;
     if (!ctx->attr_set[inst]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
             cudaGetLastError();
@@ -961,9 +964,10 @@ static int dispatch_gemm(qg_ctx* ctx, int qbits, int bt, const GemmParams& p_in,
     const int epi = (p.mode == QG_MODE_GATE_UP_SILU) ? 1 : (p.mode == QG_MODE_DOWN_ACCUM_F32) ? 2 : 0;
 #define QG_LAUNCH(Q, B)                                                                 \
     do {                                                                                \
-        if (epi == 0) return launch_gemm<Q, B, 0>(ctx, p, X, x_rows, Wq, Ws, st);       \
-        if (epi == 1) return launch_gemm<Q, B, 1>(ctx, p, X, x_rows, Wq, Ws, st);       \
-        return launch_gemm<Q, B, 2>(ctx, p, X, x_rows, Wq, Ws, st);                     \
+        if (epi == 0 && p.streamk) return launch_gemm<Q, B, 0, true>(ctx, p, X, x_rows, Wq, Ws, st);   \
+        if (epi == 0) return launch_gemm<Q, B, 0, false>(ctx, p, X, x_rows, Wq, Ws, st);                \
+        if (epi == 1) return launch_gemm<Q, B, 1, false>(ctx, p, X, x_rows, Wq, Ws, st);                \
+        return launch_gemm<Q, B, 2, false>(ctx, p, X, x_rows, Wq, Ws, st);                              \
     } while (0)
     if (qbits == QG_Q8) {
         if (bt == 256) QG_LAUNCH(8, 256);
