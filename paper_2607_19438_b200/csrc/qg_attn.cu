@@ -5,17 +5,20 @@
 //   O[i, h, :] = sum_j p[i, j] V[j, g, :],  p[i, :] = softmax_j(scale * Q[i, h, :] . K[j, g, :]),  g = h / (Hq / Hkv),
 //   keys j <= i only when causal.
 //
-// One CTA per (query tile of 128 rows, head).  S = Q K^T (128 x 128 per key tile) is a tcgen05.mma with both operands
-// in shared memory (K-major, 128-byte swizzle, staged by TMA straight from the caller's strided Q / K / V, e.g. the
-// output of a fused QKV projection) and its fp32 result in tensor memory; four softmax warps (one thread per query
-// row) read it, keep the running row maximum and sum, and write P = exp2(...) as bf16 over the same tensor-memory
-// columns; O += P V is a tcgen05.mma whose A operand is P in tensor memory and whose B operand is the V tile in shared
-// memory read N-major (V's head dimension is contiguous), accumulated in a third tensor-memory region.  Two S / P
-// buffers let the next tile's Q K^T run while the softmax warps work; when a row maximum grows, the same warps
-// rescale O in tensor memory before the next P V is issued.
-//   warp 0      TMA producer: Q once, then K and V tiles through two-stage rings
+// One CTA per (block of 256 query rows = two tiles A and B of 128, head).  Per key tile of 128 keys and per query
+// tile: S = Q K^T is a tcgen05.mma with both operands in shared memory (K-major, 128-byte swizzle, staged by TMA
+// straight from the caller's strided Q / K / V, e.g. the output of a fused QKV projection) and its fp32 result in
+// tensor memory; a group of four softmax warps (one thread per query row, the whole row of 128 scores in registers)
+// keeps the running row maximum and sum and writes P = exp2(...) as bf16 over the tensor-memory columns S came from;
+// O += P V is a tcgen05.mma whose A operand is P in tensor memory and whose B operand is the V tile in shared memory
+// read N-major (V's head dimension is contiguous), accumulated in the tile's own tensor-memory region.  The two
+// query tiles share every K / V tile and take turns on the tensor cores: while group A works on its scores the MMAs of
+// tile B run, and the other way round.  When a row maximum grows, the group rescales its O in tensor memory before the
+// next P V is issued.
+//   warp 0      TMA producer: both Q tiles once, then K and V tiles through two-stage rings
 //   warp 1      MMA issuer, allocates and frees tensor memory
-//   warps 2-5   softmax, O rescaling, final normalisation and store
+//   warps 2-5   softmax group A (TMEM lane quarter = warp % 4), O rescaling, final normalisation and store
+//   warps 6-9   the same for tile B
 // Every mbarrier wait is bounded; when one expires the CTA records QG_ERR_TIMEOUT and leaves.
 #include <cuda_bf16.h>
 #include <math.h>
@@ -25,7 +28,7 @@
 
 namespace qg {
 
-constexpr int AT_BQ = 128, AT_BKV = 128, AT_THREADS = 192;
+constexpr int AT_BQ = 128, AT_BKV = 128, AT_THREADS = 320;
 
 struct AttnParams {
     int S, Hq, Hkv, causal;
@@ -42,20 +45,20 @@ struct AttnCfg {
     static constexpr int NBOX = D / 64;
     static constexpr int TILE_BYTES = NBOX * BOX_BYTES;
     static constexpr int NST = 2;
-    static constexpr int OFF_Q = 0;
-    static constexpr int OFF_K = OFF_Q + TILE_BYTES;
+    static constexpr int OFF_Q = 0;                             // two query tiles
+    static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_V = OFF_K + NST * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_V + NST * TILE_BYTES;
     static constexpr int NBAR = 16;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;
-    static constexpr int COL_S = 0;                             // two S / P buffers of 128 columns
-    static constexpr int COL_O = 256;                           // O accumulator, D columns
+    static constexpr int COL_S = 0;                             // S / P of tile t at 128 t
+    static constexpr int COL_O = 256;                           // O of tile t at 256 + D t
     static constexpr int TMEM_COLS = 512;
-    static constexpr int OUT_PITCH = D * 2 + 16;                // bytes per staged output row
+    static constexpr int ROW_BYTES = D * 2;                     // staged output row (16-byte chunks XOR-swizzled by row)
     static_assert(D == 64 || D == 128, "head dimension");
-    static_assert(COL_O + D <= TMEM_COLS, "tensor memory budget");
-    static_assert(128 * OUT_PITCH <= NST * TILE_BYTES, "output staging reuses the K ring");
+    static_assert(COL_O + 2 * D <= TMEM_COLS, "tensor memory budget");
+    static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
 // Shared-memory operand descriptor for an N-major (or M-major) bf16 tile: 64 consecutive N elements are contiguous
@@ -108,22 +111,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     auto v_full = [&](int s) { return bar0 + 8u * (3 + s); };
     auto k_empty = [&](int s) { return bar0 + 8u * (5 + s); };
     auto v_empty = [&](int s) { return bar0 + 8u * (7 + s); };
-    auto s_full = [&](int b) { return bar0 + 8u * (9 + b); };
-    auto p_full = [&](int b) { return bar0 + 8u * (11 + b); };
-    const uint32_t pv_done = bar0 + 8u * 13;
+    auto s_full = [&](int t) { return bar0 + 8u * (9 + t); };      // per query tile: S(j) complete
+    auto p_full = [&](int t) { return bar0 + 8u * (11 + t); };     // P(j) written and O rescaled (4 warps arrive)
+    auto pv_done = [&](int t) { return bar0 + 8u * (13 + t); };    // P(j) V(j) complete
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_qt = (p.S + AT_BQ - 1) / AT_BQ;
-    const int qt = n_qt - 1 - static_cast<int>(blockIdx.x);     // the longest (last) query tiles start first
+    const int n_qb = (p.S + 2 * AT_BQ - 1) / (2 * AT_BQ);
+    const int qb = n_qb - 1 - static_cast<int>(blockIdx.x);     // the longest (last) query blocks start first
     const int h = blockIdx.y;
     const int g = h / (p.Hq / p.Hkv);
-    const int q0 = qt * AT_BQ;
-    // key tiles this query tile attends to
-    const int n_kv = p.causal ? (qt + 1) : (p.S + AT_BKV - 1) / AT_BKV;
+    const int q0 = qb * 2 * AT_BQ;
+    // key tiles each query tile attends to
+    const int n_all = (p.S + AT_BKV - 1) / AT_BKV;
+    const int n_a = p.causal ? min(2 * qb + 1, n_all) : n_all;
+    const int n_b = (q0 + AT_BQ < p.S) ? (p.causal ? min(2 * qb + 2, n_all) : n_all) : 0;
+    const int n_loop = max(n_a, n_b);
 
     pdl_launch_dependents();
     if (warp == 0) {
-        if (lane < 14) {
+        if (lane < 15) {
             const uint32_t cnt = (lane == 11 || lane == 12) ? 4u : 1u;      // p_full: one arrival per softmax warp
             mbar_init(bar0 + 8u * lane, cnt);
         }
@@ -148,12 +154,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // ------------------------------------------------ TMA producer
         bool ok = true;
         if (lane == 0) {
-            mbar_arrive_expect_tx(q_full, C::TILE_BYTES);
+            mbar_arrive_expect_tx(q_full, 2 * C::TILE_BYTES);       // rows past the sequence end arrive as zeros
 #pragma unroll
-            for (int a = 0; a < C::NBOX; ++a)
-                tma_load_2d(sbase + C::OFF_Q + a * C::BOX_BYTES, &tm_q, h * D + 64 * a, q0, q_full);
+            for (int t = 0; t < 2; ++t)
+#pragma unroll
+                for (int a = 0; a < C::NBOX; ++a)
+                    tma_load_2d(sbase + C::OFF_Q + t * C::TILE_BYTES + a * C::BOX_BYTES, &tm_q, h * D + 64 * a,
+                                q0 + t * AT_BQ, q_full);
         }
-        for (int j = 0; j < n_kv && ok; ++j) {
+        for (int j = 0; j < n_loop && ok; ++j) {
             const int s = j & 1;
             const uint32_t ph = (j >> 1) & 1u;
             if (!at_wait(k_empty(s), ph ^ 1u, abort_flag, p)) { ok = false; break; }
@@ -176,168 +185,172 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
-        // Order of issue: S(0); then for every key tile j: S(j + 1) (so that it runs while the softmax warps work on
-        // S(j)), P(j) V(j).  MMAs of one thread execute in order, so S(j + 1), which overwrites the buffer that held
-        // P(j - 1), cannot overtake P(j - 1) V(j - 1).
+        // Order of issue: S_A(0), S_B(0); then for every key tile j: P_A(j) V(j), S_A(j + 1), P_B(j) V(j), S_B(j + 1).
+        // MMAs of one thread execute in order, so S_t(j + 1), which overwrites the columns that held P_t(j), cannot
+        // overtake P_t(j) V(j); while the softmax group of one tile works, the MMAs of the other tile run.
         const uint32_t idesc_s = umma_idesc_bf16_major(AT_BQ, AT_BKV, 0u);
         const uint32_t idesc_o = umma_idesc_bf16_major(AT_BQ, D, 1u);
-        const uint32_t q_addr = sbase + C::OFF_Q;
         bool ok = at_wait(q_full, 0u, abort_flag, p);
-        auto issue_s = [&](int j) -> bool {
+        auto issue_s = [&](int t, int j, bool last_on_k) -> bool {      // S_t(j) = Q_t K(j)^T
             const int s = j & 1;
             if (!at_wait(k_full(s), (j >> 1) & 1u, abort_flag, p)) return false;
             tc_fence_after_sync();
             if (lane == 0) {
+                const uint32_t q_addr = sbase + C::OFF_Q + t * C::TILE_BYTES;
                 const uint32_t k_addr = sbase + C::OFF_K + s * C::TILE_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * C::BOX_BYTES + (kk & 3) * 32;
-                    umma_f16_ss(tmem_base + C::COL_S + s * 128, umma_desc_k_sw128(q_addr + off),
+                    umma_f16_ss(tmem_base + C::COL_S + t * 128, umma_desc_k_sw128(q_addr + off),
                                 umma_desc_k_sw128(k_addr + off), idesc_s, kk ? 1u : 0u);
                 }
-                umma_commit(s_full(s));
-                umma_commit(k_empty(s));
+                umma_commit(s_full(t));
+                if (last_on_k) umma_commit(k_empty(s));
             }
             __syncwarp();
             return true;
         };
-        if (ok && n_kv > 0) ok = issue_s(0);
-        for (int j = 0; j < n_kv && ok; ++j) {
+        auto issue_pv = [&](int t, int j, bool last_on_v) -> bool {     // O_t += P_t(j) V(j)
             const int s = j & 1;
-            const uint32_t ph = (j >> 1) & 1u;
-            if (j + 1 < n_kv && !issue_s(j + 1)) { ok = false; break; }
-            if (!at_wait(p_full(s), ph, abort_flag, p) || !at_wait(v_full(s), ph, abort_flag, p)) { ok = false; break; }
+            if (!at_wait(p_full(t), j & 1u, abort_flag, p) || !at_wait(v_full(s), (j >> 1) & 1u, abort_flag, p)) return false;
             tc_fence_after_sync();
             if (lane == 0) {
                 const uint32_t v_addr = sbase + C::OFF_V + s * C::TILE_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < AT_BKV / 16; ++kk)          // 16 keys per instruction: two 8-key groups of V
-                    umma_f16_ts(tmem_base + C::COL_O, tmem_base + C::COL_S + s * 128 + 8 * kk,
+                    umma_f16_ts(tmem_base + C::COL_O + t * D, tmem_base + C::COL_S + t * 128 + 8 * kk,
                                 umma_desc_mn_sw128(v_addr + kk * 2048, C::BOX_BYTES), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(pv_done);
-                umma_commit(v_empty(s));
+                umma_commit(pv_done(t));
+                if (last_on_v) umma_commit(v_empty(s));
             }
             __syncwarp();
+            return true;
+        };
+        if (ok && n_a > 0) ok = issue_s(0, 0, n_b == 0);
+        if (ok && n_b > 0) ok = issue_s(1, 0, true);
+        for (int j = 0; j < n_loop && ok; ++j) {
+            if (j < n_a && !issue_pv(0, j, !(j < n_b))) { ok = false; break; }
+            if (j + 1 < n_a && !issue_s(0, j + 1, !(j + 1 < n_b))) { ok = false; break; }
+            if (j < n_b && !issue_pv(1, j, true)) { ok = false; break; }
+            if (j + 1 < n_b && !issue_s(1, j + 1, true)) { ok = false; break; }
         }
     } else {
-        // ------------------------------------------------ softmax (thread = one query row)
+        // ------------------------------------------------ softmax groups (thread = one query row)
+        const int t = (warp >= 6) ? 1 : 0;                             // query tile of this group
+        const int n_t = t ? n_b : n_a;
         const int quarter = warp & 3;                                  // TMEM lanes 32 quarter .. + 31
         const int row = quarter * 32 + lane;
-        const int qi = q0 + row;                                       // query position of this thread
+        const int qi = q0 + t * AT_BQ + row;                           // query position of this thread
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        const uint32_t s_addr = lane_addr + C::COL_S + t * 128;
+        const uint32_t o_addr = lane_addr + C::COL_O + t * D;
         const float cl = p.scale_log2;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int j = 0; j < n_kv && ok; ++j) {
-            const int b = j & 1;
-            const uint32_t ph = (j >> 1) & 1u;
-            if (!at_wait(s_full(b), ph, abort_flag, p)) { ok = false; break; }
+        for (int j = 0; j < n_t && ok; ++j) {
+            if (!at_wait(s_full(t), j & 1u, abort_flag, p)) { ok = false; break; }
             tc_fence_after_sync();
-            const uint32_t s_addr = lane_addr + C::COL_S + b * 128;
+            uint32_t v[128];                                           // the row's scores against this key tile
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld_32x32(s_addr + 32 * c, *reinterpret_cast<uint32_t (*)[32]>(v + 32 * c));
+            tmem_ld_wait();
             const int key0 = j * AT_BKV;
             // keys this row may see in the tile: below `lim` (all 128 except on the diagonal and at the sequence end)
             int lim = p.S - key0;
             if (p.causal) lim = min(lim, qi - key0 + 1);
-            const bool masked = (__any_sync(0xFFFFFFFFu, lim < AT_BKV) != 0);
-            float mx = -INFINITY;
+            if (__any_sync(0xFFFFFFFFu, lim < AT_BKV)) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld_32x32(s_addr + 32 * c, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float x = __uint_as_float(v[i]);
-                    if (masked && 32 * c + i >= lim) x = -INFINITY;
-                    mx = fmaxf(mx, x);
-                }
+                for (int i = 0; i < 128; ++i)
+                    if (i >= lim) v[i] = 0xFF800000u;                  // -inf
             }
-            const float m_new = fmaxf(m, mx);
-            // rows past the sequence end see no key at all in a masked tile: keep their arithmetic finite
-            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 128; i += 4) {
+                mx0 = fmaxf(mx0, __uint_as_float(v[i]));
+                mx1 = fmaxf(mx1, __uint_as_float(v[i + 1]));
+                mx2 = fmaxf(mx2, __uint_as_float(v[i + 2]));
+                mx3 = fmaxf(mx3, __uint_as_float(v[i + 3]));
+            }
+            const float m_new = fmaxf(m, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)));
+            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // keeps a row without any visible key finite
             const float mc = m_use * cl;
-            float sum = 0.f;
+            float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld_32x32(s_addr + 32 * c, v);
-                tmem_ld_wait();
-                uint32_t pk[16];
+            for (int c = 0; c < 8; ++c) {                              // 16 scores -> 8 columns of packed bf16 pairs
+                uint32_t pk[8];
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float x0 = __uint_as_float(v[i]), x1 = __uint_as_float(v[i + 1]);
-                    float p0 = fast_exp2(fmaf(x0, cl, -mc)), p1 = fast_exp2(fmaf(x1, cl, -mc));
-                    if (masked && 32 * c + i >= lim) p0 = 0.f;
-                    if (masked && 32 * c + i + 1 >= lim) p1 = 0.f;
-                    // the sum runs over the bf16 values the tensor cores will multiply, so that numerator and
-                    // denominator of the softmax stay consistent
+                for (int i = 0; i < 16; i += 2) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(v[16 * c + i]), cl, -mc));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(v[16 * c + i + 1]), cl, -mc));
+                    s0 += p0;
+                    s1 += p1;
                     const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-                    sum += __low2float(pb) + __high2float(pb);
                     pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
                 }
-                tmem_st_32x32_x16(s_addr + 16 * c, pk);          // P over the columns of S already read
+                tmem_st_32x32_x8(s_addr + 8 * c, pk);                 // P over the columns S came from
             }
-            const float alpha = fast_exp2((m - m_use) * cl);      // exp2(-inf) = 0 on the first tile
-            l = l * alpha + sum;
+            const float alpha = fast_exp2((m - m_use) * cl);          // exp2(-inf) = 0 on the first tile
+            l = l * alpha + (s0 + s1);
             m = m_use;
             if (j > 0) {
                 // O of the earlier tiles is rescaled once their last P V has completed
-                if (!at_wait(pv_done, (j - 1) & 1u, abort_flag, p)) { ok = false; break; }
+                if (!at_wait(pv_done(t), (j - 1) & 1u, abort_flag, p)) { ok = false; break; }
                 tc_fence_after_sync();
                 if (!__all_sync(0xFFFFFFFFu, alpha == 1.0f)) {
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
-                        uint32_t v[32];
-                        tmem_ld_32x32(lane_addr + C::COL_O + 32 * c, v);
+                        uint32_t o[32];
+                        tmem_ld_32x32(o_addr + 32 * c, o);
                         tmem_ld_wait();
-                        uint32_t (&lo)[16] = *reinterpret_cast<uint32_t (*)[16]>(v);
-                        uint32_t (&hi)[16] = *reinterpret_cast<uint32_t (*)[16]>(v + 16);
+                        uint32_t (&lo)[16] = *reinterpret_cast<uint32_t (*)[16]>(o);
+                        uint32_t (&hi)[16] = *reinterpret_cast<uint32_t (*)[16]>(o + 16);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                        tmem_st_32x32_x16(lane_addr + C::COL_O + 32 * c, lo);
-                        tmem_st_32x32_x16(lane_addr + C::COL_O + 32 * c + 16, hi);
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st_32x32_x16(o_addr + 32 * c, lo);
+                        tmem_st_32x32_x16(o_addr + 32 * c + 16, hi);
                     }
                 }
             }
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_full(b));
+            if (lane == 0) mbar_arrive(p_full(t));
         }
-        // ---- normalise and store: through a padded staging tile in the (now idle) K ring, then 16-byte rows
-        const bool good = ok && n_kv > 0 && at_wait(pv_done, (n_kv - 1) & 1u, abort_flag, p);
-        uint8_t* stage = sgen + C::OFF_K;
+        // ---- normalise and store: through this tile's (now idle) Q buffer, 16-byte chunks XOR-swizzled by the row
+        const bool good = ok && n_t > 0 && at_wait(pv_done(t), (n_t - 1) & 1u, abort_flag, p);
+        uint8_t* stage = sgen + C::OFF_Q + t * C::TILE_BYTES;
         if (good) {
             tc_fence_after_sync();
             const float inv = (l > 0.f) ? 1.0f / l : 0.f;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld_32x32(lane_addr + C::COL_O + 32 * c, v);
+                uint32_t o[32];
+                tmem_ld_32x32(o_addr + 32 * c, o);
                 tmem_ld_wait();
-                uint4* dst = reinterpret_cast<uint4*>(stage + row * C::OUT_PITCH + c * 64);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     uint32_t w[4];
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(v[8 * i + 2 * t]) * inv,
-                                                                        __uint_as_float(v[8 * i + 2 * t + 1]) * inv);
-                        w[t] = *reinterpret_cast<const uint32_t*>(&o2);
+                    for (int u = 0; u < 4; ++u) {
+                        const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 2 * u]) * inv,
+                                                                        __uint_as_float(o[8 * i + 2 * u + 1]) * inv);
+                        w[u] = *reinterpret_cast<const uint32_t*>(&o2);
                     }
-                    dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4*>(stage + row * C::ROW_BYTES + (((4 * c + i) ^ (row & 7)) << 4)) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
         }
-        named_bar_sync(1, 128);            // reached by all four warps whatever happened above (every wait is bounded)
+        named_bar_sync(1 + t, 128);        // reached by all four warps of the group whatever happened above
         if (good) {
-            const int t = threadIdx.x - 64;
+            const int tid = (warp - 2 - 4 * t) * 32 + lane;
             constexpr int VPR = D / 8;                              // 16-byte vectors per row
-            for (int idx = t; idx < AT_BQ * VPR; idx += 128) {
+            for (int idx = tid; idx < AT_BQ * VPR; idx += 128) {
                 const int r = idx / VPR, vv = idx - r * VPR;
-                if (q0 + r < p.S)
-                    *reinterpret_cast<uint4*>(p.O + static_cast<size_t>(q0 + r) * p.ldo + static_cast<size_t>(h) * D + vv * 8) =
-                        *reinterpret_cast<const uint4*>(stage + r * C::OUT_PITCH + vv * 16);
+                const int qr = q0 + t * AT_BQ + r;
+                if (qr < p.S)
+                    *reinterpret_cast<uint4*>(p.O + static_cast<size_t>(qr) * p.ldo + static_cast<size_t>(h) * D + vv * 8) =
+                        *reinterpret_cast<const uint4*>(stage + r * C::ROW_BYTES + ((vv ^ (r & 7)) << 4));
             }
         }
     }
@@ -375,8 +388,8 @@ static int launch_attn(qg_ctx* ctx, const AttnParams& p, const void* Q, long lon
         }
         ctx->attr_set[inst] = true;
     }
-    const int n_qt = (p.S + AT_BQ - 1) / AT_BQ;
-    if (launch_kernel(ctx, kern, dim3(n_qt, p.Hq), dim3(AT_THREADS), C::SMEM_BYTES, st, *tm_q, *tm_k, *tm_v, p) != cudaSuccess) {
+    const int n_qb = (p.S + 2 * AT_BQ - 1) / (2 * AT_BQ);
+    if (launch_kernel(ctx, kern, dim3(n_qb, p.Hq), dim3(AT_THREADS), C::SMEM_BYTES, st, *tm_q, *tm_k, *tm_v, p) != cudaSuccess) {
         cudaGetLastError();
         return QG_ERR_CUDA;
     }
