@@ -548,6 +548,14 @@ def run_ours(args):
     # second repeats it with an event pair around every call for the per-kernel figures and the roofline (sixteen
     # extra stream operations per step cost a few per cent, so they stay out of the headline).
     ms = timed(lambda: step(dA, dL, dX), args.steps)
+    if args.profile_run:
+        qg.poll_status()
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "steps": args.steps, "ms_per_step": ms / args.steps,
+                              "launches_per_step": LAUNCHES_PER_STEP, "moe_path": args.moe_path}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     ev_steps = max(1, min(args.steps, 100))
     torch.cuda.synchronize()
     time.sleep(1.0)     # let the board's power average settle: a sustained run is clocked down under the power cap
@@ -725,6 +733,26 @@ def run_case(args):
     dev = torch.device("cuda", 0)
     lib, ctx = qg.load(), qg.context(0)
     g = torch.Generator(device=dev); g.manual_seed(0)
+    if args.case == "attention":
+        S, Hq, Hkv, d = 2048, 32, 8, 128
+        qkv = torch.randn((S, (Hq + 2 * Hkv) * d), device=dev, generator=g).to(torch.bfloat16)
+        for _ in range(3):
+            qg.prefill_attention(qkv[:, :Hq * d], qkv[:, Hq * d:(Hq + Hkv) * d], qkv[:, (Hq + Hkv) * d:], Hq, Hkv, d)
+        qg.poll_status()
+        print(json.dumps({"case": args.case, "S": S, "Hq": Hq, "Hkv": Hkv, "d": d, "passes": 3}))
+        return
+    if args.case == "small_m":
+        M, N, K = 4, 28672, 4096
+        Wq = torch.randint(-127, 128, (N, K), dtype=torch.int8, device=dev, generator=g)
+        Ws = (torch.randn((N, K // 32), device=dev, generator=g).abs() * (0.02 / 127)).to(torch.float16)
+        A = torch.randn((M, K), device=dev, generator=g).to(torch.bfloat16)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            flush.zero_()
+            qg.qgemm_small_m(8, A, Wq, Ws)
+        qg.poll_status()
+        print(json.dumps({"case": args.case, "M": M, "N": N, "K": K, "passes": 3}))
+        return
     H, F, k = MOE["H"], MOE["F"], MOE["k"]
     E, M = 16, 256
     R = M * k
@@ -751,12 +779,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-sweep", action="store_true", help="skip the per-configuration sweep block")
+    ap.add_argument("--profile-run", action="store_true",
+                    help="warm-up and the timed steps only (no per-call region, sustained run, end-to-end leg, sweep or CPU "
+                         "baseline): a short target for profiler launch lists; prints a reduced JSON line")
     ap.add_argument("--moe-path", default="staged", choices=["fused", "staged"],
                     help="staged: permute, routing-weighted bf16 rows, slot-ordered combine (deterministic, faster on "
                          "B200); fused: token gather in the gate/up loads + fp32 accumulate in the down epilogue")
-    ap.add_argument("--case", default=None, choices=["moe_small"],
+    ap.add_argument("--case", default=None, choices=["moe_small", "attention", "small_m"],
                     help="run one small case a few times and exit (for profiler captures): moe_small = the cfg-3 MoE "
-                         "layer shape with 16 experts and 256 tokens (128 rows per expert)")
+                         "layer shape with 16 experts and 256 tokens (128 rows per expert); attention = cfg-4 heads "
+                         "(32 / 8, d = 128) at 2048 positions; small_m = the cfg-4 gate/up weights (28672 x 4096, Q8) "
+                         "times 4 tokens")
     args = ap.parse_args()
     if args.case:
         run_case(args)
