@@ -113,6 +113,11 @@ int qg_set_schedule(qg_ctx* ctx, int token_tile, int streamk_mode) {
     return QG_OK;
 }
 
+#ifdef QG_PROFILE
+// profiling builds only: device buffer for the GEMM kernel's cycle counters and milestones
+void qg_debug_set_stats(qg_ctx* ctx, long long* dev_buf) { if (ctx) ctx->stats = dev_buf; }
+#endif
+
 int qg_test_inject(qg_ctx* ctx, unsigned wait_limit_polls, int skip_kblock) {
     if (!ctx) return QG_ERR_NULL;
     ctx->wait_limit = wait_limit_polls ? wait_limit_polls : qg::DEFAULT_WAIT_LIMIT;

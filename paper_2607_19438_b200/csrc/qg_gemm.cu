@@ -355,13 +355,14 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     // offsets, routing tables) or may still read (the output buffer) is touched only after pdl_wait().  The weights
     // are constants of the model, so in the dense case their producer and the dequantising warps start at once.
     pdl_launch_dependents();
+    if (warp == 0) { QG_MARK(0); }
+    QG_SPAN(0);
     const bool grouped = (p.offsets != nullptr);
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     volatile int* abort_flag = misc + 1;
 
     if (warp == 0) {   // barrier initialisation spread over the lanes of one warp (a single thread needs ~50 steps)
         if (lane < C::SX) { mbar_init(full(lane), 1 + 8); mbar_init(done(lane), 1); }
-        if (lane < C::SR) { mbar_init(r_full(lane), 1); mbar_init(r_empty(lane), 4); }
         // an accumulator is released by the 4 epilogue + 16 dequantising warps of both CTAs
         if (lane >= 16 && lane < 18) { mbar_init(acc_full(lane - 16), 2); mbar_init(acc_empty(lane - 16), C::HELP ? 40 : 8); }
         if (lane == 31) { misc[1] = 0; mbar_init(last_full, 1); }
@@ -376,7 +377,14 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         tmem_relinquish_pair();
     }
     const int n_pw = (p.n_wt + 1) >> 1;
+    // The packed-weight ring is private to this CTA and to warp 2, its producer: that warp initialises the ring's
+    // barriers itself and, as soon as it knows the pair's first tile, sends the first four k-blocks of weights on
+    // their way, so that they travel while the pair synchronises and the tile tables are built.
+    bool w_pre_issued = false;
     if (warp == 2) {  // prefix[e] = pair tiles before expert e; prefix[E] = total
+        if (lane < C::SR) { mbar_init(r_full(lane), 1); mbar_init(r_empty(lane), 4); }
+        fence_mbar_init();
+        fence_proxy_async_smem();
         if (grouped) pdl_wait();
         int carry = 0;
         for (int e0 = 0; e0 < p.E; e0 += 32) {
@@ -396,6 +404,28 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             carry += __shfl_sync(0xFFFFFFFFu, inc, 31);
         }
         if (lane == 0) prefix[p.E] = carry;
+        __syncwarp();
+        if (!SK && pair < carry) {
+            const Tile tl = decode_tile(pair, prefix, p, BT);
+            const int wt = 2 * tl.pw + static_cast<int>(rank);
+            const int row_a = tl.e * p.N + wt * ((EPI == 1) ? 64 : 128);
+            const int row_b = row_a + ((EPI == 1) ? (p.N / 2) : 64);
+            if (lane == 0) {
+                const uint32_t sd = sbase + C::OFF_SC;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    mbar_arrive_expect_tx(r_full(j), C::RAW_BYTES + (j == 0 ? C::SC_BYTES : 0));
+                    const uint32_t dst = sbase + C::OFF_RAW + j * C::RAW_BYTES;
+                    tma_load_2d(dst, &tm_w, j * C::RAW_ROW, row_a, r_full(j));
+                    tma_load_2d(dst + C::RAW_BYTES / 2, &tm_w, j * C::RAW_ROW, row_b, r_full(j));
+                    if (j == 0) {
+                        tma_load_2d(sd, &tm_s, 0, row_a, r_full(0));
+                        tma_load_2d(sd + C::SC_BYTES / 2, &tm_s, 0, row_b, r_full(0));
+                    }
+                }
+            }
+            w_pre_issued = true;
+        }
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -447,6 +477,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             tab[j] = decode_tile(pair + j * n_pairs, prefix, p, BT);
     }
     __syncthreads();
+    if (warp == 0) { QG_MARK(1); }
     auto tile_at = [&](int j) -> Tile {
         return (j < C::TAB_N) ? tab[j] : decode_tile(pair + j * n_pairs, prefix, p, BT);
     };
@@ -465,6 +496,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     if (warp == 0) {
         // ------------------------------------------------ activation producer (this CTA's half of the token tile)
         uint32_t s = 0, ph = 0;      // first stage of the next batch (0, 2, 4, 6) and the parity of its next "done" phase
+        uint32_t sent_kb = 0;        // k-blocks sent so far: the first eight find the ring empty and need no wait
         const uint32_t full_leader = map_to_cta(full(0), 0);
         bool ok = true;
         QG_DECL();
@@ -488,9 +520,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 QG_T0();
                 // a stage is free once the MMAs that read it eight k-blocks ago are done (even and odd stages
                 // belong to different MMA warps, so both are checked)
-                if (!wait_bar<false>(done(s), ph ^ 1u, abort_flag, p) ||
-                    !wait_bar<false>(done(s + 1), ph ^ 1u, abort_flag, p)) { ok = false; break; }
+                if (sent_kb >= 8u &&
+                    (!wait_bar<false>(done(s), ph ^ 1u, abort_flag, p) ||
+                     !wait_bar<false>(done(s + 1), ph ^ 1u, abort_flag, p))) { ok = false; break; }
+                sent_kb += 2u;
                 QG_ACC(0);
+                if (jt == 0 && kb == pc.kb0) { QG_MARK(7); }
                 if (p.gather_k > 0) {
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
@@ -519,6 +554,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     } else if (warp == 2) {
         // ------------------------------------------------ packed weight + scale producer (local ring)
         uint32_t s = 0, ph = 0, sg = 0;     // first raw stage of the batch (0 or 4), parity, scale buffer
+        uint32_t batches = 0;               // batches sent so far: the first SR / 4 find the ring empty and need no wait
         bool ok = true;
         QG_DECL();
         for (int jt = 0; jt < my_tiles && ok; ++jt) {
@@ -529,12 +565,17 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const int row_b = row_a + (gate_up ? (p.N / 2) : 64);
             for (int kb = pc.kb0; kb < pc.kb1; kb += 4) {
                 QG_T0();
+                if (batches >= C::SR / 4) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (ok && !wait_bar<false>(r_empty(s + j), ph ^ 1u, abort_flag, p)) ok = false;
-                if (!ok) break;
+                    for (int j = 0; j < 4; ++j)
+                        if (ok && !wait_bar<false>(r_empty(s + j), ph ^ 1u, abort_flag, p)) ok = false;
+                    if (!ok) break;
+                }
                 QG_ACC(1);
-                if (lane == 0) {
+                if (jt == 0 && kb == pc.kb0) { QG_MARK(8); }
+                const bool sent = (batches == 0 && w_pre_issued);       // the first batch left in the prologue
+                ++batches;
+                if (lane == 0 && !sent) {
                     const uint32_t sd = sbase + C::OFF_SC + sg * C::SC_BYTES;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -598,6 +639,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                     QG_T0();
                     if (!ready && !spin_wait_bar(full(st), (i >> 3) & 1u, abort_flag, p)) { ok = false; break; }
                     QG_ACC(3);
+                    if (w == 0 && j == 0 && kb == pc.kb0) { QG_MARK(2); }
                     tc_fence_after_sync();
                     // start the wait for this warp's next k-block before issuing, so its latency is hidden
                     const uint32_t in = i + 2u;
@@ -614,6 +656,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 }
                 if (ok && lane == 0) umma_commit_pair(acc_full(a));
                 __syncwarp();
+                if (w == 0 && static_cast<int>(j) == my_tiles - 1) { QG_MARK(3); }
             }
             __syncwarp();
             if (lane == 0 && w == 0) QG_FLUSH();
@@ -687,6 +730,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             if (!wait_bar<false>(r_full((n % NB) << 2), phr, abort_flag, p)) break;
             if (!wait_bar<false>(r_full(sr), phr, abort_flag, p)) break;
             QG_ACC(5);
+            if (n == 0 && warp == 8) { QG_MARK(10); }
             const uint32_t raw = sbase + C::OFF_RAW + sr * C::RAW_BYTES + raw_row;
             const uint32_t scw = *reinterpret_cast<const uint32_t*>(
                 sgen + C::OFF_SC + (n % C::NSB) * C::SC_BYTES + row * 16 + g * 4);
@@ -742,6 +786,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(full_leader + 8u * (((n & 1u) << 2) + g));   // k-block stage i % 8
+            if (n == 0 && warp == 8) { QG_MARK(9); }
             ta += 4;
             if (ta >= C::SA) ta -= C::SA;
             QG_ACC(7);
@@ -775,6 +820,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             tc_fence_after_sync();
             if (!C::HELP && et == 0 && static_cast<int>(j) == my_tiles - 1) mbar_arrive(last_full);
             QG_ACC(8);
+            if (qd == 0 && static_cast<int>(j) == my_tiles - 1) { QG_MARK(4); }
             const int n_mma = min(BT, (tl.tok_end - tl.tok0 + 15) & ~15);
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(qd * 32) << 16) + a * BT;
             const int n_epi = (wt < p.n_wt) ? n_mma : 0;
@@ -847,12 +893,14 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(acc_empty_base + 8u * a);
             QG_ACC(9);
+            if (qd == 0 && static_cast<int>(j) == my_tiles - 1) { QG_MARK(5); }
         }
         if (et == 0) QG_FLUSH();
     }
 
     // ---------------------------------------------------- teardown
     __syncthreads();
+    if (warp == 0) { QG_MARK(6); }
     if (*abort_flag) {
         // copies may still be in flight towards this CTA's shared memory: give them time to land
         for (int i = 0; i < 64; ++i) __nanosleep(2000);
@@ -861,6 +909,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     cluster_sync_all();          // the peer no longer reads this CTA's shared memory or signals its barriers
     tc_fence_after_sync();
     if (warp == 3) tmem_dealloc_pair(tmem_base, C::TMEM_COLS);
+    QG_SPAN(1);
 }
 
 template <int QBITS, int BT, int EPI, bool SK>
