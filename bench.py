@@ -409,6 +409,9 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
                "call_us": {lab: v[0] / n_it * 1e3 for lab, v in agg.items()},
                "gemms_tflops": gemm_fl / (gemm_ms * 1e-3) / 1e12, "layer_tok_per_s": M * n_it / (tot_ms * 1e-3),
                "hbm_gbs": {lab: agg[lab][2] * n_it / (agg[lab][0] * 1e-3) / 1e9 for lab in ("route_permute", "combine")},
+               "hbm_gbs_note": "algorithmic bytes over the time of the call repeated back to back; up to M = 2048 the rows it "
+                               "reads (64 MB) stay in the 126 MB L2 between repetitions, so the figure can exceed the HBM "
+                               "peak; inside a layer pass the same calls take the times of the headline's `kernels` block",
                "composite_bound_us": max(t_tensor, t_hbm) * 1e6,
                "bound": "hbm (expert weights)" if t_hbm > t_tensor else "tensor"}
         row["frac_of_measured_peak"] = row["gemms_tflops"] / peak_tf
