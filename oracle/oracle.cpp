@@ -22,6 +22,12 @@
 //   expert GEMM the dense definition applied per expert segment   (Sec. 3.1 "MoE expert GEMM")
 //   gate/up     H = silu(G) * U with silu(g) = g / (1 + exp(-g))  (Sec. 3.1 "Fused MoE gate/up")
 //   combine     y[t] = sum over slots s (ascending) of w[t][s] * D[row of (t, s)]
+//   MX formats  (block-scaled operands native to the tensor cores of the target GPU; not in the paper, whose
+//               kernels keep the checkpoint's own quantisation): element codes are OCP FP8 E4M3 (1-4-3, bias 7,
+//               largest finite 448, no infinity), one power-of-two scale byte (E8M0: 2^(b - 127)) per 32
+//               consecutive k.  quantise: e = floor(log2(max|x| of the block)) - 8, elements = x / 2^e rounded to
+//               the nearest E4M3 value (ties to the even code), magnitudes above 448 clamped to 448.
+//               product: C[m][n] = sum_k (a[m][k] 2^ea[m][k/32]) (w[n][k] 2^ew[n][k/32]).
 //   attention   O[i, h] = sum_j softmax_j(scale * q[i, h] . k[j, g(h)]) v[j, g(h)], j <= i if causal,
 //               g(h) = h / (Hq / Hkv)                           (Sec. 3.1 "Prefill attention": the
 //               paper only requires the tensor path to equal the plain softmax(Q K^T) V)
@@ -247,6 +253,75 @@ void orc_combine(int64_t M, int k, int64_t H, const double* D, const int32_t* pa
             }
             y[t * H + c] = acc;
         }
+}
+
+// ---- MX (block-scaled FP8) reference ------------------------------------------------------------------------------
+// Value of an E4M3 code: sign, 4 exponent bits (bias 7), 3 mantissa bits; exponent 0 is subnormal (m / 8 * 2^-6);
+// exponent 15 with mantissa 7 is NaN, every other code is finite (so 0x7E = 448 is the largest).
+double e4m3_value(uint8_t c) {
+    const int sign = c >> 7, expo = (c >> 3) & 0xF, man = c & 7;
+    double v;
+    if (expo == 0) v = std::ldexp(static_cast<double>(man), -9);
+    else if (expo == 15 && man == 7) v = std::nan("");
+    else v = std::ldexp(static_cast<double>(8 + man), expo - 10);
+    return sign ? -v : v;
+}
+
+void orc_e4m3_to_f64(int64_t n, const uint8_t* in, double* out) {
+    for (int64_t i = 0; i < n; ++i) out[i] = e4m3_value(in[i]);
+}
+
+// Nearest E4M3 code of x by search over all finite codes of x's sign: smallest distance, ties to the code with an even
+// mantissa bit; |x| > 448 gives 448.  (Brute force on purpose.)
+uint8_t e4m3_nearest(double x) {
+    const uint8_t sign = std::signbit(x) ? 0x80 : 0x00;
+    const double ax = std::fabs(x);
+    int best = 0;
+    double best_d = INFINITY;
+    for (int c = 0; c <= 0x7E; ++c) {
+        const double d = std::fabs(e4m3_value(static_cast<uint8_t>(c)) - ax);
+        if (d < best_d || (d == best_d && (c & 1) == 0 && (best & 1) == 1)) { best_d = d; best = c; }
+    }
+    return static_cast<uint8_t>(sign | best);
+}
+
+// x fp64 [rows, K] -> codes [rows, K], scale bytes [rows, K/32] (plain row-major; the GPU library stores them in
+// 512-byte tiles, a pure permutation handled by the test harness).
+void orc_mx_quantize(int64_t rows, int64_t K, const double* x, uint8_t* codes, uint8_t* sf) {
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < K / 32; ++b) {
+            const double* xb = x + r * K + b * 32;
+            double amax = 0.0;
+            for (int i = 0; i < 32; ++i) amax = std::fmax(amax, std::fabs(xb[i]));
+            int e = -127;
+            if (amax > 0.0) {
+                int ex;
+                std::frexp(amax, &ex);              // amax = f * 2^ex, f in [0.5, 1): floor(log2(amax)) = ex - 1
+                e = ex - 1 - 8;
+                if (e < -127) e = -127;
+                if (e > 127) e = 127;
+            }
+            sf[r * (K / 32) + b] = static_cast<uint8_t>(e + 127);
+            for (int i = 0; i < 32; ++i) codes[r * K + b * 32 + i] = e4m3_nearest(std::ldexp(xb[i], -e));
+        }
+    }
+}
+
+void orc_mx_gemm(int64_t M, int64_t N, int64_t K, const uint8_t* a, const uint8_t* asf, const uint8_t* w,
+                 const uint8_t* wsf, double* C) {
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                const double av = std::ldexp(e4m3_value(a[m * K + k]), static_cast<int>(asf[m * (K / 32) + k / 32]) - 127);
+                const double wv = std::ldexp(e4m3_value(w[n * K + k]), static_cast<int>(wsf[n * (K / 32) + k / 32]) - 127);
+                acc += av * wv;
+            }
+            C[m * N + n] = acc;
+        }
+    }
 }
 
 // Scaled-dot-product attention for one sequence, plain definition.  Q [S, Hq, d], K and V [S, Hkv, d] as bf16 bits with

@@ -199,3 +199,31 @@ def attention(Q, K, V, Hq, Hkv, d, causal=True, scale=None, qpos=None):
                         C.c_int64(K.strides[0] // 2), _p(V), C.c_int64(V.strides[0] // 2), C.c_double(scale),
                         C.c_int(1 if causal else 0), C.c_int64(qpos.size), _p(qpos), _p(out))
     return out
+
+
+def e4m3_to_f64(codes):
+    c = _c(codes, np.uint8)
+    out = np.empty(c.shape, np.float64)
+    lib().orc_e4m3_to_f64(C.c_int64(c.size), _p(c), _p(out))
+    return out
+
+
+def mx_quantize(x):
+    """x fp64 [rows, K] -> (E4M3 codes uint8 [rows, K], E8M0 scale bytes uint8 [rows, K/32]); blocks of 32 along K."""
+    x = _c(x, np.float64)
+    rows, K = x.shape
+    assert K % 32 == 0
+    codes = np.empty((rows, K), np.uint8)
+    sf = np.empty((rows, K // 32), np.uint8)
+    lib().orc_mx_quantize(C.c_int64(rows), C.c_int64(K), _p(x), _p(codes), _p(sf))
+    return codes, sf
+
+
+def mx_gemm(a, asf, w, wsf):
+    """C[m, n] = sum_k (a[m,k] 2^(asf[m,k/32]-127)) (w[n,k] 2^(wsf[n,k/32]-127)), fp64; scale bytes in plain layout."""
+    a, asf, w, wsf = _c(a, np.uint8), _c(asf, np.uint8), _c(w, np.uint8), _c(wsf, np.uint8)
+    M, K = a.shape
+    N = w.shape[0]
+    out = np.empty((M, N), np.float64)
+    lib().orc_mx_gemm(C.c_int64(M), C.c_int64(N), C.c_int64(K), _p(a), _p(asf), _p(w), _p(wsf), _p(out))
+    return out

@@ -137,3 +137,24 @@ def moe_problem(qbits: int, M: int, H: int, E: int, F: int, seed: int = 0, skewe
     W2q = gen(E * H, F, seed, TID_W2Q).reshape(E, H, -1)
     W2s = scales(E * H, F // 32, qmax, seed, TID_W2S).reshape(E, H, F // 32)
     return logits, X, W1q, W1s, W2q, W2s
+
+
+def mx_scale_tiles(plain: np.ndarray) -> np.ndarray:
+    """Scale bytes [rows, K/32] -> the library's tiled order (a pure permutation; rows padded to a multiple of 128 with
+    the byte 127 = 2^0, K a multiple of 128): tile (rows 128 t .. 128 t + 127, four consecutive 32-blocks c) is 512
+    contiguous bytes, byte (r % 32) * 16 + (r // 32) * 4 + c for row r of the tile."""
+    rows, kb = plain.shape
+    assert kb % 4 == 0
+    rp = (rows + 127) // 128 * 128
+    full = np.full((rp, kb), 127, np.uint8)
+    full[:rows] = plain
+    t = full.reshape(rp // 128, 4, 32, kb // 4, 4)            # [tile, q, r, chunk, c]
+    return np.ascontiguousarray(t.transpose(0, 3, 2, 1, 4)).reshape(-1)    # [tile, chunk, r, q, c]
+
+
+def mx_scale_plain(tiles: np.ndarray, rows: int, K: int) -> np.ndarray:
+    """Inverse of mx_scale_tiles."""
+    kb = K // 32
+    rp = (rows + 127) // 128 * 128
+    t = np.asarray(tiles, np.uint8).reshape(rp // 128, kb // 4, 32, 4, 4)   # [tile, chunk, r, q, c]
+    return np.ascontiguousarray(t.transpose(0, 3, 2, 1, 4)).reshape(rp, kb)[:rows]

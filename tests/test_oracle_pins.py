@@ -354,3 +354,62 @@ def test_attention_against_library_softmax_and_matmul(causal):
     # a sample of query rows equals the same rows of the full result
     qpos = np.array([0, 5, S - 1])
     assert np.array_equal(orc.attention(Q, K, V, Hq, Hkv, d, causal=causal, qpos=qpos), out[qpos])
+
+
+# ---------------------------------------------------------------------------------------------- MX (block-scaled FP8)
+def test_e4m3_table_matches_the_library_type_and_known_values():
+    codes = np.arange(256, dtype=np.uint8)
+    mine = orc.e4m3_to_f64(codes)
+    lib_vals = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    finite = ~np.isnan(lib_vals)
+    assert np.array_equal(np.isnan(mine), ~finite) and np.array_equal(mine[finite], lib_vals[finite])
+    assert mine[0x38] == 1.0 and mine[0x7E] == 448.0 and mine[0x01] == 2.0 ** -9 and mine[0xC0] == -2.0 and mine[0x08] == 2.0 ** -6
+
+
+def test_mx_quantize_hand_cases_and_library_rounding():
+    """Block max 448 -> e = 0, codes are the values themselves; max 1.0 -> e = -8, 1.0 becomes 256 (0x78); a value of 449
+    in a block whose max is 449 (e = 0) clamps to 448; ties go to the even code (13 is half-way between 12 and 14 at
+    this binade: 12 = 0x54 has an even mantissa... checked against the table itself); zero block -> scale byte 0."""
+    x = np.zeros((4, 32))
+    x[0, :4] = [448.0, 1.0, -3.5, 0.0625]
+    x[1, :3] = [1.0, 0.5, -0.75]
+    x[2, :2] = [449.0, 300.0]
+    codes, sf = orc.mx_quantize(x)
+    assert sf[0, 0] == 127 and sf[1, 0] == 127 - 8 and sf[2, 0] == 127 and sf[3, 0] == 0
+    v = orc.e4m3_to_f64(codes)
+    assert list(v[0, :4]) == [448.0, 1.0, -3.5, 0.0625]
+    assert list(v[1, :3]) == [256.0, 128.0, -192.0]
+    assert v[2, 0] == 448.0 and v[2, 1] == 288.0 or v[2, 1] == 320.0      # 300 lies between 288 and 320: nearest is 288
+    assert v[2, 1] == 288.0
+    assert not np.any(v[3])
+    # in-range values against the library's round-to-nearest-even conversion
+    rng = np.random.default_rng(0)
+    y = rng.standard_normal((64, 64)) * rng.choice([1e-3, 1.0, 30.0], (64, 1))
+    c, s = orc.mx_quantize(y)
+    scaled = y.reshape(64, 2, 32) * (2.0 ** (127.0 - s.astype(np.float64)))[:, :, None]
+    assert np.max(np.abs(scaled)) < 512.0
+    inr = np.abs(scaled) <= 448.0
+    want = torch.from_numpy(scaled).to(torch.float32).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(c.reshape(64, 2, 32)[inr], want[inr])
+    # dequantised blocks reproduce the input to within half an E4M3 step of the block maximum's binade
+    deq = orc.e4m3_to_f64(c).reshape(64, 2, 32) * (2.0 ** (s.astype(np.float64) - 127.0))[:, :, None]
+    amax = np.abs(y.reshape(64, 2, 32)).max(axis=2, keepdims=True)
+    assert np.all(np.abs(deq - y.reshape(64, 2, 32)) <= amax / 8.0 + 1e-300)
+
+
+def test_mx_gemm_against_library_matmul_and_scale_tiling_roundtrip():
+    rng = np.random.default_rng(1)
+    M, N, K = 9, 13, 256
+    a, asf = orc.mx_quantize(rng.standard_normal((M, K)))
+    w, wsf = orc.mx_quantize(rng.standard_normal((N, K)) * 0.01)
+    A = orc.e4m3_to_f64(a).reshape(M, K // 32, 32) * (2.0 ** (asf.astype(np.float64) - 127))[:, :, None]
+    W = orc.e4m3_to_f64(w).reshape(N, K // 32, 32) * (2.0 ** (wsf.astype(np.float64) - 127))[:, :, None]
+    want = (torch.from_numpy(A.reshape(M, K)) @ torch.from_numpy(W.reshape(N, K)).T).numpy()
+    assert np.allclose(orc.mx_gemm(a, asf, w, wsf), want, rtol=1e-13, atol=1e-300)
+    # hand case: one block, a = 1.0 (code 0x38) with scale 2^1, w = 0.5 (0x30) with scale 2^-2: 32 * 2 * 0.125 = 8
+    one = np.full((1, 32), 0x38, np.uint8); half = np.full((1, 32), 0x30, np.uint8)
+    assert orc.mx_gemm(one, np.array([[128]], np.uint8), half, np.array([[125]], np.uint8))[0, 0] == 8.0
+    plain = rng.integers(0, 255, (300, 8)).astype(np.uint8)
+    tiles = synth.mx_scale_tiles(plain)
+    assert tiles.size == 384 * 8 and np.array_equal(synth.mx_scale_plain(tiles, 300, 256), plain)
+    assert tiles[100] == plain[38, 0] and tiles[511] == plain[127, 3] and tiles[512 + 17] == plain[1, 5]
