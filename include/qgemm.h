@@ -129,6 +129,29 @@ int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, co
                   const void* Wscale, void* C, void* stream);
 
 /*
+ * Block-scaled FP8 operands (no counterpart in the paper, whose kernels keep the checkpoint's quantisation and
+ * dequantise on the way to the tensor units; on sm_100a the tensor cores apply one power-of-two scale per 32
+ * consecutive k themselves, at twice the bf16 rate).  Format of an operand with `rows` rows:
+ *   codes   uint8 [rows, K], OCP FP8 E4M3 (bias 7, largest finite 448), K % 128 == 0
+ *   scales  one E8M0 byte (2^(b - 127)) per row and 32 consecutive k, qg_mx_scale_bytes(rows, K) bytes in tiles of
+ *           128 rows x 4 blocks: tile (rows 128 t .., blocks 4 c ..) is 512 contiguous bytes at ((t * K/128) + c) * 512,
+ *           byte (r % 32) * 16 + (r / 32) * 4 + b for row r and block b of the tile (rows padded to 128 with 2^0)
+ * qg_mx_quantize re-encodes bf16 rows X [rows, K], qg_mx_pack_weights re-encodes block-quantised weights (the value
+ * q * scale of the formats above; a one-time step per model): per block e = floor(log2(max |x|)) - 8 clamped to
+ * [-127, 127] (-127 for an all-zero block), code = x / 2^e rounded to nearest even, clamped to +-448.  Both are lossy.
+ * qgemm_mx_dense:  C[m, n] = sum_k (a[m, k] 2^ea[m, k/32]) (w[n, k] 2^ew[n, k/32]), fp32 accumulate, bf16 [M, N] out;
+ * N % 8 == 0, M arbitrary.  The products are exact and the sums fp32, so against the exact value of this definition the
+ * result is within the tolerance of the other GEMMs; against the bf16 x Q8 / Q4 product it differs by the
+ * re-encoding error of both operands (about 3e-2 relative Frobenius for N(0,1) activations).
+ */
+size_t qg_mx_scale_bytes(int rows, int K);
+int qg_mx_quantize(qg_ctx* ctx, int rows, int K, const void* X, void* codes, void* scales, void* stream);
+int qg_mx_pack_weights(qg_ctx* ctx, int qbits, int N, int K, const void* Wq, const void* Wscale, void* codes,
+                       void* scales, void* stream);
+int qgemm_mx_dense(qg_ctx* ctx, int M, int N, int K, const void* A_codes, const void* A_scales, const void* W_codes,
+                   const void* W_scales, void* C, void* stream);
+
+/*
  * Prefill attention (Sec. 3.1: the attention operator of prompt processing with both matrix products on the tensor
  * units and the softmax kept exact, so that it equals the plain definition):
  *   O[i, h, :] = sum_j softmax_j(scale * Q[i, h, :] . K[j, g, :]) * V[j, g, :],   g = h / (Hq / Hkv),

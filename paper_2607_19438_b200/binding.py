@@ -20,6 +20,7 @@ D_BF16, D_F32_ACC = 0, 1
 
 EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_plan_dense", "qg_set_schedule", "qg_route_workspace_bytes",
            "qgemm_dense", "qgemm_small_m", "qgemm_dense_gate_up_silu", "prefill_attention",
+           "qg_mx_scale_bytes", "qg_mx_quantize", "qg_mx_pack_weights", "qgemm_mx_dense",
            "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_grouped_qgemm_gather", "moe_combine"]
 
 
@@ -56,6 +57,11 @@ def load():
         lib.qgemm_dense_gate_up_silu.argtypes = [vp, ci, ci, ci, ci, vp, vp, vp, vp, vp]
         ll = C.c_longlong
         lib.prefill_attention.argtypes = [vp, ci, ci, ci, ci, vp, ll, vp, ll, vp, ll, vp, ll, ci, C.c_float, vp]
+        lib.qg_mx_scale_bytes.restype = C.c_size_t
+        lib.qg_mx_scale_bytes.argtypes = [ci, ci]
+        lib.qg_mx_quantize.argtypes = [vp, ci, ci, vp, vp, vp, vp]
+        lib.qg_mx_pack_weights.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp]
+        lib.qgemm_mx_dense.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp]
         lib.moe_route.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp, C.c_size_t, vp]
         lib.moe_route_static.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, vp]
         lib.moe_permute.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
@@ -175,6 +181,37 @@ def prefill_attention(Q, K, V, Hq, Hkv, d, causal=True, scale=0.0, out=None):
     _check(load().prefill_attention(context(), S, Hq, Hkv, d, _ptr(Q), Q.stride(0), _ptr(K), K.stride(0), _ptr(V),
                                     V.stride(0), _ptr(out), out.stride(0), 1 if causal else 0, float(scale), _stream()),
            "prefill_attention")
+    return out
+
+
+def mx_quantize(X):
+    """bf16 [rows, K] -> (E4M3 codes uint8 [rows, K], E8M0 scale bytes in the library's tiled order)."""
+    rows, K = X.shape
+    codes = torch.empty((rows, K), dtype=torch.uint8, device=X.device)
+    sf = torch.empty(max(16, int(load().qg_mx_scale_bytes(rows, K))), dtype=torch.uint8, device=X.device)
+    _check(load().qg_mx_quantize(context(), rows, K, _ptr(X), _ptr(codes), _ptr(sf), _stream()), "qg_mx_quantize")
+    return codes, sf
+
+
+def mx_pack_weights(qbits, Wq, Wscale):
+    """Q8 / Q4 weights + fp16 scales -> (E4M3 codes uint8 [N, K], E8M0 scale bytes, tiled)."""
+    N = Wq.shape[0]
+    K = Wscale.shape[1] * 32
+    codes = torch.empty((N, K), dtype=torch.uint8, device=Wq.device)
+    sf = torch.empty(max(16, int(load().qg_mx_scale_bytes(N, K))), dtype=torch.uint8, device=Wq.device)
+    _check(load().qg_mx_pack_weights(context(), qbits, N, K, _ptr(Wq), _ptr(Wscale), _ptr(codes), _ptr(sf), _stream()),
+           "qg_mx_pack_weights")
+    return codes, sf
+
+
+def qgemm_mx_dense(A_codes, A_sf, W_codes, W_sf, out=None):
+    """Block-scaled FP8 GEMM: codes uint8 [M, K] / [N, K], scale bytes tiled -> bf16 [M, N]."""
+    M, K = A_codes.shape
+    N = W_codes.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=A_codes.device)
+    _check(load().qgemm_mx_dense(context(), M, N, K, _ptr(A_codes), _ptr(A_sf), _ptr(W_codes), _ptr(W_sf), _ptr(out),
+                                 _stream()), "qgemm_mx_dense")
     return out
 
 
