@@ -119,23 +119,41 @@ mx_quantize_kernel(int rows, int rows_padded, int K, const void* __restrict__ sr
 }
 
 // ------------------------------------------------------------------------------------------------ GEMM
-constexpr int MX_BM = 128, MX_BN = 256, MX_BK = 128, MX_ST = 4, MX_THREADS = 192;
-constexpr int MX_A_BYTES = MX_BM * MX_BK, MX_B_BYTES = MX_BN * MX_BK, MX_SFA_BYTES = 512, MX_SFB_BYTES = 1024;
-constexpr int MX_STAGE = MX_A_BYTES + MX_B_BYTES + MX_SFA_BYTES + MX_SFB_BYTES + 512;     // 51200: stages stay 1024-byte aligned
-constexpr int MX_OFF_BAR = MX_ST * MX_STAGE;
-constexpr int MX_SMEM = MX_OFF_BAR + 16 * 8 + 32 + 1024;
-constexpr int MX_COL_SF = 256;                     // scale columns: stage s at 256 + 16 s (4 for the tokens, 8 for the weights)
+// Persistent CTA pairs (cta_group::2).  A pair owns tiles of 256 tokens x 192 weight rows: each CTA stages its own 128
+// token rows (the MMA's A operand, M = 256 over the pair) and its half of the weight rows (B, 96 of N = 192), so a CTA
+// moves 28 KB per 128-k chunk for 128 x 192 x 128 products; two 192-column fp32 accumulators per CTA alternate between
+// the MMAs and the epilogue; the scale tiles of a chunk (one for this CTA's tokens, two for the weight rows) take 16
+// tensor-memory columns per stage.
+// The four MMAs of a chunk keep the tensor cores busy for 384 cycles only, and a lone thread is slow: it issues a
+// bulk-tensor copy about every 130 cycles and needs some hundred cycles for a wait, a commit and the address arithmetic
+// of a chunk.  So the loads of a stage are spread over three warps (token codes, weight codes, scale tiles), and the
+// three scale copies and four MMAs of a chunk are one statement with the descriptors advanced inside it.  The ring has
+// seven stages: load latency + MMAs + commit are about 2200 cycles from the release of a stage to its next release.
+constexpr int MX_BM = 128, MX_BN = 192, MX_BK = 128, MX_ST = 7, MX_THREADS = 256;
+constexpr int MX_A_BYTES = MX_BM * MX_BK, MX_B_BYTES = (MX_BN / 2) * MX_BK, MX_SF_BYTES = 512;
+constexpr int MX_STAGE = MX_A_BYTES + MX_B_BYTES;                           // codes of a stage: 28 KB, 1024-byte aligned
+constexpr int MX_OFF_B = MX_A_BYTES;
+constexpr int MX_SF_STAGE = 3 * MX_SF_BYTES;                                // token tile, two weight tiles
+constexpr int MX_OFF_SF = MX_ST * MX_STAGE;
+constexpr int MX_LOADED = MX_STAGE + MX_SF_STAGE;                           // bytes one CTA receives per stage
+constexpr int MX_OFF_BAR = MX_OFF_SF + MX_ST * MX_SF_STAGE;
+constexpr int MX_NBAR = 2 * MX_ST + 4;                                      // full, empty, acc_full[2], acc_empty[2]
+constexpr int MX_SMEM = MX_OFF_BAR + MX_NBAR * 8 + 32 + 1024;
+constexpr int MX_COL_SF = 2 * MX_BN;               // scale columns: stage s at 384 + 16 s (4 for the tokens, 8 for the weights)
+static_assert(MX_STAGE % 1024 == 0 && MX_COL_SF + 16 * MX_ST <= 512 && MX_SMEM <= 232448, "budgets");
 
 struct MxParams {
     int M, N, K;
-    const uint8_t* a_sf;
-    const uint8_t* w_sf;
+    int tiles_m, tiles;         // 256-token rows of tiles; all tiles (token index fastest)
     __nv_bfloat16* C;
     int* status;
     uint32_t wait_limit;
 };
 
+// Bounded wait: a few non-blocking tests first (the barrier is usually complete or about to be).
 __device__ __forceinline__ bool mx_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, const MxParams& p) {
+    for (int it = 0; it < 16; ++it)
+        if (mbar_test_wait_cluster(bar, parity)) return true;
     for (uint32_t it = 0; it < p.wait_limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
@@ -144,115 +162,166 @@ __device__ __forceinline__ bool mx_wait(uint32_t bar, uint32_t parity, volatile 
     atomicCAS(p.status, 0, QG_ERR_TIMEOUT);
     return false;
 }
-// Untiled bulk copy global -> shared (16-byte aligned, size a multiple of 16), completion bytes on `bar`.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+// tcgen05.commit of this thread's cta_group::2 operations onto the barrier at the same offset in both CTAs.
+__device__ __forceinline__ void mx_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(static_cast<unsigned short>(3)) : "memory");
 }
-// Shared-memory descriptor of a scale tile for tcgen05.cp: 32 rows of 16 bytes, no swizzle, 8-row groups 128 bytes apart.
-__device__ __forceinline__ uint64_t mx_sf_desc(uint32_t saddr) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((saddr & 0x3FFFF) >> 4);
-    d |= static_cast<uint64_t>(16 >> 4) << 16;
-    d |= static_cast<uint64_t>(128 >> 4) << 32;
-    d |= static_cast<uint64_t>(1) << 46;
-    return d;
+// One 128-k chunk: the three scale tiles go from shared to tensor memory (tcgen05.cp, in both CTAs; descriptor: 32
+// rows of 16 bytes, no swizzle, 8-row groups 128 bytes apart; the tiles are 512 bytes apart), then the four MMAs
+// (K = 32 each).  a_lo / b_lo: low words of the operand descriptors of the chunk's first 32 k (128-byte swizzle, so 32 k
+// further is +2 in 16-byte units); idesc0: instruction descriptor with scale ids 0 (E4M3 x E4M3, both K-major, E8M0
+// scales; the ids select the 32-block of the chunk); acc0 = 0 overwrites the accumulator.
+__device__ __forceinline__ void mx_chunk(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc0,
+                                         uint32_t sf_t, uint32_t sfb_t, uint32_t acc0, uint32_t sf_lo) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a0, a1, a2, a3, b0, b1, b2, b3, s0, s1, s2;\n\t"
+        ".reg .b32 x1, x2, x3, y1, y2, y3, i1, i2, i3, z1, z2, t1, t2, sh;\n\t"
+        "setp.ne.b32 p0, %7, 0;\n\tsetp.eq.b32 p1, %7, %7;\n\t"
+        "mov.u32 sh, 0x4008;\n\tadd.u32 z1, %8, 32;\n\tadd.u32 z2, %8, 64;\n\tadd.u32 t1, %5, 4;\n\tadd.u32 t2, %5, 8;\n\t"
+        "mov.b64 s0, {%8, sh};\n\tmov.b64 s1, {z1, sh};\n\tmov.b64 s2, {z2, sh};\n\t"
+        "tcgen05.cp.cta_group::2.32x128b.warpx4 [%5], s0;\n\t"
+        "tcgen05.cp.cta_group::2.32x128b.warpx4 [t1], s1;\n\t"
+        "tcgen05.cp.cta_group::2.32x128b.warpx4 [t2], s2;\n\t"
+        "add.u32 x1, %1, 2;\n\tadd.u32 x2, %1, 4;\n\tadd.u32 x3, %1, 6;\n\t"
+        "add.u32 y1, %2, 2;\n\tadd.u32 y2, %2, 4;\n\tadd.u32 y3, %2, 6;\n\t"
+        "add.u32 i1, %4, 0x20000010;\n\tadd.u32 i2, %4, 0x40000020;\n\tadd.u32 i3, %4, 0x60000030;\n\t"
+        "mov.b64 a0, {%1, %3};\n\tmov.b64 a1, {x1, %3};\n\tmov.b64 a2, {x2, %3};\n\tmov.b64 a3, {x3, %3};\n\t"
+        "mov.b64 b0, {%2, %3};\n\tmov.b64 b1, {y1, %3};\n\tmov.b64 b2, {y2, %3};\n\tmov.b64 b3, {y3, %3};\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale [%0], a0, b0, %4, [%5], [%6], p0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale [%0], a1, b1, i1, [%5], [%6], p1;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale [%0], a2, b2, i2, [%5], [%6], p1;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale [%0], a3, b3, i3, [%5], [%6], p1;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc0), "r"(sf_t), "r"(sfb_t), "r"(acc0), "r"(sf_lo)
+        : "memory");
 }
 
-__global__ void __launch_bounds__(MX_THREADS, 1)
-qgemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w, const MxParams p) {
+// tm_a / tm_w: the code matrices (boxes of 128 k x 128 token rows / 96 weight rows, 128-byte swizzle); tm_sa / tm_sw:
+// the scale tiles as 32-bit words, one row per 128 matrix rows, 128 words per chunk (box = one tile / two tiles of
+// consecutive rows).  Everything outside a matrix reads as zero, and a
+// zero scale byte times zero codes contributes nothing, so ragged edges need no special case in the loads.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MX_THREADS, 1)
+qgemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+                const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ CUtensorMap tm_sw, const MxParams p) {
     extern __shared__ uint8_t smem_dyn[];
     const uint32_t sbase = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     uint8_t* sgen = smem_dyn + (sbase - smem_u32(smem_dyn));
-    volatile int* misc = reinterpret_cast<volatile int*>(sgen + MX_OFF_BAR + 16 * 8);     // [0] tmem base, [1] abort
+    volatile int* misc = reinterpret_cast<volatile int*>(sgen + MX_OFF_BAR + MX_NBAR * 8);     // [0] tmem base, [1] abort
     volatile int* abort_flag = misc + 1;
     const uint32_t bar0 = sbase + MX_OFF_BAR;
-    auto full = [&](int s) { return bar0 + 8u * s; };
-    auto empty = [&](int s) { return bar0 + 8u * (MX_ST + s); };
-    const uint32_t acc_full = bar0 + 8u * (2 * MX_ST);
+    auto full = [&](uint32_t s) { return bar0 + 8u * s; };                              // even CTA only
+    auto empty = [&](uint32_t s) { return bar0 + 8u * (MX_ST + s); };                   // both CTAs
+    auto acc_full = [&](uint32_t a) { return bar0 + 8u * (2 * MX_ST + a); };
+    auto acc_empty = [&](uint32_t a) { return bar0 + 8u * (2 * MX_ST + 2 + a); };       // even CTA only
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * MX_BM, n0 = blockIdx.y * MX_BN;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
     const int nch = p.K / MX_BK;
-    const int n_tiles_w = min(2, (p.N - n0 + 127) >> 7);           // weight scale tiles this CTA needs (1 or 2)
 
     pdl_launch_dependents();
     if (warp == 0) {
-        if (lane < 2 * MX_ST + 1) mbar_init(bar0 + 8u * lane, 1);
+        if (lane < MX_NBAR) mbar_init(bar0 + 8u * lane, lane < MX_NBAR - 2 ? 1 : 8);     // acc_empty: 4 epilogue warps x 2 CTAs
         if (lane == 31) misc[1] = 0;
         fence_mbar_init();
         fence_proxy_async_smem();
-        if (lane == 30) prefetch_tmap(&tm_a);
-        if (lane == 29) prefetch_tmap(&tm_w);
+        if (lane == 30) { prefetch_tmap(&tm_a); prefetch_tmap(&tm_sa); }
+        if (lane == 29) { prefetch_tmap(&tm_w); prefetch_tmap(&tm_sw); }
     }
     if (warp == 1) {
-        tmem_alloc(sbase + MX_OFF_BAR + 16 * 8, 512);
+        tmem_alloc(sbase + MX_OFF_BAR + MX_NBAR * 8, 512);
         tmem_relinquish();
     }
     tc_fence_before_sync();
     __syncthreads();
+    cluster_sync_all();          // both CTAs' barriers are initialised and both halves of tensor memory allocated
     tc_fence_after_sync();
     pdl_wait();
     const uint32_t tmem_base = static_cast<uint32_t>(misc[0]);
+    // chunks this pair works through, over all of its tiles
+    const int my_tiles = (p.tiles - pair + npairs - 1) / npairs;
+    const uint32_t total = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(nch);
 
-    if (warp == 0) {
-        // ------------------------------------------------ producer
-        bool ok = true;
-        for (int j = 0; j < nch && ok; ++j) {
-            const int s = j % MX_ST;
-            const uint32_t ph = (j / MX_ST) & 1u;
-            if (j >= MX_ST && !mx_wait(empty(s), ph ^ 1u, abort_flag, p)) { ok = false; break; }
+    if (warp == 0 || warp == 2 || warp == 3) {
+        // ------------------------------------------------ producers: this CTA's share of every stage; warp 0 the token
+        // codes, warp 2 the weight codes, warp 3 the scale tiles.  The even CTA's warp 0 arms the stage's barrier for
+        // the bytes of all three warps and both CTAs.
+        const uint32_t full_leader = map_to_cta(full(0), 0);
+        int t = pair, j = 0;
+        int m0 = 0, n0 = 0, sa_row = 0, sw_row = 0;
+        auto locate = [&]() {
+            const int tm = t % p.tiles_m, tn = t / p.tiles_m;
+            m0 = tm * 2 * MX_BM + static_cast<int>(rank) * MX_BM;
+            n0 = tn * MX_BN + static_cast<int>(rank) * (MX_BN / 2);      // this CTA's half of the weight rows
+            sa_row = 2 * tm + static_cast<int>(rank);                    // this CTA's token scale tiles
+            sw_row = (tn * MX_BN) >> 7;                                  // first of the two weight scale tiles
+        };
+        locate();
+        uint32_t s = 0, ph = 0;
+        for (uint32_t g = 0; g < total; ++g) {
+            if (g >= MX_ST && !mx_wait(empty(s), ph ^ 1u, abort_flag, p)) break;
             if (lane == 0) {
-                const uint32_t st = sbase + s * MX_STAGE;
-                mbar_arrive_expect_tx(full(s), MX_A_BYTES + MX_B_BYTES + MX_SFA_BYTES + 512u * n_tiles_w);
-                tma_load_2d(st, &tm_a, j * MX_BK, m0, full(s));
-                tma_load_2d(st + MX_A_BYTES, &tm_w, j * MX_BK, n0, full(s));
-                bulk_load(st + MX_A_BYTES + MX_B_BYTES, p.a_sf + (static_cast<size_t>(blockIdx.x) * nch + j) * 512, 512, full(s));
-                for (int t = 0; t < n_tiles_w; ++t)
-                    bulk_load(st + MX_A_BYTES + MX_B_BYTES + MX_SFA_BYTES + t * 512,
-                              p.w_sf + (static_cast<size_t>(2 * blockIdx.y + t) * nch + j) * 512, 512, full(s));
+                const uint32_t fb = full_leader + 8u * s;
+                if (warp == 0) {
+                    if (rank == 0) mbar_arrive_expect_tx(full(s), 2u * MX_LOADED);
+                    tma_load_2d_pair(sbase + s * MX_STAGE, &tm_a, j * MX_BK, m0, fb);
+                } else if (warp == 2) {
+                    tma_load_2d_pair(sbase + s * MX_STAGE + MX_OFF_B, &tm_w, j * MX_BK, n0, fb);
+                } else {
+                    const uint32_t sf = sbase + MX_OFF_SF + s * MX_SF_STAGE;
+                    tma_load_2d_pair(sf, &tm_sa, j * 128, sa_row, fb);
+                    tma_load_2d_pair(sf + MX_SF_BYTES, &tm_sw, j * 128, sw_row, fb);         // two tiles: rows sw_row, sw_row + 1
+                }
             }
             __syncwarp();
+            if (++j == nch) { j = 0; t += npairs; locate(); }
+            if (++s == MX_ST) { s = 0; ph ^= 1u; }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------ scale copies and MMAs
-        bool ok = true;
-        for (int j = 0; j < nch && ok; ++j) {
-            const int s = j % MX_ST;
-            if (!mx_wait(full(s), (j / MX_ST) & 1u, abort_flag, p)) { ok = false; break; }
-            tc_fence_after_sync();
-            if (lane == 0) {
-                const uint32_t st = sbase + s * MX_STAGE;
-                const uint32_t sfa_t = tmem_base + MX_COL_SF + 16 * s, sfb_t = sfa_t + 4;
-                asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(sfa_t), "l"(mx_sf_desc(st + MX_A_BYTES + MX_B_BYTES)) : "memory");
-                for (int t = 0; t < n_tiles_w; ++t)
-                    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;"
-                                 ::"r"(sfb_t + 4 * t), "l"(mx_sf_desc(st + MX_A_BYTES + MX_B_BYTES + MX_SFA_BYTES + t * 512)) : "memory");
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    // block-scaled instruction descriptor: E4M3 x E4M3, both K-major, E8M0 scales, ids = block of the chunk
-                    const uint32_t idesc = (static_cast<uint32_t>(kk) << 4) | ((MX_BN >> 3) << 17) | (1u << 23) |
-                                           ((MX_BM >> 4) << 24) | (static_cast<uint32_t>(kk) << 29);
-                    const uint64_t da = umma_desc_k_sw128(st + 32 * kk), db = umma_desc_k_sw128(st + MX_A_BYTES + 32 * kk);
-                    const uint32_t acc = (j > 0 || kk > 0) ? 1u : 0u;
-                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                                 "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-                                 ::"r"(tmem_base), "l"(da), "l"(db), "r"(idesc), "r"(acc), "r"(sfa_t), "r"(sfb_t) : "memory");
+        // ------------------------------------------------ scale copies and MMAs (even CTA, for the pair)
+        if (rank == 0) {
+            const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);          // group stride, version, 128-byte swizzle
+            const uint32_t idesc0 = ((MX_BN >> 3) << 17) | (1u << 23) | (((2 * MX_BM) >> 4) << 24);
+            uint32_t s = 0, ph = 0, jt = 0;
+            bool ok = true;
+            for (int t = pair; t < p.tiles && ok; t += npairs, ++jt) {
+                const int n0 = (t / p.tiles_m) * MX_BN;
+                const uint32_t a = jt & 1u;
+                if (jt >= 2 && !mx_wait(acc_empty(a), ((jt >> 1) & 1u) ^ 1u, abort_flag, p)) { ok = false; break; }
+                const uint32_t d_tmem = tmem_base + a * MX_BN;
+                // weight scale tiles at columns +4 .. +11 of the stage: the tile's first row is row n0 % 128 of the first
+                const uint32_t sfb_off = 4 + ((static_cast<uint32_t>(n0) & 127u) >> 5);
+                for (int j = 0; j < nch; ++j) {
+                    if (!mx_wait(full(s), ph, abort_flag, p)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    if (elect_one()) {
+                        const uint32_t st = sbase + s * MX_STAGE;
+                        const uint32_t sf_t = tmem_base + MX_COL_SF + 16 * s;
+                        mx_chunk(d_tmem, (st >> 4) | (1u << 16), ((st + MX_OFF_B) >> 4) | (1u << 16), hi, idesc0, sf_t,
+                                 sf_t + sfb_off, j > 0 ? 1u : 0u, ((sbase + MX_OFF_SF + s * MX_SF_STAGE) >> 4) | (1u << 16));
+                        mx_commit(empty(s));
+                        if (j == nch - 1) mx_commit(acc_full(a));
+                    }
+                    __syncwarp();
+                    if (++s == MX_ST) { s = 0; ph ^= 1u; }
                 }
-                umma_commit(empty(s));
-                if (j == nch - 1) umma_commit(acc_full);
             }
-            __syncwarp();
         }
     } else {
         // ------------------------------------------------ epilogue (thread = token row; TMEM lane quarter = warp % 4)
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
-        const bool good = mx_wait(acc_full, 0u, abort_flag, p);
-        uint8_t* stage = sgen;                               // the ring is idle now: [128 rows][512 B], chunks XOR-swizzled
-        if (good) {
+        const uint32_t acc_empty_leader = map_to_cta(acc_empty(0), 0);
+        uint32_t jt = 0;
+        for (int t = pair; t < p.tiles; t += npairs, ++jt) {
+            const int tm = t % p.tiles_m, tn = t / p.tiles_m;
+            const int m = tm * 2 * MX_BM + static_cast<int>(rank) * MX_BM + row;
+            const int n0 = tn * MX_BN;
+            const uint32_t a = jt & 1u;
+            if (!mx_wait(acc_full(a), (jt >> 1) & 1u, abort_flag, p)) break;
             tc_fence_after_sync();
-            const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-#pragma unroll
+            const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + a * MX_BN;
+            __nv_bfloat16* crow = p.C + static_cast<size_t>(m < p.M ? m : 0) * p.N + n0;
+#pragma unroll 1
             for (int c = 0; c < MX_BN / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld_32x32(lane_addr + 32 * c, v);
@@ -265,27 +334,21 @@ qgemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
                         const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(v[8 * i + 2 * u]), __uint_as_float(v[8 * i + 2 * u + 1]));
                         w[u] = *reinterpret_cast<const uint32_t*>(&o2);
                     }
-                    *reinterpret_cast<uint4*>(stage + row * 512 + (((4 * c + i) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    if (m < p.M && n0 + 32 * c + 8 * i < p.N)
+                        *reinterpret_cast<uint4*>(crow + 32 * c + 8 * i) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
-        }
-        named_bar_sync(1, 128);              // reached by all four warps whatever happened above (every wait is bounded)
-        if (good) {
-            const int tid = threadIdx.x - 64;
-            for (int idx = tid; idx < MX_BM * 32; idx += 128) {
-                const int r = idx >> 5, vv = idx & 31;
-                const int m = m0 + r, n = n0 + vv * 8;
-                if (m < p.M && n < p.N)
-                    *reinterpret_cast<uint4*>(p.C + static_cast<size_t>(m) * p.N + n) =
-                        *reinterpret_cast<const uint4*>(stage + r * 512 + ((vv ^ (r & 7)) << 4));
-            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8u * a);
         }
     }
     tc_fence_before_sync();
     __syncthreads();
     if (*abort_flag) {
-        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);       // copies still in flight land before the memory is released
     }
+    cluster_sync_all();          // the peer no longer signals this CTA's barriers or reads its shared memory
     tc_fence_after_sync();
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
@@ -350,12 +413,19 @@ int qgemm_mx_dense(qg_ctx* ctx, int M, int N, int K, const void* A_codes, const 
         !qg::aligned16(Cout))
         return QG_ERR_ALIGN;
     if (const int rc = qg::check_device(ctx)) return rc;
-    const CUtensorMap *tm_a, *tm_w;
+    const CUtensorMap *tm_a, *tm_w, *tm_sa, *tm_sw;
+    const int nch = K / qg::MX_BK;
     int rc = qg::get_tmap_2d(ctx, &tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, A_codes, K, M, qg::MX_BK, qg::MX_BM,
                              CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc == QG_OK)
-        rc = qg::get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W_codes, K, N, qg::MX_BK, qg::MX_BN,
+        rc = qg::get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W_codes, K, N, qg::MX_BK, qg::MX_BN / 2,
                              CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc == QG_OK)
+        rc = qg::get_tmap_2d(ctx, &tm_sa, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, A_scales, static_cast<uint64_t>(nch) * 128,
+                             static_cast<uint64_t>((M + 127) / 128), 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (rc == QG_OK)
+        rc = qg::get_tmap_2d(ctx, &tm_sw, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, W_scales, static_cast<uint64_t>(nch) * 128,
+                             static_cast<uint64_t>((N + 127) / 128), 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc != QG_OK) return rc;
     constexpr int inst = 30;
     if (!ctx->attr_set[inst]) {
@@ -367,11 +437,12 @@ int qgemm_mx_dense(qg_ctx* ctx, int M, int N, int K, const void* A_codes, const 
     }
     qg::MxParams p{};
     p.M = M; p.N = N; p.K = K;
-    p.a_sf = static_cast<const uint8_t*>(A_scales); p.w_sf = static_cast<const uint8_t*>(W_scales);
+    p.tiles_m = (M + 2 * qg::MX_BM - 1) / (2 * qg::MX_BM);
+    p.tiles = p.tiles_m * ((N + qg::MX_BN - 1) / qg::MX_BN);
     p.C = static_cast<__nv_bfloat16*>(Cout); p.status = ctx->d_status; p.wait_limit = ctx->wait_limit;
-    const dim3 grid((M + qg::MX_BM - 1) / qg::MX_BM, (N + qg::MX_BN - 1) / qg::MX_BN);
-    return qg::launch_rc(qg::launch_kernel(ctx, qg::qgemm_mx_kernel, grid, dim3(qg::MX_THREADS), qg::MX_SMEM,
-                                           static_cast<cudaStream_t>(stream), *tm_a, *tm_w, p));
+    const int pairs = p.tiles < ctx->sm_count / 2 ? p.tiles : ctx->sm_count / 2;
+    return qg::launch_rc(qg::launch_kernel(ctx, qg::qgemm_mx_kernel, dim3(2 * pairs), dim3(qg::MX_THREADS), qg::MX_SMEM,
+                                           static_cast<cudaStream_t>(stream), *tm_a, *tm_w, *tm_sa, *tm_sw, p));
 }
 
 }  // extern "C"
