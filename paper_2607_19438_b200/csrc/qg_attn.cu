@@ -61,18 +61,6 @@ struct AttnCfg {
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
-// Shared-memory operand descriptor for an N-major (or M-major) bf16 tile: 64 consecutive N elements are contiguous
-// (128 bytes, 128-byte swizzle), consecutive k are 128 bytes apart in groups of eight (1024 bytes), the next 64 N
-// elements start lbo_bytes further on.
-__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t lbo_bytes) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((saddr & 0x3FFFF) >> 4);
-    d |= static_cast<uint64_t>(lbo_bytes >> 4) << 16;
-    d |= static_cast<uint64_t>(1024 >> 4) << 32;
-    d |= static_cast<uint64_t>(1) << 46;
-    d |= static_cast<uint64_t>(2) << 61;
-    return d;
-}
 // Instruction descriptor: f32 accumulate, bf16 x bf16, A K-major, B K-major (b_mn = 0) or N-major (1), tile M x N.
 __device__ __forceinline__ uint32_t umma_idesc_bf16_major(uint32_t M, uint32_t N, uint32_t b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
@@ -84,8 +72,47 @@ __device__ __forceinline__ float fast_exp2(float x) {     // 2^x, exp2(-inf) = 0
     return y;
 }
 
+// Four consecutive K = 16 steps in one statement (a lone thread is slow at address arithmetic, so the descriptors are
+// advanced inside it).  lo words: start address >> 4 plus the fixed fields; `hi` is shared by all descriptors.
+// Both operands in shared memory, K-major with 128-byte swizzle: 16 k further is +2 in 16-byte units.
+__device__ __forceinline__ void umma_ss_x4(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                           uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a0, a1, a2, a3, b0, b1, b2, b3;\n\t.reg .b32 x1, x2, x3, y1, y2, y3;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, %5, %5;\n\t"
+        "add.u32 x1, %1, 2;\n\tadd.u32 x2, %1, 4;\n\tadd.u32 x3, %1, 6;\n\t"
+        "add.u32 y1, %2, 2;\n\tadd.u32 y2, %2, 4;\n\tadd.u32 y3, %2, 6;\n\t"
+        "mov.b64 a0, {%1, %3};\n\tmov.b64 a1, {x1, %3};\n\tmov.b64 a2, {x2, %3};\n\tmov.b64 a3, {x3, %3};\n\t"
+        "mov.b64 b0, {%2, %3};\n\tmov.b64 b1, {y1, %3};\n\tmov.b64 b2, {y2, %3};\n\tmov.b64 b3, {y3, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a0, b0, %4, p0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %4, p1;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc0)
+        : "memory");
+}
+// A from tensor memory (8 columns of packed bf16 pairs per step), B in shared memory N-major: 16 k further is 2048
+// bytes (+128 in 16-byte units).
+__device__ __forceinline__ void umma_ts_x4(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                           uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 b0, b1, b2, b3;\n\t.reg .b32 x1, x2, x3, y1, y2, y3;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, %5, %5;\n\t"
+        "add.u32 x1, %1, 8;\n\tadd.u32 x2, %1, 16;\n\tadd.u32 x3, %1, 24;\n\t"
+        "add.u32 y1, %2, 128;\n\tadd.u32 y2, %2, 256;\n\tadd.u32 y3, %2, 384;\n\t"
+        "mov.b64 b0, {%2, %3};\n\tmov.b64 b1, {y1, %3};\n\tmov.b64 b2, {y2, %3};\n\tmov.b64 b3, {y3, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], b0, %4, p0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [x1], b1, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [x2], b2, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [x3], b3, %4, p1;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc0)
+        : "memory");
+}
+
 __device__ __forceinline__ bool at_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, const AttnParams& p) {
     const uint32_t limit = p.wait_limit;
+    for (int it = 0; it < 16; ++it)
+        if (mbar_test_wait_cluster(bar, parity)) return true;
     for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
@@ -117,8 +144,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_qb = (p.S + 2 * AT_BQ - 1) / (2 * AT_BQ);
-    const int qb = n_qb - 1 - static_cast<int>(blockIdx.x);     // the longest (last) query blocks start first
-    const int h = blockIdx.y;
+    // Blocks are dispatched with x fastest: all heads of the longest (last) query block first, then the next longest, so
+    // that under a causal mask no long block starts late; neighbouring heads share their K / V head in L2.
+    const int h = blockIdx.x;
+    const int qb = n_qb - 1 - static_cast<int>(blockIdx.y);
     const int g = h / (p.Hq / p.Hkv);
     const int q0 = qb * 2 * AT_BQ;
     // key tiles each query tile attends to
@@ -191,19 +220,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t idesc_s = umma_idesc_bf16_major(AT_BQ, AT_BKV, 0u);
         const uint32_t idesc_o = umma_idesc_bf16_major(AT_BQ, D, 1u);
         bool ok = at_wait(q_full, 0u, abort_flag, p);
+        const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);     // group stride, version, 128-byte swizzle
         auto issue_s = [&](int t, int j, bool last_on_k) -> bool {      // S_t(j) = Q_t K(j)^T
             const int s = j & 1;
             if (!at_wait(k_full(s), (j >> 1) & 1u, abort_flag, p)) return false;
             tc_fence_after_sync();
-            if (lane == 0) {
-                const uint32_t q_addr = sbase + C::OFF_Q + t * C::TILE_BYTES;
-                const uint32_t k_addr = sbase + C::OFF_K + s * C::TILE_BYTES;
+            if (elect_one()) {
+                const uint32_t q_lo = ((sbase + C::OFF_Q + t * C::TILE_BYTES) >> 4) | (1u << 16);
+                const uint32_t k_lo = ((sbase + C::OFF_K + s * C::TILE_BYTES) >> 4) | (1u << 16);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * C::BOX_BYTES + (kk & 3) * 32;
-                    umma_f16_ss(tmem_base + C::COL_S + t * 128, umma_desc_k_sw128(q_addr + off),
-                                umma_desc_k_sw128(k_addr + off), idesc_s, kk ? 1u : 0u);
-                }
+                for (int b = 0; b < C::NBOX; ++b)          // 64 head dimensions (one box) per statement
+                    umma_ss_x4(tmem_base + C::COL_S + t * 128, q_lo + b * (C::BOX_BYTES >> 4), k_lo + b * (C::BOX_BYTES >> 4),
+                               desc_hi, idesc_s, b ? 1u : 0u);
                 umma_commit(s_full(t));
                 if (last_on_k) umma_commit(k_empty(s));
             }
@@ -214,12 +242,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int s = j & 1;
             if (!at_wait(p_full(t), j & 1u, abort_flag, p) || !at_wait(v_full(s), (j >> 1) & 1u, abort_flag, p)) return false;
             tc_fence_after_sync();
-            if (lane == 0) {
-                const uint32_t v_addr = sbase + C::OFF_V + s * C::TILE_BYTES;
+            if (elect_one()) {
+                // 16 keys per instruction: two 8-key groups of V; the next 64 head dimensions are one box further
+                const uint32_t v_lo = ((sbase + C::OFF_V + s * C::TILE_BYTES) >> 4) | ((C::BOX_BYTES >> 4) << 16);
 #pragma unroll
-                for (int kk = 0; kk < AT_BKV / 16; ++kk)          // 16 keys per instruction: two 8-key groups of V
-                    umma_f16_ts(tmem_base + C::COL_O + t * D, tmem_base + C::COL_S + t * 128 + 8 * kk,
-                                umma_desc_mn_sw128(v_addr + kk * 2048, C::BOX_BYTES), idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+                for (int b = 0; b < AT_BKV / 64; ++b)
+                    umma_ts_x4(tmem_base + C::COL_O + t * D, tmem_base + C::COL_S + t * 128 + 32 * b, v_lo + b * 512,
+                               desc_hi, idesc_o, (j > 0 || b > 0) ? 1u : 0u);
                 umma_commit(pv_done(t));
                 if (last_on_v) umma_commit(v_empty(s));
             }
@@ -389,7 +418,7 @@ static int launch_attn(qg_ctx* ctx, const AttnParams& p, const void* Q, long lon
         ctx->attr_set[inst] = true;
     }
     const int n_qb = (p.S + 2 * AT_BQ - 1) / (2 * AT_BQ);
-    if (launch_kernel(ctx, kern, dim3(n_qb, p.Hq), dim3(AT_THREADS), C::SMEM_BYTES, st, *tm_q, *tm_k, *tm_v, p) != cudaSuccess) {
+    if (launch_kernel(ctx, kern, dim3(p.Hq, n_qb), dim3(AT_THREADS), C::SMEM_BYTES, st, *tm_q, *tm_k, *tm_v, p) != cudaSuccess) {
         cudaGetLastError();
         return QG_ERR_CUDA;
     }
