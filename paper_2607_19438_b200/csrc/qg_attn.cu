@@ -49,7 +49,7 @@ struct AttnCfg {
     static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
     static constexpr int OFF_V = OFF_K + NST * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_V + NST * TILE_BYTES;
-    static constexpr int NBAR = 16;
+    static constexpr int NBAR = 20;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;
     static constexpr int COL_S = 0;                             // S / P of tile t at 128 t
@@ -64,6 +64,27 @@ struct AttnCfg {
 // Instruction descriptor: f32 accumulate, bf16 x bf16, A K-major, B K-major (b_mn = 0) or N-major (1), tile M x N.
 __device__ __forceinline__ uint32_t umma_idesc_bf16_major(uint32_t M, uint32_t N, uint32_t b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+// (x0, x1) * c + d on both halves of a packed pair (each half IEEE-exact like fmaf).
+__device__ __forceinline__ void fma2(float& y0, float& y1, float x0, float x1, uint64_t c2, uint64_t d2) {
+    asm("{\n\t.reg .b64 t;\n\tmov.b64 t, {%2, %3};\n\tfma.rn.f32x2 t, t, %4, %5;\n\tmov.b64 {%0, %1}, t;\n\t}"
+        : "=f"(y0), "=f"(y1) : "f"(x0), "f"(x1), "l"(c2), "l"(d2));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, float x0, float x1) {      // a + (x0, x1), packed
+    uint64_t r;
+    asm("{\n\t.reg .b64 t;\n\tmov.b64 t, {%2, %3};\n\tadd.rn.f32x2 %0, %1, t;\n\t}" : "=l"(r) : "l"(a), "f"(x0), "f"(x1));
+    return r;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
 }
 
 __device__ __forceinline__ float fast_exp2(float x) {     // 2^x, exp2(-inf) = 0
@@ -139,8 +160,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     auto k_empty = [&](int s) { return bar0 + 8u * (5 + s); };
     auto v_empty = [&](int s) { return bar0 + 8u * (7 + s); };
     auto s_full = [&](int t) { return bar0 + 8u * (9 + t); };      // per query tile: S(j) complete
-    auto p_full = [&](int t) { return bar0 + 8u * (11 + t); };     // P(j) written and O rescaled (4 warps arrive)
-    auto pv_done = [&](int t) { return bar0 + 8u * (13 + t); };    // P(j) V(j) complete
+    auto p_full = [&](int t, int h) { return bar0 + 8u * (11 + 2 * t + h); };   // P(j) of keys 64 h .. written (and O
+                                                                                 // rescaled): 4 warps arrive
+    auto pv_done = [&](int t) { return bar0 + 8u * (15 + t); };    // P(j) V(j) complete
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_qb = (p.S + 2 * AT_BQ - 1) / (2 * AT_BQ);
@@ -158,8 +180,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     pdl_launch_dependents();
     if (warp == 0) {
-        if (lane < 15) {
-            const uint32_t cnt = (lane == 11 || lane == 12) ? 4u : 1u;      // p_full: one arrival per softmax warp
+        if (lane < 17) {
+            const uint32_t cnt = (lane >= 11 && lane <= 14) ? 4u : 1u;      // p_full: one arrival per softmax warp
             mbar_init(bar0 + 8u * lane, cnt);
         }
         if (lane == 31) misc[1] = 0;
@@ -240,15 +262,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         };
         auto issue_pv = [&](int t, int j, bool last_on_v) -> bool {     // O_t += P_t(j) V(j)
             const int s = j & 1;
-            if (!at_wait(p_full(t), j & 1u, abort_flag, p) || !at_wait(v_full(s), (j >> 1) & 1u, abort_flag, p)) return false;
+            // 16 keys per instruction: two 8-key groups of V; the next 64 head dimensions are one box further.  The
+            // first 64 keys' products are issued as soon as their half of P is there, while the group still works on
+            // the other half (an MMA with its A operand in tensor memory takes about 125 cycles to issue).
+            const uint32_t v_lo = ((sbase + C::OFF_V + s * C::TILE_BYTES) >> 4) | ((C::BOX_BYTES >> 4) << 16);
+            if (!at_wait(p_full(t, 0), j & 1u, abort_flag, p) || !at_wait(v_full(s), (j >> 1) & 1u, abort_flag, p)) return false;
+            tc_fence_after_sync();
+            if (elect_one())
+                umma_ts_x4(tmem_base + C::COL_O + t * D, tmem_base + C::COL_S + t * 128, v_lo, desc_hi, idesc_o, j > 0 ? 1u : 0u);
+            __syncwarp();
+            if (!at_wait(p_full(t, 1), j & 1u, abort_flag, p)) return false;
             tc_fence_after_sync();
             if (elect_one()) {
-                // 16 keys per instruction: two 8-key groups of V; the next 64 head dimensions are one box further
-                const uint32_t v_lo = ((sbase + C::OFF_V + s * C::TILE_BYTES) >> 4) | ((C::BOX_BYTES >> 4) << 16);
-#pragma unroll
-                for (int b = 0; b < AT_BKV / 64; ++b)
-                    umma_ts_x4(tmem_base + C::COL_O + t * D, tmem_base + C::COL_S + t * 128 + 32 * b, v_lo + b * 512,
-                               desc_hi, idesc_o, (j > 0 || b > 0) ? 1u : 0u);
+                umma_ts_x4(tmem_base + C::COL_O + t * D, tmem_base + C::COL_S + t * 128 + 32, v_lo + 512, desc_hi, idesc_o, 1u);
                 umma_commit(pv_done(t));
                 if (last_on_v) umma_commit(v_empty(s));
             }
@@ -294,56 +320,65 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 128; i += 4) {
-                mx0 = fmaxf(mx0, __uint_as_float(v[i]));
-                mx1 = fmaxf(mx1, __uint_as_float(v[i + 1]));
-                mx2 = fmaxf(mx2, __uint_as_float(v[i + 2]));
-                mx3 = fmaxf(mx3, __uint_as_float(v[i + 3]));
+            for (int i = 0; i < 128; i += 8) {
+                mx0 = max3(mx0, __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+                mx1 = max3(mx1, __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                mx2 = max3(mx2, __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+                mx3 = max3(mx3, __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
             }
-            const float m_new = fmaxf(m, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)));
-            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // keeps a row without any visible key finite
-            const float mc = m_use * cl;
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {                              // 16 scores -> 8 columns of packed bf16 pairs
-                uint32_t pk[8];
-#pragma unroll
-                for (int i = 0; i < 16; i += 2) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(v[16 * c + i]), cl, -mc));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(v[16 * c + i + 1]), cl, -mc));
-                    s0 += p0;
-                    s1 += p1;
-                    const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-                    pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
-                }
-                tmem_st_32x32_x8(s_addr + 8 * c, pk);                 // P over the columns S came from
-            }
+            // The exponent's reference m follows the running maximum lazily: it moves only when some row of the warp
+            // has grown by more than 2^8 in the exponent (any reference gives the same quotient O / l; P stays below
+            // 256, exact enough in bf16 and far from overflow in the fp32 sums), so that the output accumulator, which
+            // may only be touched between two P V products, has to be rescaled rarely.
+            const float m_new = fmaxf(max3(m, mx0, mx1), fmaxf(mx2, mx3));
+            const bool moved = __any_sync(0xFFFFFFFFu, (m_new - m) * cl > 8.0f);      // -inf -> anything counts
+            const float m_pick = moved ? m_new : m;
+            const float m_use = (m_pick == -INFINITY) ? 0.f : m_pick;   // keeps a row without any visible key finite
             const float alpha = fast_exp2((m - m_use) * cl);          // exp2(-inf) = 0 on the first tile
-            l = l * alpha + (s0 + s1);
             m = m_use;
-            if (j > 0) {
+            if (j > 0 && moved) {
                 // O of the earlier tiles is rescaled once their last P V has completed
                 if (!at_wait(pv_done(t), (j - 1) & 1u, abort_flag, p)) { ok = false; break; }
                 tc_fence_after_sync();
-                if (!__all_sync(0xFFFFFFFFu, alpha == 1.0f)) {
 #pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t o[32];
-                        tmem_ld_32x32(o_addr + 32 * c, o);
-                        tmem_ld_wait();
-                        uint32_t (&lo)[16] = *reinterpret_cast<uint32_t (*)[16]>(o);
-                        uint32_t (&hi)[16] = *reinterpret_cast<uint32_t (*)[16]>(o + 16);
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld_32x32(o_addr + 32 * c, o);
+                    tmem_ld_wait();
+                    uint32_t (&lo)[16] = *reinterpret_cast<uint32_t (*)[16]>(o);
+                    uint32_t (&hi)[16] = *reinterpret_cast<uint32_t (*)[16]>(o + 16);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st_32x32_x16(o_addr + 32 * c, lo);
-                        tmem_st_32x32_x16(o_addr + 32 * c + 16, hi);
-                    }
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st_32x32_x16(o_addr + 32 * c, lo);
+                    tmem_st_32x32_x16(o_addr + 32 * c + 16, hi);
                 }
             }
-            tmem_st_wait();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(p_full(t));
+            const uint64_t cl2 = pack2(cl, cl), mc2 = pack2(-m_use * cl, -m_use * cl);
+            uint64_t sum2 = pack2(0.f, 0.f);
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {                           // P in two halves of 64 keys, each signalled
+#pragma unroll
+                for (int c = 4 * hh; c < 4 * hh + 4; ++c) {            // 16 scores -> 8 columns of packed bf16 pairs
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 2) {
+                        float e0, e1;
+                        fma2(e0, e1, __uint_as_float(v[16 * c + i]), __uint_as_float(v[16 * c + i + 1]), cl2, mc2);
+                        const float p0 = fast_exp2(e0), p1 = fast_exp2(e1);
+                        sum2 = add2(sum2, p0, p1);
+                        const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+                        pk[i >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+                    }
+                    tmem_st_32x32_x8(s_addr + 8 * c, pk);             // P over the columns S came from
+                }
+                tmem_st_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(p_full(t, hh));
+            }
+            float s0, s1;
+            asm("mov.b64 {%0, %1}, %2;" : "=f"(s0), "=f"(s1) : "l"(sum2));
+            l = l * alpha + (s0 + s1);
         }
         // ---- normalise and store: through this tile's (now idle) Q buffer, 16-byte chunks XOR-swizzled by the row
         const bool good = ok && n_t > 0 && at_wait(pv_done(t), (n_t - 1) & 1u, abort_flag, p);
