@@ -828,10 +828,15 @@ def run_case(args):
     import ctypes as C
     import torch
     from paper_2607_19438_b200 import binding as qg
+    if args.case == "roles":
+        from paper_2607_19438_b200 import build as qg_build
+        qg.LIB_PATH = qg_build.build_profile()
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     lib, ctx = qg.load(), qg.context(0)
     g = torch.Generator(device=dev); g.manual_seed(0)
+    if args.case == "roles":
+        return run_roles(lib, ctx, qg, dev, g)
     if args.case == "attention":
         S, Hq, Hkv, d = 2048, 32, 8, 128
         qkv = torch.randn((S, (Hq + 2 * Hkv) * d), device=dev, generator=g).to(torch.bfloat16)
@@ -883,6 +888,65 @@ def run_case(args):
     print(json.dumps({"case": args.case, "E": E, "M": M, "rows_per_expert": R / E, "passes": 3}))
 
 
+def run_roles(lib, ctx, qg, dev, g):
+    """Cycle accounting of the GEMM kernel's roles (profiling build of the library): for one launch each of two dense
+    and the two grouped GEMMs of the bench step, the cycles the first CTA's producer, MMA-issuing, conversion and
+    epilogue warps spent in each of their waits, next to the cycles from the CTA's start to its last commit."""
+    import ctypes as C
+    import torch
+    lib.qg_debug_set_stats.argtypes = [C.c_void_p, C.c_void_p]
+    lib.qg_debug_set_stats.restype = None
+    stats = torch.zeros(148 * 12 + 16 + 2 * 148 + 8, dtype=torch.int64, device=dev)
+    names = ["x_producer_wait", "w_producer_wait", "mma_wait_accumulator", "mma_wait_stage_full", None,
+             "convert_wait_packed", "convert_wait_stage_free", "convert_arithmetic_and_store", "epilogue_wait",
+             "epilogue_drain", "mma_issue", None]
+    rows = []
+
+    def measure(label, call, kblocks_per_tile):
+        lib.qg_debug_set_stats(ctx, None)
+        for _ in range(3):
+            call()
+        stats.zero_()
+        torch.cuda.synchronize()
+        lib.qg_debug_set_stats(ctx, C.c_void_p(stats.data_ptr()))
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(); call(); e1.record()
+        torch.cuda.synchronize()
+        lib.qg_debug_set_stats(ctx, None)
+        st = stats.cpu().numpy()
+        marks = st[148 * 12:148 * 12 + 16]
+        row = {"call": label, "event_us_profiling_build": round(e0.elapsed_time(e1) * 1e3, 1),
+               "cta0_cycles_start_to_last_commit": int(marks[3] - marks[0]),
+               "cta0_cycles_start_to_first_stage_full": int(marks[2] - marks[0]),
+               "k_blocks_per_tile": kblocks_per_tile,
+               "cta0_cycles_in": {n: int(st[i]) for i, n in enumerate(names) if n}}
+        rows.append(row)
+
+    for (M, N, K) in [(2048, 2048, 2048), (2048, 2048, 8192)]:
+        Wq = torch.randint(-127, 128, (N, K), dtype=torch.int8, device=dev, generator=g)
+        Ws = (torch.randn((N, K // 32), device=dev, generator=g).abs() * (0.02 / 127)).to(torch.float16)
+        A = torch.randn((M, K), device=dev, generator=g).to(torch.bfloat16)
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+        measure(f"dense Q8 {M}x{N}x{K}", lambda: qg.qgemm_dense(8, A, Wq, Ws, out=out), K // 64)
+    H, F, k, E, M = MOE["H"], MOE["F"], MOE["k"], MOE["E"], 2048
+    W1q = torch.randint(0, 256, (E, 2 * F, H // 2), dtype=torch.uint8, device=dev, generator=g)
+    W2q = torch.randint(0, 256, (E, H, F // 2), dtype=torch.uint8, device=dev, generator=g)
+    W1s = (torch.randn((E, 2 * F, H // 32), device=dev, generator=g).abs() * (0.02 / 7)).to(torch.float16)
+    W2s = (torch.randn((E, H, F // 32), device=dev, generator=g).abs() * (0.02 / 7)).to(torch.float16)
+    L = torch.randn((M, E), device=dev, generator=g)
+    X = torch.randn((M, H), device=dev, generator=g).to(torch.bfloat16)
+    r = qg.moe_route(L, k, X=X)
+    Hh = qg.moe_grouped_qgemm(qg.MODE_GATE_UP_SILU, 4, r["Xperm"], r["offsets"], W1q, W1s)
+    measure(f"MoE Q4 gate/up, {M} tokens, {E} experts", lambda: qg.moe_grouped_qgemm(
+        qg.MODE_GATE_UP_SILU, 4, r["Xperm"], r["offsets"], W1q, W1s, out=Hh), H // 64)
+    Dw = torch.empty((M * k, H), dtype=torch.bfloat16, device=dev)
+    measure(f"MoE Q4 down, {M} tokens, {E} experts", lambda: qg.moe_grouped_qgemm(
+        qg.MODE_DOWN_WEIGHTED, 4, Hh, r["offsets"], W2q, W2s, topk_w=r["topk_w"].view(-1), row_pair=r["row_pair"], k=k,
+        out=Dw), F // 64)
+    qg.poll_status()
+    print(json.dumps({"case": "roles", "rows": rows}, indent=1))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -896,11 +960,12 @@ def main():
     ap.add_argument("--moe-path", default="staged", choices=["fused", "staged"],
                     help="staged: permute, routing-weighted bf16 rows, slot-ordered combine (deterministic, faster on "
                          "B200); fused: token gather in the gate/up loads + fp32 accumulate in the down epilogue")
-    ap.add_argument("--case", default=None, choices=["moe_small", "attention", "small_m", "mx"],
+    ap.add_argument("--case", default=None, choices=["moe_small", "attention", "small_m", "mx", "roles"],
                     help="run one small case a few times and exit (for profiler captures): moe_small = the cfg-3 MoE "
                          "layer shape with 16 experts and 256 tokens (128 rows per expert); attention = cfg-4 heads "
                          "(32 / 8, d = 128) at 2048 positions; small_m = the cfg-4 gate/up weights (28672 x 4096, Q8) "
-                         "times 4 tokens; mx = the block-scaled FP8 GEMM 2048 x 16384 x 2048")
+                         "times 4 tokens; mx = the block-scaled FP8 GEMM 2048 x 16384 x 2048; roles = per-role wait cycles of the "
+                         "GEMM kernel from a -DQG_PROFILE build of the library (not a profiler target)")
     args = ap.parse_args()
     if args.case:
         run_case(args)

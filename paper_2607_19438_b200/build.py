@@ -33,6 +33,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+PROFILE_LIB = os.path.join(HERE, "libqgemm_b200_prof.so")
+
+
+def build_profile(force: bool = False) -> str:
+    """The same library with -DQG_PROFILE: the GEMM kernel's roles add up the cycles they spend in each of their waits
+    (read back with qg_debug_set_stats).  Slower than the product build; used by `bench.py --case roles` only."""
+    if force or not os.path.exists(PROFILE_LIB) or os.path.getmtime(PROFILE_LIB) < os.path.getmtime(build()):
+        subprocess.check_call([NVCC] + FLAGS + ["-DQG_PROFILE", "-o", PROFILE_LIB] + sources())
+    return PROFILE_LIB
+
+
 if __name__ == "__main__":
     import sys
     print(build(force=True, verbose="-v" in sys.argv))
+    if "--profile" in sys.argv:
+        print(build_profile(force=True))
