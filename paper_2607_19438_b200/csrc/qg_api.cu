@@ -141,7 +141,7 @@ int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, in
     for (int i = 0; i < ctx->tmap_count; ++i) {
         const TmapEntry& e = ctx->tmaps[i];
         if (e.base == base && e.inner == inner && e.rows == rows && e.box_inner == box_inner && e.box_rows == box_rows &&
-            e.row_stride == row_stride_bytes &&
+            e.row_stride == row_stride_bytes && e.planes == 0 &&
             e.dt == static_cast<int>(dt) && e.elem_bytes == elem_bytes && e.swz == static_cast<int>(swz)) {
             *out = &e.map;
             return QG_OK;
@@ -158,6 +158,40 @@ int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, in
                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return QG_ERR_CUDA;
     e.base = base; e.inner = inner; e.rows = rows; e.row_stride = row_stride_bytes; e.box_inner = box_inner; e.box_rows = box_rows;
+    e.planes = 0; e.plane_stride = 0; e.box_planes = 0;
+    e.dt = static_cast<int>(dt); e.elem_bytes = elem_bytes; e.swz = static_cast<int>(swz);
+    *out = &e.map;
+    ctx->tmap_next = (ctx->tmap_next + 1) % TMAP_CACHE;
+    if (ctx->tmap_count < TMAP_CACHE) ++ctx->tmap_count;
+    return QG_OK;
+}
+
+int get_tmap_3d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
+                uint64_t inner, uint64_t rows, uint64_t planes, uint64_t plane_stride_bytes, uint32_t box_inner,
+                uint32_t box_rows, uint32_t box_planes, CUtensorMapSwizzle swz) {
+    const uint64_t row_stride_bytes = inner * static_cast<uint64_t>(elem_bytes);
+    for (int i = 0; i < ctx->tmap_count; ++i) {
+        const TmapEntry& e = ctx->tmaps[i];
+        if (e.base == base && e.inner == inner && e.rows == rows && e.box_inner == box_inner && e.box_rows == box_rows &&
+            e.row_stride == row_stride_bytes && e.planes == planes && e.plane_stride == plane_stride_bytes &&
+            e.box_planes == box_planes &&
+            e.dt == static_cast<int>(dt) && e.elem_bytes == elem_bytes && e.swz == static_cast<int>(swz)) {
+            *out = &e.map;
+            return QG_OK;
+        }
+    }
+    TmapEntry& e = ctx->tmaps[ctx->tmap_next];
+    cuuint64_t dims[3] = {inner, rows, planes};
+    cuuint64_t strides[2] = {row_stride_bytes, plane_stride_bytes};
+    cuuint32_t box[3] = {box_inner, box_rows, box_planes};
+    cuuint32_t estr[3] = {1, 1, 1};
+    e.base = nullptr;      // not a valid entry while it is being rewritten
+    CUresult r = ctx->encode_tiled(&e.map, dt, 3, const_cast<void*>(base), dims, strides, box, estr,
+                                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return QG_ERR_CUDA;
+    e.base = base; e.inner = inner; e.rows = rows; e.row_stride = row_stride_bytes; e.box_inner = box_inner; e.box_rows = box_rows;
+    e.planes = planes; e.plane_stride = plane_stride_bytes; e.box_planes = box_planes;
     e.dt = static_cast<int>(dt); e.elem_bytes = elem_bytes; e.swz = static_cast<int>(swz);
     *out = &e.map;
     ctx->tmap_next = (ctx->tmap_next + 1) % TMAP_CACHE;

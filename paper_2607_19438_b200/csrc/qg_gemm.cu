@@ -381,8 +381,15 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
     // barriers itself and, as soon as it knows the pair's first tile, sends the first four k-blocks of weights on
     // their way, so that they travel while the pair synchronises and the tile tables are built.
     bool w_pre_issued = false;
+    // One copy fetches this CTA's 128 weight rows of a k-block (or their scales): a 128-row box, or in gate/up mode a
+    // box of 64 rows x 2 planes of a 3-D map whose planes are the gate and the up halves of the experts' matrices.
+    auto load_w = [&](uint32_t dst, const CUtensorMap* tm, int x, int e, int wt, uint32_t bar) {
+        if constexpr (EPI == 1) tma_load_3d(dst, tm, x, wt * 64, 2 * e, bar);
+        else tma_load_2d(dst, tm, x, e * p.N + wt * 128, bar);
+    };
     if (warp == 2) {  // prefix[e] = pair tiles before expert e; prefix[E] = total
-        if (lane < C::SR) { mbar_init(r_full(lane), 1); mbar_init(r_empty(lane), 4); }
+        // one barrier pair per batch of four stages (the batch's first stage carries it): 16 converting warps release it
+        if (lane < C::SR) { mbar_init(r_full(lane), 1); mbar_init(r_empty(lane), 16); }
         fence_mbar_init();
         fence_proxy_async_smem();
         if (grouped) pdl_wait();
@@ -408,21 +415,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         if (!SK && pair < carry) {
             const Tile tl = decode_tile(pair, prefix, p, BT);
             const int wt = 2 * tl.pw + static_cast<int>(rank);
-            const int row_a = tl.e * p.N + wt * ((EPI == 1) ? 64 : 128);
-            const int row_b = row_a + ((EPI == 1) ? (p.N / 2) : 64);
             if (lane == 0) {
-                const uint32_t sd = sbase + C::OFF_SC;
+                mbar_arrive_expect_tx(r_full(0), 4 * C::RAW_BYTES + C::SC_BYTES);
+                load_w(sbase + C::OFF_SC, &tm_s, 0, tl.e, wt, r_full(0));
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    mbar_arrive_expect_tx(r_full(j), C::RAW_BYTES + (j == 0 ? C::SC_BYTES : 0));
-                    const uint32_t dst = sbase + C::OFF_RAW + j * C::RAW_BYTES;
-                    tma_load_2d(dst, &tm_w, j * C::RAW_ROW, row_a, r_full(j));
-                    tma_load_2d(dst + C::RAW_BYTES / 2, &tm_w, j * C::RAW_ROW, row_b, r_full(j));
-                    if (j == 0) {
-                        tma_load_2d(sd, &tm_s, 0, row_a, r_full(0));
-                        tma_load_2d(sd + C::SC_BYTES / 2, &tm_s, 0, row_b, r_full(0));
-                    }
-                }
+                for (int j = 0; j < 4; ++j)
+                    load_w(sbase + C::OFF_RAW + j * C::RAW_BYTES, &tm_w, j * C::RAW_ROW, tl.e, wt, r_full(0));
             }
             w_pre_issued = true;
         }
@@ -487,7 +485,6 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
         pc.kb0 = 0; pc.kb1 = nkb; pc.i0 = j * nkb; pc.nsrc = 0;
         return pc;
     };
-    constexpr bool gate_up = (EPI == 1);
 
     // Control warps walk their loops with all 32 lanes (converged) and keep the per-k-block instruction count small:
     // a lone thread retires only one dependent instruction every few cycles and an mbarrier round trip costs a few
@@ -561,33 +558,21 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
             const Tile tl = tile_at(jt);
             const Piece pc = piece_at(jt);
             const int wt = 2 * tl.pw + static_cast<int>(rank);
-            const int row_a = tl.e * p.N + wt * (gate_up ? 64 : 128);
-            const int row_b = row_a + (gate_up ? (p.N / 2) : 64);
             for (int kb = pc.kb0; kb < pc.kb1; kb += 4) {
                 QG_T0();
-                if (batches >= C::SR / 4) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (ok && !wait_bar<false>(r_empty(s + j), ph ^ 1u, abort_flag, p)) ok = false;
-                    if (!ok) break;
-                }
+                if (batches >= C::SR / 4 && !wait_bar<false>(r_empty(s), ph ^ 1u, abort_flag, p)) { ok = false; break; }
                 QG_ACC(1);
                 if (jt == 0 && kb == pc.kb0) { QG_MARK(8); }
                 const bool sent = (batches == 0 && w_pre_issued);       // the first batch left in the prologue
                 ++batches;
                 if (lane == 0 && !sent) {
-                    const uint32_t sd = sbase + C::OFF_SC + sg * C::SC_BYTES;
+                    // five copies and one barrier per batch: the 8 scales per row that cover these four k-blocks,
+                    // then the packed codes of each k-block
+                    mbar_arrive_expect_tx(r_full(s), 4 * C::RAW_BYTES + C::SC_BYTES);
+                    load_w(sbase + C::OFF_SC + sg * C::SC_BYTES, &tm_s, (kb >> 2) * 8, tl.e, wt, r_full(s));
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        mbar_arrive_expect_tx(r_full(s + j), C::RAW_BYTES + (j == 0 ? C::SC_BYTES : 0));
-                        const uint32_t dst = sbase + C::OFF_RAW + (s + j) * C::RAW_BYTES;
-                        tma_load_2d(dst, &tm_w, (kb + j) * C::RAW_ROW, row_a, r_full(s + j));
-                        tma_load_2d(dst + C::RAW_BYTES / 2, &tm_w, (kb + j) * C::RAW_ROW, row_b, r_full(s + j));
-                        if (j == 0) {   // the 8 scales per row that cover these four k-blocks
-                            tma_load_2d(sd, &tm_s, (kb >> 2) * 8, row_a, r_full(s));
-                            tma_load_2d(sd + C::SC_BYTES / 2, &tm_s, (kb >> 2) * 8, row_b, r_full(s));
-                        }
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        load_w(sbase + C::OFF_RAW + (s + j) * C::RAW_BYTES, &tm_w, (kb + j) * C::RAW_ROW, tl.e, wt, r_full(s));
                 }
                 __syncwarp();
                 if (++sg == C::NSB) sg = 0;
@@ -726,9 +711,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 if (++in2 == per_tile(t2)) { in2 = 0; ++t2; }
             }
             QG_T0();
-            // the scales of this group of four k-blocks arrive with the first of them (stage 0 or 4)
+            // the four k-blocks of a batch and their scales arrive on the barrier of the batch's first stage
             if (!wait_bar<false>(r_full((n % NB) << 2), phr, abort_flag, p)) break;
-            if (!wait_bar<false>(r_full(sr), phr, abort_flag, p)) break;
             QG_ACC(5);
             if (n == 0 && warp == 8) { QG_MARK(10); }
             const uint32_t raw = sbase + C::OFF_RAW + sr * C::RAW_BYTES + raw_row;
@@ -765,7 +749,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ C
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(r_empty(sr));             // the packed codes are in registers now
+            if (lane == 0) mbar_arrive(r_empty((n % NB) << 2));  // the packed codes are in registers now
             QG_ACC(7);
             // its TMEM stage (i % SA) is free once the MMAs of k-block i - SA have completed
             {
@@ -922,12 +906,19 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_ro
     // activations: a box of half a token tile, or of a single row when the rows are gathered four at a time
     int rc = get_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, x_rows, BK,
                          p.gather_k > 0 ? 1 : C::XH_ROWS, CU_TENSOR_MAP_SWIZZLE_128B);
+    // weights and scales: a box of this CTA's 128 rows; in gate/up mode 64 gate rows + 64 up rows, as two planes of a
+    // 3-D view (k, row within a half, half of an expert's matrix)
+    const uint64_t kbytes = (QBITS == 8) ? p.K : p.K / 2;
+    const CUtensorMapSwizzle wswz = (QBITS == 8) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
     if (rc == QG_OK)
-        rc = get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, (QBITS == 8) ? p.K : p.K / 2, wrows,
-                         C::RAW_ROW, 64, (QBITS == 8) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+        rc = (EPI == 1) ? get_tmap_3d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, kbytes, p.N / 2, 2ull * p.E,
+                                      kbytes * (p.N / 2), C::RAW_ROW, 64, 2, wswz)
+                        : get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, kbytes, wrows, C::RAW_ROW, 128, wswz);
     if (rc == QG_OK)
-        rc = get_tmap_2d(ctx, &tm_s, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, Ws, p.K / 32, wrows, 8, 64,
-                         CU_TENSOR_MAP_SWIZZLE_NONE);
+        rc = (EPI == 1) ? get_tmap_3d(ctx, &tm_s, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, Ws, p.K / 32, p.N / 2, 2ull * p.E,
+                                      static_cast<uint64_t>(p.K / 32) * 2 * (p.N / 2), 8, 64, 2, CU_TENSOR_MAP_SWIZZLE_NONE)
+                        : get_tmap_2d(ctx, &tm_s, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, Ws, p.K / 32, wrows, 8, 128,
+                                      CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc != QG_OK) return rc;
     auto kern = qgemm_kernel<QBITS, BT, EPI, SK>;
     // the shared-memory attribute belongs to the function on one device: set once per context and instantiation

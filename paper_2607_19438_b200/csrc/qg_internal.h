@@ -14,6 +14,8 @@ struct TmapEntry {
     const void* base;
     uint64_t inner, rows, row_stride;
     uint32_t box_inner, box_rows;
+    uint64_t planes, plane_stride;   // third dimension of a 3-D map (0 for 2-D maps)
+    uint32_t box_planes;
     int dt, elem_bytes, swz;
     CUtensorMap map;
 };
@@ -70,4 +72,9 @@ int check_device(const qg_ctx* ctx);
 int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
                 uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz,
                 uint64_t row_stride_bytes = 0);
+// The same with a third dimension: `planes` planes of `rows` rows, plane_stride_bytes apart; box = box_inner x box_rows x
+// box_planes, which lands in shared memory plane after plane.
+int get_tmap_3d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
+                uint64_t inner, uint64_t rows, uint64_t planes, uint64_t plane_stride_bytes, uint32_t box_inner,
+                uint32_t box_rows, uint32_t box_planes, CUtensorMapSwizzle swz);
 }  // namespace qg
