@@ -255,6 +255,32 @@ void orc_combine(int64_t M, int k, int64_t H, const double* D, const int32_t* pa
         }
 }
 
+// --- router logits: L[t][e] = sum_{h ascending} X[t][h] * Wr[e][h] (both already widened to double). ---
+void orc_router_logits(int64_t M, int64_t H, int64_t E, const double* X, const double* Wr, double* L) {
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < M; ++t)
+        for (int64_t e = 0; e < E; ++e) {
+            double acc = 0.0;
+            for (int64_t h = 0; h < H; ++h) acc += X[t * H + h] * Wr[e * H + h];
+            L[t * E + e] = acc;
+        }
+}
+
+// --- combine with a shared expert: the routed sum in slot order, then the shared expert's row. ---
+void orc_combine_shared(int64_t M, int k, int64_t H, const double* D, const int32_t* pair_row, const double* w,
+                        const double* shared, double* y) {
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < M; ++t)
+        for (int64_t c = 0; c < H; ++c) {
+            double acc = 0.0;
+            for (int s = 0; s < k; ++s) {
+                const double d = D[static_cast<int64_t>(pair_row[t * k + s]) * H + c];
+                acc += (w ? w[t * k + s] : 1.0) * d;
+            }
+            y[t * H + c] = acc + shared[t * H + c];
+        }
+}
+
 // ---- MX (block-scaled FP8) reference ------------------------------------------------------------------------------
 // Value of an E4M3 code: sign, 4 exponent bits (bias 7), 3 mantissa bits; exponent 0 is subnormal (m / 8 * 2^-6);
 // exponent 15 with mantissa 7 is NaN, every other code is finite (so 0x7E = 448 is the largest).

@@ -168,6 +168,27 @@ def combine(D, pair_row, k, w=None):
     return y
 
 
+def combine_shared(D, pair_row, k, shared, w=None):
+    """combine() plus the shared expert's output row (a dense FFN every token passes through), added last."""
+    D, pair_row, shared = _c(D, np.float64), _c(pair_row, np.int32), _c(shared, np.float64)
+    M = pair_row.size // k
+    H = D.shape[1]
+    y = np.empty((M, H), np.float64)
+    wp = _p(_c(w, np.float64)) if w is not None else None
+    lib().orc_combine_shared(C.c_int64(M), C.c_int(k), C.c_int64(H), _p(D), _p(pair_row), wp, _p(shared), _p(y))
+    return y
+
+
+def router_logits(X, Wr):
+    """Router projection (hidden -> experts) that feeds route(): L = X Wr^T, X [M, H] and Wr [E, H] as doubles."""
+    X, Wr = _c(X, np.float64), _c(Wr, np.float64)
+    M, H = X.shape
+    E = Wr.shape[0]
+    L = np.empty((M, E), np.float64)
+    lib().orc_router_logits(C.c_int64(M), C.c_int64(H), C.c_int64(E), _p(X), _p(Wr), _p(L))
+    return L
+
+
 def moe_layer(qbits, logits, X, W1q, W1s, W2q, W2s, k):
     """End-to-end MoE layer with no intermediate rounding; returns a dict of every stage."""
     E = logits.shape[1]

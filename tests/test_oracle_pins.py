@@ -278,6 +278,33 @@ def test_combine_definition():
     assert orc.combine(D, pair_row, 2).tolist() == [[6.0, 8.0], [12.0, 14.0], [12.0, 14.0]]
 
 
+def test_combine_shared_adds_the_shared_row_last():
+    """Hand case: the routed sums of test_combine_definition plus a shared row; a zero shared expert changes nothing;
+    with no routed weight (w = 0) the result is the shared row itself."""
+    D = np.arange(12, dtype=np.float64).reshape(6, 2)
+    pair_row = np.array([3, 0, 5, 1, 2, 4], np.int32)
+    w = np.array([[0.5, 0.5], [1.0, 0.0], [0.25, 0.75]])
+    shared = np.array([[100.0, -1.0], [0.5, 0.25], [-7.0, 2.0]])
+    y = orc.combine_shared(D, pair_row, 2, shared, w)
+    assert y.tolist() == [[3.0 + 100.0, 4.0 - 1.0], [10.5, 11.25], [7.0 - 7.0, 8.0 + 2.0]]
+    assert np.array_equal(orc.combine_shared(D, pair_row, 2, np.zeros((3, 2)), w), orc.combine(D, pair_row, 2, w))
+    assert np.array_equal(orc.combine_shared(D, pair_row, 2, shared, np.zeros((3, 2))), shared)
+
+
+def test_router_logits_definition():
+    """Hand case (a transposed operand or a swapped index gives other numbers), one-hot rows that pick out single
+    weights, and an fp64 library matmul on a ragged shape."""
+    X = np.array([[1.0, 2.0, 3.0], [0.0, -1.0, 0.5]])
+    Wr = np.array([[1.0, 0.0, 0.0], [0.0, 1.0, 1.0], [2.0, 2.0, 2.0], [-1.0, 0.5, 0.25]])
+    L = orc.router_logits(X, Wr)
+    assert L.tolist() == [[1.0, 5.0, 12.0, 0.75], [0.0, -0.5, -1.0, -0.375]]
+    rng = np.random.default_rng(3)
+    Wr = rng.standard_normal((7, 5))
+    assert np.array_equal(orc.router_logits(np.eye(5), Wr), Wr.T)
+    X = rng.standard_normal((33, 129)); Wr = rng.standard_normal((10, 129))
+    np.testing.assert_allclose(orc.router_logits(X, Wr), X @ Wr.T, rtol=1e-12, atol=1e-12)
+
+
 def test_one_hot_logits_select_one_expert():
     M, H, E, F, k = 6, 64, 4, 32, 2
     logits, X, W1q, W1s, W2q, W2s = synth.moe_problem(4, M, H, E, F, seed=8)
