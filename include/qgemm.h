@@ -247,6 +247,23 @@ int moe_grouped_qgemm_gather(qg_ctx* ctx, int mode, int qbits, int M, int R, int
 int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
                 const float* topk_w, void* Y, void* stream);
 
+/*
+ * Combine with a shared expert (the 35B-A3B family of Sec. 4 adds an always-active expert to the routed ones; the
+ * paper gives no formula, plain definition): as moe_combine, then the row shared[t, :] is added last, in fp32, before
+ * the single rounding to bf16.  shared bf16 [M, H] is the output of a dense feed-forward block over all tokens
+ * (qgemm_dense_gate_up_silu followed by qgemm_dense).  Errors as moe_combine; QG_ERR_NULL if shared is NULL.
+ */
+int moe_combine_shared(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
+                       const float* topk_w, const void* shared, void* Y, void* stream);
+
+/*
+ * Router projection (Sec. 3.2 treats the router as the producer of the per-token expert scores; plain definition):
+ *   logits[t, e] = sum_h X[t, h] * Wr[e, h],  X bf16 [M, H], Wr bf16 [E, H] (router weights are not quantised),
+ *   logits f32 [M, E] row-major: the input of moe_route.  Products exact, fp32 sums in a fixed order (reproducible).
+ * All pointers device, 16-byte aligned (X, Wr).  H % 64 == 0, H >= 64, E >= 1, else QG_ERR_SHAPE; M == 0 is a no-op.
+ */
+int moe_router_logits(qg_ctx* ctx, int M, int H, int E, const void* X, const void* Wr, float* logits, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

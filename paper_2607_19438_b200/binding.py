@@ -21,7 +21,8 @@ D_BF16, D_F32_ACC = 0, 1
 EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_plan_dense", "qg_set_schedule", "qg_route_workspace_bytes",
            "qgemm_dense", "qgemm_small_m", "qgemm_dense_gate_up_silu", "prefill_attention",
            "qg_mx_scale_bytes", "qg_mx_quantize", "qg_mx_pack_weights", "qgemm_mx_dense",
-           "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_grouped_qgemm_gather", "moe_combine"]
+           "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_grouped_qgemm_gather", "moe_combine",
+           "moe_combine_shared", "moe_router_logits"]
 
 
 class QGemmError(RuntimeError):
@@ -68,6 +69,8 @@ def load():
         lib.moe_grouped_qgemm.argtypes = [vp, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, ci, vp, vp]
         lib.moe_grouped_qgemm_gather.argtypes = [vp, ci, ci, ci, ci, ci, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp]
         lib.moe_combine.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp, vp, vp]
+        lib.moe_combine_shared.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
+        lib.moe_router_logits.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
         _lib = lib
     return _lib
 
@@ -302,7 +305,8 @@ def moe_grouped_qgemm_gather(mode, qbits, X, row_pair, k, offsets, Wq, Wscale, t
     return out
 
 
-def moe_combine(D, pair_row, k, topk_w=None, d_kind=D_BF16, out=None):
+def moe_combine(D, pair_row, k, topk_w=None, d_kind=D_BF16, out=None, shared=None):
+    """shared (bf16 [M, H], the shared expert's output) is added last when given (moe_combine_shared)."""
     if d_kind == D_F32_ACC:
         M, H = D.shape
     else:
@@ -310,6 +314,20 @@ def moe_combine(D, pair_row, k, topk_w=None, d_kind=D_BF16, out=None):
         M = D.shape[0] // k
     if out is None:
         out = torch.empty((M, H), dtype=torch.bfloat16, device=D.device)
-    _check(load().moe_combine(context(), M, k, H, _ptr(D), d_kind, _ptr(pair_row), _ptr(topk_w), _ptr(out), _stream()),
-           "moe_combine")
+    if shared is None:
+        _check(load().moe_combine(context(), M, k, H, _ptr(D), d_kind, _ptr(pair_row), _ptr(topk_w), _ptr(out), _stream()),
+               "moe_combine")
+    else:
+        _check(load().moe_combine_shared(context(), M, k, H, _ptr(D), d_kind, _ptr(pair_row), _ptr(topk_w), _ptr(shared),
+                                         _ptr(out), _stream()), "moe_combine_shared")
+    return out
+
+
+def moe_router_logits(X, Wr, out=None):
+    """X bf16 [M, H], Wr bf16 [E, H] -> fp32 logits [M, E], the input of moe_route."""
+    M, H = X.shape
+    E = Wr.shape[0]
+    if out is None:
+        out = torch.empty((M, E), dtype=torch.float32, device=X.device)
+    _check(load().moe_router_logits(context(), M, H, E, _ptr(X), _ptr(Wr), _ptr(out), _stream()), "moe_router_logits")
     return out

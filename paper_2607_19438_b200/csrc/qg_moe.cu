@@ -221,7 +221,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // Y[t, :] = sum_s w(t, s) * D[pair_row[t k + s], :] in slot order; one block per token.
 __global__ void __launch_bounds__(256)
 combine_kernel(int M, int k, int H8, const int4* __restrict__ D, const int32_t* __restrict__ pair_row,
-               const float* __restrict__ topk_w, int4* __restrict__ Y) {
+               const float* __restrict__ topk_w, const int4* __restrict__ shared, int4* __restrict__ Y) {
     const int t = blockIdx.x;
     pdl_launch_dependents();
     pdl_wait();
@@ -245,6 +245,7 @@ combine_kernel(int M, int k, int H8, const int4* __restrict__ D, const int32_t* 
             for (int j = 0; j < 8; ++j)
                 if (row[j] >= 0) add8(acc, d[j], w[j]);
         }
+        if (shared) add8(acc, __ldg(shared + static_cast<size_t>(t) * H8 + v), 1.0f);    // the shared expert's row, last
         int4 o;
         o.x = pack_bf16x2(acc[0], acc[1]); o.y = pack_bf16x2(acc[2], acc[3]);
         o.z = pack_bf16x2(acc[4], acc[5]); o.w = pack_bf16x2(acc[6], acc[7]);
@@ -254,15 +255,17 @@ combine_kernel(int M, int k, int H8, const int4* __restrict__ D, const int32_t* 
 
 // Y = bf16(acc) for the f32 accumulator produced by the atomic-accumulate epilogue.
 __global__ void __launch_bounds__(256)
-round_f32_kernel(size_t n8, const float4* __restrict__ acc, int4* __restrict__ Y) {
+round_f32_kernel(size_t n8, const float4* __restrict__ acc, const int4* __restrict__ shared, int4* __restrict__ Y) {
     pdl_launch_dependents();
     pdl_wait();
     for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n8;
          i += static_cast<size_t>(gridDim.x) * blockDim.x) {
         const float4 a = acc[2 * i], b = acc[2 * i + 1];
+        float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        if (shared) add8(v, __ldg(shared + i), 1.0f);
         int4 o;
-        o.x = pack_bf16x2(a.x, a.y); o.y = pack_bf16x2(a.z, a.w);
-        o.z = pack_bf16x2(b.x, b.y); o.w = pack_bf16x2(b.z, b.w);
+        o.x = pack_bf16x2(v[0], v[1]); o.y = pack_bf16x2(v[2], v[3]);
+        o.z = pack_bf16x2(v[4], v[5]); o.w = pack_bf16x2(v[6], v[7]);
         Y[i] = o;
     }
 }
@@ -401,25 +404,38 @@ int moe_route_static(qg_ctx* ctx, int M, int E, int k, const float* logits, int3
                       H, qg::g_route_static_ptr[dev], stream);
 }
 
-int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
-                const float* topk_w, void* Y, void* stream) {
+static int combine_impl(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
+                        const float* topk_w, const void* shared, void* Y, void* stream) {
     if (!ctx) return QG_ERR_NULL;
     if (M < 0 || k < 1 || H < 8 || H % 8) return QG_ERR_SHAPE;
     if (d_kind != QG_D_BF16 && d_kind != QG_D_F32_ACC) return QG_ERR_SHAPE;
     if (M == 0) return QG_OK;
     if (!D || !Y) return QG_ERR_NULL;
-    if (!qg::aligned16(D) || !qg::aligned16(Y)) return QG_ERR_ALIGN;
+    if (!qg::aligned16(D) || !qg::aligned16(Y) || !qg::aligned16(shared)) return QG_ERR_ALIGN;
     if (const int rc = qg::check_device(ctx)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (d_kind == QG_D_F32_ACC) {
         const size_t n8 = static_cast<size_t>(M) * H / 8;
         const int blocks = static_cast<int>(min(static_cast<size_t>(ctx->sm_count) * 8, (n8 + 255) / 256));
         return qg::launch_rc(qg::launch_kernel(ctx, qg::round_f32_kernel, dim3(blocks), dim3(256), 0, st, n8,
-                                               static_cast<const float4*>(D), static_cast<int4*>(Y)));
+                                               static_cast<const float4*>(D), static_cast<const int4*>(shared),
+                                               static_cast<int4*>(Y)));
     }
     if (!pair_row) return QG_ERR_NULL;
     return qg::launch_rc(qg::launch_kernel(ctx, qg::combine_kernel, dim3(M), dim3(256), 0, st, M, k, H / 8,
-                                           static_cast<const int4*>(D), pair_row, topk_w, static_cast<int4*>(Y)));
+                                           static_cast<const int4*>(D), pair_row, topk_w,
+                                           static_cast<const int4*>(shared), static_cast<int4*>(Y)));
+}
+
+int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
+                const float* topk_w, void* Y, void* stream) {
+    return combine_impl(ctx, M, k, H, D, d_kind, pair_row, topk_w, nullptr, Y, stream);
+}
+
+int moe_combine_shared(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, const int32_t* pair_row,
+                       const float* topk_w, const void* shared, void* Y, void* stream) {
+    if (M > 0 && !shared) return QG_ERR_NULL;
+    return combine_impl(ctx, M, k, H, D, d_kind, pair_row, topk_w, shared, Y, stream);
 }
 
 }  // extern "C"
