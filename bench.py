@@ -472,6 +472,19 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
                         "call_us": {lab: v[0] / n_it * 1e3 for lab, v in aggf.items()},
                         "gemms_tflops": gemm_fl / (gemm_ms_f * 1e-3) / 1e12,
                         "layer_tok_per_s": M * n_it / (tot_ms_f * 1e-3)}
+        if not skewed:
+            # the two pieces around the routed experts: router projection (hidden -> experts, bf16) and the combine that
+            # adds a shared expert's row; each repeated back to back (a few microseconds each: launch-bound figures)
+            Wr = (torch.randn((E, H), device=dev, generator=g) * 0.05).to(torch.bfloat16)
+            shared = torch.randn((M, H), device=dev, generator=g).to(torch.bfloat16)
+            windows.pop()
+            ex = timed_calls([("router_logits", 2.0 * M * H * E, 2.0 * M * H + 2.0 * E * H + 4.0 * M * E,
+                               lambda it: chk(lib.moe_router_logits(ctx, M, H, E, P(X), P(Wr), P(L), S), "router"))], n_it)
+            windows.pop()
+            ex2 = timed_calls([("combine_shared", 0.0, 2.0 * R * H + 4.0 * M * H, lambda it: chk(lib.moe_combine_shared(
+                ctx, M, k, H, P(o["Dw"]), qg.D_BF16, P(o["pair_row"]), None, P(shared), P(o["y"]), S), "combine shared"))], n_it)
+            row["router_and_shared_expert"] = {"router_logits_us": ex["router_logits"][0] / n_it * 1e3,
+                                               "combine_shared_us": ex2["combine_shared"][0] / n_it * 1e3}
         out["moe"].append(row)
     out["_windows"] = windows
     return out
