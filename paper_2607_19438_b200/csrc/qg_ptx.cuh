@@ -310,4 +310,41 @@ __device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// Four consecutive K = 16 steps in one statement (a lone thread is slow at address arithmetic, so the descriptors are
+// advanced inside it).  lo words: start address >> 4 plus the fixed fields; `hi` is shared by all descriptors.
+// Both operands in shared memory, K-major with 128-byte swizzle: 16 k further is +2 in 16-byte units.
+__device__ __forceinline__ void umma_ss_x4(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                           uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a0, a1, a2, a3, b0, b1, b2, b3;\n\t.reg .b32 x1, x2, x3, y1, y2, y3;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, %5, %5;\n\t"
+        "add.u32 x1, %1, 2;\n\tadd.u32 x2, %1, 4;\n\tadd.u32 x3, %1, 6;\n\t"
+        "add.u32 y1, %2, 2;\n\tadd.u32 y2, %2, 4;\n\tadd.u32 y3, %2, 6;\n\t"
+        "mov.b64 a0, {%1, %3};\n\tmov.b64 a1, {x1, %3};\n\tmov.b64 a2, {x2, %3};\n\tmov.b64 a3, {x3, %3};\n\t"
+        "mov.b64 b0, {%2, %3};\n\tmov.b64 b1, {y1, %3};\n\tmov.b64 b2, {y2, %3};\n\tmov.b64 b3, {y3, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a0, b0, %4, p0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %4, p1;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc0)
+        : "memory");
+}
+// A from tensor memory (8 columns of packed bf16 pairs per step), B in shared memory N-major: 16 k further is 2048
+// bytes (+128 in 16-byte units).
+__device__ __forceinline__ void umma_ts_x4(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                           uint32_t acc0) {
+    asm volatile(
+        "{\n\t.reg .pred p0, p1;\n\t.reg .b64 b0, b1, b2, b3;\n\t.reg .b32 x1, x2, x3, y1, y2, y3;\n\t"
+        "setp.ne.b32 p0, %5, 0;\n\tsetp.eq.b32 p1, %5, %5;\n\t"
+        "add.u32 x1, %1, 8;\n\tadd.u32 x2, %1, 16;\n\tadd.u32 x3, %1, 24;\n\t"
+        "add.u32 y1, %2, 128;\n\tadd.u32 y2, %2, 256;\n\tadd.u32 y3, %2, 384;\n\t"
+        "mov.b64 b0, {%2, %3};\n\tmov.b64 b1, {y1, %3};\n\tmov.b64 b2, {y2, %3};\n\tmov.b64 b3, {y3, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], b0, %4, p0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [x1], b1, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [x2], b2, %4, p1;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [x3], b3, %4, p1;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc0)
+        : "memory");
+}
+
 }  // namespace qg
