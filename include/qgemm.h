@@ -120,10 +120,11 @@ int qgemm_dense_gate_up_silu(qg_ctx* ctx, int qbits, int M, int F, int K, const 
 /*
  * The same product for 1 <= M <= 16 tokens (else QG_ERR_SHAPE): the decode-side and small verification-batch
  * regime that Sec. 2.3 describes as bound by memory bandwidth and Sec. 5.2 names as future work for the tensor
- * path.  Every weight byte is used once, so this kernel streams the packed weights at HBM speed and reduces its
- * K slices in a fixed order (results do not depend on scheduling).  Same formats, constraints and numerics
- * (weights rounded once to bf16, fp32 accumulate) as qgemm_dense; uses the context's scratch, so calls on one
- * context must not overlap on the GPU.
+ * path.  Every weight byte is used once, so this call streams the packed weights: matrices below about 48 M weights
+ * (and fewer than 16384 rows) by a kernel of its own that reduces its K slices in a fixed order (results do not depend
+ * on scheduling), larger ones by qgemm_dense's kernel, which is faster there (and whose last bf16 place may differ
+ * between runs, see qgemm_dense).  Same formats, constraints and numerics (weights rounded once to bf16, fp32
+ * accumulate) as qgemm_dense; uses the context's scratch, so calls on one context must not overlap on the GPU.
  */
 int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq,
                   const void* Wscale, void* C, void* stream);

@@ -205,6 +205,9 @@ qgemv_kernel(const GemvParams p) {
 
 }  // namespace qg
 
+extern "C" int qgemm_dense(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq, const void* Wscale,
+                           void* Cout, void* stream);
+
 extern "C" int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq,
                              const void* Wscale, void* Cout, void* stream) {
     if (!ctx) return QG_ERR_NULL;
@@ -214,6 +217,12 @@ extern "C" int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const 
     if (!A || !Wq || !Wscale || !Cout) return QG_ERR_NULL;
     if (!qg::aligned16(A) || !qg::aligned16(Wq) || !qg::aligned16(Wscale) || !qg::aligned16(Cout)) return QG_ERR_ALIGN;
     if (const int rc = qg::check_device(ctx)) return rc;
+    // Large matrices go to the prefill kernel with its 128-token tile: once there are weight tiles for every SM pair
+    // (or K is long), its TMA-fed conversion pipeline streams the weights faster than this kernel's per-lane loads
+    // (measured at 1, 4 and 16 tokens, cold L2: 28672 x 4096 Q8 55 against 70 us, 16384 x 3072 Q4 27 against 39 us,
+    // 4096 x 14336 Q8 38 against 48 us; below about 48 M weights this kernel wins, e.g. 8192 x 4096 Q8 25 against 28).
+    if (static_cast<long long>(N) * K >= (48LL << 20) || N >= 16384)
+        return qgemm_dense(ctx, qbits, M, N, K, A, Wq, Wscale, Cout, stream);
     const int tiles = (N + qg::GV_ROWS - 1) / qg::GV_ROWS;
     // K slice: halved while that raises the block count towards three blocks per SM, with at most eight slices
     int KS = qg::GV_MAX_KS;

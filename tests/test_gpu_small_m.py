@@ -72,3 +72,16 @@ def test_small_m_extreme_scales_and_argument_checks():
         qg.qgemm_small_m(qbits, A17, util.dev(Wq), util.dev_f16(Ws))
     assert e.value.code == -2
     assert qg.qgemm_small_m(qbits, A17[:0], util.dev(Wq), util.dev_f16(Ws)).shape == (0, N)
+
+
+@pytest.mark.parametrize("qbits,M,N,K", [(8, 4, 16384, 2048), (4, 16, 6144, 8192), (8, 1, 4096, 14336)],
+                         ids=["q8-many-rows", "q4-48M-weights", "q8-long-k"])
+def test_small_m_large_matrices_take_the_prefill_kernel(qbits, M, N, K):
+    """At 16384 rows or 48 M weights and more the call is served by qgemm_dense's kernel (same numerics; the last bf16
+    place may differ between runs, so only the oracle comparison and the guards are asserted)."""
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=7)
+    g = util.Guarded((M, N), torch.bfloat16)
+    qg.qgemm_small_m(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws), out=g.t)
+    qg.poll_status()
+    assert g.intact() and not bool(g.untouched_inside().any().item())
+    util.assert_close(util.host_bf16_f64(g.t), orc.qgemm_dense(qbits, A, Wq, Ws), f"small-M via prefill kernel q{qbits} {M}x{N}x{K}")
