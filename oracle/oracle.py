@@ -248,3 +248,15 @@ def mx_gemm(a, asf, w, wsf):
     out = np.empty((M, N), np.float64)
     lib().orc_mx_gemm(C.c_int64(M), C.c_int64(N), C.c_int64(K), _p(a), _p(asf), _p(w), _p(wsf), _p(out))
     return out
+
+
+def mx_grouped_gemm(a, asf, offsets, w, wsf):
+    """mx_gemm per expert segment: rows offsets[e] .. offsets[e+1] of (a, asf) against expert e's (w[e], wsf[e])."""
+    a, asf = _c(a, np.uint8), _c(asf, np.uint8)
+    E, N = w.shape[0], w.shape[1]
+    out = np.zeros((a.shape[0], N), np.float64)
+    for e in range(E):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        if hi > lo:
+            out[lo:hi] = mx_gemm(a[lo:hi], asf[lo:hi], w[e], wsf[e])
+    return out

@@ -152,6 +152,13 @@ def mx_scale_tiles(plain: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(t.transpose(0, 3, 2, 1, 4)).reshape(-1)    # [tile, chunk, r, q, c]
 
 
+def mx_scale_tiles_grouped(plain: np.ndarray, offsets: np.ndarray) -> np.ndarray:
+    """mx_scale_tiles per expert segment: the rows of segment e (offsets[e] .. offsets[e+1]) are tiled on their own, so a
+    segment's tiles start at its first row; the tiles of all segments follow one another (empty segments have none)."""
+    parts = [mx_scale_tiles(plain[offsets[e]:offsets[e + 1]]) for e in range(len(offsets) - 1) if offsets[e + 1] > offsets[e]]
+    return np.concatenate(parts) if parts else np.zeros(0, np.uint8)
+
+
 def mx_scale_plain(tiles: np.ndarray, rows: int, K: int) -> np.ndarray:
     """Inverse of mx_scale_tiles."""
     kb = K // 32

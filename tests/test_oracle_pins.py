@@ -440,3 +440,22 @@ def test_mx_gemm_against_library_matmul_and_scale_tiling_roundtrip():
     tiles = synth.mx_scale_tiles(plain)
     assert tiles.size == 384 * 8 and np.array_equal(synth.mx_scale_plain(tiles, 300, 256), plain)
     assert tiles[100] == plain[38, 0] and tiles[511] == plain[127, 3] and tiles[512 + 17] == plain[1, 5]
+
+
+def test_mx_grouped_gemm_is_the_per_segment_product():
+    """Two experts with different weights: each output row equals the dense MX product of its row with its own expert's
+    weights (checked against mx_gemm on single rows), an empty expert contributes nothing, and the grouped scale tiling
+    restarts at every segment (the first row of segment 1 sits at row 0 of a new tile)."""
+    rng = np.random.default_rng(11)
+    K, N = 128, 5
+    offsets = np.array([0, 3, 3, 7], np.int32)
+    a, asf = orc.mx_quantize(rng.standard_normal((7, K)))
+    w = np.zeros((3, N, K), np.uint8); wsf = np.zeros((3, N, K // 32), np.uint8)
+    for e in range(3):
+        w[e], wsf[e] = orc.mx_quantize(rng.standard_normal((N, K)) * (e + 1))
+    out = orc.mx_grouped_gemm(a, asf, offsets, w, wsf)
+    for r, e in [(0, 0), (2, 0), (3, 2), (6, 2)]:
+        assert np.array_equal(out[r], orc.mx_gemm(a[r:r + 1], asf[r:r + 1], w[e], wsf[e])[0])
+    tiles = synth.mx_scale_tiles_grouped(asf, offsets)
+    assert tiles.size == 2 * 512                               # one tile per non-empty segment
+    assert tiles[512 + 0 * 16 + 0 * 4 + 1] == asf[3, 1] and tiles[2 * 16 + 3] == asf[2, 3]
