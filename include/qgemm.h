@@ -249,6 +249,29 @@ int moe_combine(qg_ctx* ctx, int M, int k, int H, const void* D, int d_kind, con
                 const float* topk_w, void* Y, void* stream);
 
 /*
+ * The expert projections over block-scaled FP8 operands (no counterpart in the paper; format, re-encoding rule and
+ * accuracy class as for qgemm_mx_dense).  At about 128 rows per expert moe_grouped_qgemm runs at the rate at which the
+ * expert weights can be converted to bf16; here nothing is converted.
+ *
+ * qg_mx_quantize_grouped re-encodes the sorted rows X bf16 [R, K] (segment e = rows expert_offsets[e] ..
+ * expert_offsets[e+1], E <= 1024 segments): codes [R, K] in row order, scale tiles laid out per segment (tile layout of
+ * qg_mx_quantize; a segment's first row is row 0 of a tile, the tiles of all non-empty segments follow one another; tile
+ * rows past the end of a segment hold the byte 0).  `scales` needs qg_mx_grouped_scale_bytes(R, E, K) bytes, an upper
+ * bound.  The expert weights [E, N, K] are packed by qg_mx_pack_weights with E * N rows.
+ *
+ * moe_grouped_qgemm_mx: Out as in moe_grouped_qgemm for mode QG_MODE_PLAIN, QG_MODE_GATE_UP_SILU (N = 2F, F % 64 == 0) or
+ * QG_MODE_DOWN_WEIGHTED (needs topk_w and row_pair), from the products
+ *   sum_k a[r, k] 2^(sa[r, k/32] - 127) * w_e[n, k] 2^(sw_e[n, k/32] - 127), fp32 accumulation in a fixed order, one
+ * rounding to bf16.  K % 128 == 0, N % 64 == 0, else QG_ERR_SHAPE; all pointers device, 16-byte aligned.
+ */
+size_t qg_mx_grouped_scale_bytes(int R, int E, int K);
+int qg_mx_quantize_grouped(qg_ctx* ctx, int R, int E, int K, const void* X, const int32_t* expert_offsets, void* codes,
+                           void* scales, void* stream);
+int moe_grouped_qgemm_mx(qg_ctx* ctx, int mode, int R, int E, int N, int K, const void* A_codes, const void* A_scales,
+                         const int32_t* expert_offsets, const void* W_codes, const void* W_scales, const float* topk_w,
+                         const int32_t* row_pair, void* Out, void* stream);
+
+/*
  * Combine with a shared expert (the 35B-A3B family of Sec. 4 adds an always-active expert to the routed ones; the
  * paper gives no formula, plain definition): as moe_combine, then the row shared[t, :] is added last, in fp32, before
  * the single rounding to bf16.  shared bf16 [M, H] is the output of a dense feed-forward block over all tokens

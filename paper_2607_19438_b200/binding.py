@@ -22,7 +22,8 @@ EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_
            "qgemm_dense", "qgemm_small_m", "qgemm_dense_gate_up_silu", "prefill_attention",
            "qg_mx_scale_bytes", "qg_mx_quantize", "qg_mx_pack_weights", "qgemm_mx_dense",
            "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_grouped_qgemm_gather", "moe_combine",
-           "moe_combine_shared", "moe_router_logits"]
+           "moe_combine_shared", "moe_router_logits",
+           "qg_mx_grouped_scale_bytes", "qg_mx_quantize_grouped", "moe_grouped_qgemm_mx"]
 
 
 class QGemmError(RuntimeError):
@@ -71,6 +72,10 @@ def load():
         lib.moe_combine.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp, vp, vp]
         lib.moe_combine_shared.argtypes = [vp, ci, ci, ci, vp, ci, vp, vp, vp, vp, vp]
         lib.moe_router_logits.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp]
+        lib.qg_mx_grouped_scale_bytes.restype = C.c_size_t
+        lib.qg_mx_grouped_scale_bytes.argtypes = [ci, ci, ci]
+        lib.qg_mx_quantize_grouped.argtypes = [vp, ci, ci, ci, vp, vp, vp, vp, vp]
+        lib.moe_grouped_qgemm_mx.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         _lib = lib
     return _lib
 
@@ -215,6 +220,28 @@ def qgemm_mx_dense(A_codes, A_sf, W_codes, W_sf, out=None):
         out = torch.empty((M, N), dtype=torch.bfloat16, device=A_codes.device)
     _check(load().qgemm_mx_dense(context(), M, N, K, _ptr(A_codes), _ptr(A_sf), _ptr(W_codes), _ptr(W_sf), _ptr(out),
                                  _stream()), "qgemm_mx_dense")
+    return out
+
+
+def mx_quantize_grouped(X, offsets):
+    """Sorted rows X bf16 [R, K], int32 offsets [E + 1] -> (codes uint8 [R, K], scale tiles laid out per segment)."""
+    R, K = X.shape
+    E = offsets.numel() - 1
+    codes = torch.empty((R, K), dtype=torch.uint8, device=X.device)
+    sf = torch.zeros(max(16, load().qg_mx_grouped_scale_bytes(R, E, K)), dtype=torch.uint8, device=X.device)
+    _check(load().qg_mx_quantize_grouped(context(), R, E, K, _ptr(X), _ptr(offsets), _ptr(codes), _ptr(sf), _stream()),
+           "qg_mx_quantize_grouped")
+    return codes, sf
+
+
+def moe_grouped_qgemm_mx(mode, A_codes, A_sf, offsets, W_codes, W_sf, N, topk_w=None, row_pair=None, out=None):
+    """A_codes uint8 [R, K] with per-segment scale tiles; W_codes uint8 [E * N, K] with scale tiles (mx_pack_weights)."""
+    R, K = A_codes.shape
+    E = offsets.numel() - 1
+    if out is None:
+        out = torch.empty((R, N // 2 if mode == MODE_GATE_UP_SILU else N), dtype=torch.bfloat16, device=A_codes.device)
+    _check(load().moe_grouped_qgemm_mx(context(), mode, R, E, N, K, _ptr(A_codes), _ptr(A_sf), _ptr(offsets), _ptr(W_codes),
+                                       _ptr(W_sf), _ptr(topk_w), _ptr(row_pair), _ptr(out), _stream()), "moe_grouped_qgemm_mx")
     return out
 
 

@@ -49,6 +49,85 @@ __device__ __forceinline__ size_t mx_scale_offset(int row, int block, int K) {
     return (static_cast<size_t>(t) * (K >> 7) + (block >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (block & 3);
 }
 
+// 32 values -> 32 E4M3 codes (two 16-byte stores) and the block's scale byte.
+__device__ __forceinline__ void mx_encode_block(const float (&x)[32], uint8_t* code_dst, uint8_t* sf_dst) {
+    float amax = 0.f;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) amax = fmaxf(amax, fabsf(x[t]));
+    const int e = mx_block_exponent(amax);
+    const float inv = __int_as_float((127 - e) << 23);        // 2^-e, exponent field 8 .. 254
+    uint32_t out[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+        out[t] = static_cast<uint32_t>(cvt_e4m3x2(x[4 * t] * inv, x[4 * t + 1] * inv)) |
+                 (static_cast<uint32_t>(cvt_e4m3x2(x[4 * t + 2] * inv, x[4 * t + 3] * inv)) << 16);
+    uint4* dst = reinterpret_cast<uint4*>(code_dst);
+    dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+    dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
+    *sf_dst = static_cast<uint8_t>(e + 127);
+}
+__device__ __forceinline__ void mx_load_bf16_block(const __nv_bfloat16* src, float (&x)[32]) {
+    const uint4* p = reinterpret_cast<const uint4*>(src);
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+        const uint4 u = p[v];
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            x[8 * v + 2 * t] = __uint_as_float(w[t] << 16);
+            x[8 * v + 2 * t + 1] = __uint_as_float(w[t] & 0xFFFF0000u);
+        }
+    }
+}
+
+// Rows sorted by expert (bf16 [R, K], segment e = rows offsets[e] .. offsets[e+1]): codes stay in row order, the scale
+// tiles are laid out per segment (a segment's first row is row 0 of a tile; tiles of all segments follow one another), so
+// that a 128-row token tile of a segment has its scales in one tile.  One thread per (tile slot row, 32-block); slot rows
+// past the end of their segment get the scale byte 0 (2^-127) and no codes.
+__global__ void __launch_bounds__(256)
+mx_quantize_grouped_kernel(int E, int K, const __nv_bfloat16* __restrict__ X, const int32_t* __restrict__ offsets,
+                           uint8_t* __restrict__ codes, uint8_t* __restrict__ sf) {
+    __shared__ int tile_base[1024 + 1];
+    pdl_launch_dependents();
+    pdl_wait();
+    if (threadIdx.x < 32) {
+        int carry = 0;
+        for (int e0 = 0; e0 < E; e0 += 32) {
+            const int e = e0 + threadIdx.x;
+            const int n = (e < E) ? (offsets[e + 1] - offsets[e] + 127) >> 7 : 0;
+            int inc = n;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (static_cast<int>(threadIdx.x) >= d) inc += o;
+            }
+            if (e < E) tile_base[e] = carry + inc - n;
+            carry += __shfl_sync(0xFFFFFFFFu, inc, 31);
+        }
+        if (threadIdx.x == 0) tile_base[E] = carry;
+    }
+    __syncthreads();
+    const int nb = K >> 5;
+    const long long total = static_cast<long long>(tile_base[E]) * 128 * nb;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int slot = static_cast<int>(i / nb), b = static_cast<int>(i - static_cast<long long>(slot) * nb);
+        const int t = slot >> 7;
+        int lo = 0, hi = E - 1;                          // last expert whose first tile is <= t (empty ones share it)
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (tile_base[mid] <= t) lo = mid; else hi = mid - 1;
+        }
+        const int local = ((t - tile_base[lo]) << 7) + (slot & 127);
+        const int row = offsets[lo] + local;
+        uint8_t* sfd = sf + mx_scale_offset(slot, b, K);
+        if (row >= offsets[lo + 1]) { *sfd = 0; continue; }
+        float x[32];
+        mx_load_bf16_block(X + static_cast<size_t>(row) * K + b * 32, x);
+        mx_encode_block(x, codes + static_cast<size_t>(row) * K + b * 32, sfd);
+    }
+}
+
 // SRC: 0 bf16 rows, 8 / 4 block-quantised weights (codes + fp16 scale).  One thread per (row, 32-block).
 template <int SRC>
 __global__ void __launch_bounds__(256)
@@ -67,17 +146,7 @@ mx_quantize_kernel(int rows, int rows_padded, int K, const void* __restrict__ sr
         }
         float x[32];
         if constexpr (SRC == 0) {
-            const uint4* p = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(src) + static_cast<size_t>(row) * K + b * 32);
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-                const uint4 u = p[v];
-                const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    x[8 * v + 2 * t] = __uint_as_float(w[t] << 16);
-                    x[8 * v + 2 * t + 1] = __uint_as_float(w[t] & 0xFFFF0000u);
-                }
-            }
+            mx_load_bf16_block(static_cast<const __nv_bfloat16*>(src) + static_cast<size_t>(row) * K + b * 32, x);
         } else if constexpr (SRC == 8) {
             const float s = __half2float(src_scale[static_cast<size_t>(row) * nb + b]);
             const uint4* p = reinterpret_cast<const uint4*>(static_cast<const int8_t*>(src) + static_cast<size_t>(row) * K + b * 32);
@@ -101,20 +170,7 @@ mx_quantize_kernel(int rows, int rows_padded, int K, const void* __restrict__ sr
                 for (int c = 0; c < 8; ++c)
                     x[8 * t + c] = static_cast<float>(static_cast<int>((w[t] >> (4 * c)) & 0xF) - 8) * s;
         }
-        float amax = 0.f;
-#pragma unroll
-        for (int t = 0; t < 32; ++t) amax = fmaxf(amax, fabsf(x[t]));
-        const int e = mx_block_exponent(amax);
-        const float inv = __int_as_float((127 - e) << 23);        // 2^-e, exponent field 8 .. 254
-        uint32_t out[8];
-#pragma unroll
-        for (int t = 0; t < 8; ++t)
-            out[t] = static_cast<uint32_t>(cvt_e4m3x2(x[4 * t] * inv, x[4 * t + 1] * inv)) |
-                     (static_cast<uint32_t>(cvt_e4m3x2(x[4 * t + 2] * inv, x[4 * t + 3] * inv)) << 16);
-        uint4* dst = reinterpret_cast<uint4*>(codes + static_cast<size_t>(row) * K + b * 32);
-        dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
-        dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
-        sf[mx_scale_offset(row, b, K)] = static_cast<uint8_t>(e + 127);
+        mx_encode_block(x, codes + static_cast<size_t>(row) * K + b * 32, sf + mx_scale_offset(row, b, K));
     }
 }
 
@@ -387,6 +443,27 @@ int qg_mx_quantize(qg_ctx* ctx, int rows, int K, const void* X, void* codes, voi
     if (!qg::aligned16(X) || !qg::aligned16(codes) || !qg::aligned16(scales)) return QG_ERR_ALIGN;
     if (const int rc = qg::check_device(ctx)) return rc;
     return qg::launch_quantize<0>(ctx, rows, K, X, nullptr, codes, scales, static_cast<cudaStream_t>(stream));
+}
+
+size_t qg_mx_grouped_scale_bytes(int R, int E, int K) {
+    if (R < 0 || E < 1 || K <= 0) return 0;
+    return (static_cast<size_t>((R + 127) / 128) + static_cast<size_t>(E)) * (K / 128) * 512;
+}
+
+int qg_mx_quantize_grouped(qg_ctx* ctx, int R, int E, int K, const void* X, const int32_t* expert_offsets, void* codes,
+                           void* scales, void* stream) {
+    if (!ctx) return QG_ERR_NULL;
+    if (R < 0 || E < 1 || E > 1024 || K < 128 || K % 128) return QG_ERR_SHAPE;
+    if (R == 0) return QG_OK;
+    if (!X || !expert_offsets || !codes || !scales) return QG_ERR_NULL;
+    if (!qg::aligned16(X) || !qg::aligned16(codes) || !qg::aligned16(scales)) return QG_ERR_ALIGN;
+    if (const int rc = qg::check_device(ctx)) return rc;
+    const long long slots = (static_cast<long long>((R + 127) / 128) + E) * 128 * (K / 32);     // upper bound
+    const long long want = (slots + 255) / 256, cap = static_cast<long long>(ctx->sm_count) * 16;
+    const int blocks = static_cast<int>(want < cap ? want : cap);
+    return qg::launch_rc(qg::launch_kernel(ctx, qg::mx_quantize_grouped_kernel, dim3(blocks), dim3(256), 0,
+                                           static_cast<cudaStream_t>(stream), E, K, static_cast<const __nv_bfloat16*>(X),
+                                           expert_offsets, static_cast<uint8_t*>(codes), static_cast<uint8_t*>(scales)));
 }
 
 int qg_mx_pack_weights(qg_ctx* ctx, int qbits, int N, int K, const void* Wq, const void* Wscale, void* codes, void* scales,
