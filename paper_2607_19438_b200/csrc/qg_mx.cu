@@ -175,7 +175,8 @@ mx_quantize_kernel(int rows, int rows_padded, int K, const void* __restrict__ sr
 }
 
 // ------------------------------------------------------------------------------------------------ GEMM
-// Persistent CTA pairs (cta_group::2).  A pair owns tiles of 256 tokens x 192 weight rows: each CTA stages its own 128
+// Persistent CTA pairs (cta_group::2).  A pair owns tiles of 256 tokens x 192 weight rows (256 in the one-wave shape, see
+// MxCfg; the figures below are for 192): each CTA stages its own 128
 // token rows (the MMA's A operand, M = 256 over the pair) and its half of the weight rows (B, 96 of N = 192), so a CTA
 // moves 28 KB per 128-k chunk for 128 x 192 x 128 products; two 192-column fp32 accumulators per CTA alternate between
 // the MMAs and the epilogue; the scale tiles of a chunk (one for this CTA's tokens, two for the weight rows) take 16
@@ -185,18 +186,26 @@ mx_quantize_kernel(int rows, int rows_padded, int K, const void* __restrict__ sr
 // of a chunk.  So the loads of a stage are spread over three warps (token codes, weight codes, scale tiles), and the
 // three scale copies and four MMAs of a chunk are one statement with the descriptors advanced inside it.  The ring has
 // seven stages: load latency + MMAs + commit are about 2200 cycles from the release of a stage to its next release.
-constexpr int MX_BM = 128, MX_BN = 192, MX_BK = 128, MX_ST = 7, MX_THREADS = 256;
-constexpr int MX_A_BYTES = MX_BM * MX_BK, MX_B_BYTES = (MX_BN / 2) * MX_BK, MX_SF_BYTES = 512;
-constexpr int MX_STAGE = MX_A_BYTES + MX_B_BYTES;                           // codes of a stage: 28 KB, 1024-byte aligned
+constexpr int MX_BM = 128, MX_BK = 128, MX_THREADS = 256, MX_A_BYTES = MX_BM * MX_BK, MX_SF_BYTES = 512;
 constexpr int MX_OFF_B = MX_A_BYTES;
 constexpr int MX_SF_STAGE = 3 * MX_SF_BYTES;                                // token tile, two weight tiles
-constexpr int MX_OFF_SF = MX_ST * MX_STAGE;
-constexpr int MX_LOADED = MX_STAGE + MX_SF_STAGE;                           // bytes one CTA receives per stage
-constexpr int MX_OFF_BAR = MX_OFF_SF + MX_ST * MX_SF_STAGE;
-constexpr int MX_NBAR = 2 * MX_ST + 4;                                      // full, empty, acc_full[2], acc_empty[2]
-constexpr int MX_SMEM = MX_OFF_BAR + MX_NBAR * 8 + 32 + 1024;
-constexpr int MX_COL_SF = 2 * MX_BN;               // scale columns: stage s at 384 + 16 s (4 for the tokens, 8 for the weights)
-static_assert(MX_STAGE % 1024 == 0 && MX_COL_SF + 16 * MX_ST <= 512 && MX_SMEM <= 232448, "budgets");
+// Two shapes: BN = 192 with two accumulators (the epilogue overlaps the next tile's main loop), and BN = 256 with one,
+// for problems whose 256 x 256 tiles fit into one wave of CTA pairs (nothing follows a pair's only tile, and the wider
+// tile needs a quarter fewer bytes per product).
+template <int BN>
+struct MxCfg {
+    static constexpr int NACC = (BN > 192) ? 1 : 2;
+    static constexpr int ST = (BN > 192) ? 6 : 7;
+    static constexpr int B_BYTES = (BN / 2) * MX_BK;
+    static constexpr int STAGE = MX_A_BYTES + B_BYTES;                      // codes of a stage, 1024-byte aligned
+    static constexpr int OFF_SF = ST * STAGE;
+    static constexpr int LOADED = STAGE + MX_SF_STAGE;                      // bytes one CTA receives per stage
+    static constexpr int OFF_BAR = OFF_SF + ST * MX_SF_STAGE;
+    static constexpr int NBAR = 2 * ST + 4;                                 // full, empty, acc_full[2], acc_empty[2]
+    static constexpr int SMEM = OFF_BAR + NBAR * 8 + 32 + 1024;
+    static constexpr int COL_SF = NACC * BN;        // scale columns: 16 per stage (4 for the tokens, 8 for the weights)
+    static_assert(STAGE % 1024 == 0 && COL_SF + 16 * ST <= 512 && SMEM <= 232448, "budgets");
+};
 
 struct MxParams {
     int M, N, K;
@@ -256,19 +265,21 @@ __device__ __forceinline__ void mx_chunk(uint32_t d_tmem, uint32_t a_lo, uint32_
 // the scale tiles as 32-bit words, one row per 128 matrix rows, 128 words per chunk (box = one tile / two tiles of
 // consecutive rows).  Everything outside a matrix reads as zero, and a
 // zero scale byte times zero codes contributes nothing, so ragged edges need no special case in the loads.
+template <int BN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MX_THREADS, 1)
 qgemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
                 const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ CUtensorMap tm_sw, const MxParams p) {
+    using C = MxCfg<BN>;
     extern __shared__ uint8_t smem_dyn[];
     const uint32_t sbase = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     uint8_t* sgen = smem_dyn + (sbase - smem_u32(smem_dyn));
-    volatile int* misc = reinterpret_cast<volatile int*>(sgen + MX_OFF_BAR + MX_NBAR * 8);     // [0] tmem base, [1] abort
+    volatile int* misc = reinterpret_cast<volatile int*>(sgen + C::OFF_BAR + C::NBAR * 8);     // [0] tmem base, [1] abort
     volatile int* abort_flag = misc + 1;
-    const uint32_t bar0 = sbase + MX_OFF_BAR;
+    const uint32_t bar0 = sbase + C::OFF_BAR;
     auto full = [&](uint32_t s) { return bar0 + 8u * s; };                              // even CTA only
-    auto empty = [&](uint32_t s) { return bar0 + 8u * (MX_ST + s); };                   // both CTAs
-    auto acc_full = [&](uint32_t a) { return bar0 + 8u * (2 * MX_ST + a); };
-    auto acc_empty = [&](uint32_t a) { return bar0 + 8u * (2 * MX_ST + 2 + a); };       // even CTA only
+    auto empty = [&](uint32_t s) { return bar0 + 8u * (C::ST + s); };                   // both CTAs
+    auto acc_full = [&](uint32_t a) { return bar0 + 8u * (2 * C::ST + a); };
+    auto acc_empty = [&](uint32_t a) { return bar0 + 8u * (2 * C::ST + 2 + a); };       // even CTA only
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
@@ -276,7 +287,7 @@ qgemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
 
     pdl_launch_dependents();
     if (warp == 0) {
-        if (lane < MX_NBAR) mbar_init(bar0 + 8u * lane, lane < MX_NBAR - 2 ? 1 : 8);     // acc_empty: 4 epilogue warps x 2 CTAs
+        if (lane < C::NBAR) mbar_init(bar0 + 8u * lane, lane < C::NBAR - 2 ? 1 : 8);     // acc_empty: 4 epilogue warps x 2 CTAs
         if (lane == 31) misc[1] = 0;
         fence_mbar_init();
         fence_proxy_async_smem();
@@ -284,7 +295,7 @@ qgemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         if (lane == 29) { prefetch_tmap(&tm_w); prefetch_tmap(&tm_sw); }
     }
     if (warp == 1) {
-        tmem_alloc(sbase + MX_OFF_BAR + MX_NBAR * 8, 512);
+        tmem_alloc(sbase + C::OFF_BAR + C::NBAR * 8, 512);
         tmem_relinquish();
     }
     tc_fence_before_sync();
@@ -307,58 +318,59 @@ qgemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         auto locate = [&]() {
             const int tm = t % p.tiles_m, tn = t / p.tiles_m;
             m0 = tm * 2 * MX_BM + static_cast<int>(rank) * MX_BM;
-            n0 = tn * MX_BN + static_cast<int>(rank) * (MX_BN / 2);      // this CTA's half of the weight rows
+            n0 = tn * BN + static_cast<int>(rank) * (BN / 2);      // this CTA's half of the weight rows
             sa_row = 2 * tm + static_cast<int>(rank);                    // this CTA's token scale tiles
-            sw_row = (tn * MX_BN) >> 7;                                  // first of the two weight scale tiles
+            sw_row = (tn * BN) >> 7;                                  // first of the two weight scale tiles
         };
         locate();
         uint32_t s = 0, ph = 0;
         for (uint32_t g = 0; g < total; ++g) {
-            if (g >= MX_ST && !mx_wait(empty(s), ph ^ 1u, abort_flag, p)) break;
+            if (g >= C::ST && !mx_wait(empty(s), ph ^ 1u, abort_flag, p)) break;
             if (lane == 0) {
                 const uint32_t fb = full_leader + 8u * s;
                 if (warp == 0) {
-                    if (rank == 0) mbar_arrive_expect_tx(full(s), 2u * MX_LOADED);
-                    tma_load_2d_pair(sbase + s * MX_STAGE, &tm_a, j * MX_BK, m0, fb);
+                    if (rank == 0) mbar_arrive_expect_tx(full(s), 2u * C::LOADED);
+                    tma_load_2d_pair(sbase + s * C::STAGE, &tm_a, j * MX_BK, m0, fb);
                 } else if (warp == 2) {
-                    tma_load_2d_pair(sbase + s * MX_STAGE + MX_OFF_B, &tm_w, j * MX_BK, n0, fb);
+                    tma_load_2d_pair(sbase + s * C::STAGE + MX_OFF_B, &tm_w, j * MX_BK, n0, fb);
                 } else {
-                    const uint32_t sf = sbase + MX_OFF_SF + s * MX_SF_STAGE;
+                    const uint32_t sf = sbase + C::OFF_SF + s * MX_SF_STAGE;
                     tma_load_2d_pair(sf, &tm_sa, j * 128, sa_row, fb);
                     tma_load_2d_pair(sf + MX_SF_BYTES, &tm_sw, j * 128, sw_row, fb);         // two tiles: rows sw_row, sw_row + 1
                 }
             }
             __syncwarp();
             if (++j == nch) { j = 0; t += npairs; locate(); }
-            if (++s == MX_ST) { s = 0; ph ^= 1u; }
+            if (++s == C::ST) { s = 0; ph ^= 1u; }
         }
     } else if (warp == 1) {
         // ------------------------------------------------ scale copies and MMAs (even CTA, for the pair)
         if (rank == 0) {
             const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);          // group stride, version, 128-byte swizzle
-            const uint32_t idesc0 = ((MX_BN >> 3) << 17) | (1u << 23) | (((2 * MX_BM) >> 4) << 24);
+            const uint32_t idesc0 = ((BN >> 3) << 17) | (1u << 23) | (((2 * MX_BM) >> 4) << 24);
             uint32_t s = 0, ph = 0, jt = 0;
             bool ok = true;
             for (int t = pair; t < p.tiles && ok; t += npairs, ++jt) {
-                const int n0 = (t / p.tiles_m) * MX_BN;
-                const uint32_t a = jt & 1u;
-                if (jt >= 2 && !mx_wait(acc_empty(a), ((jt >> 1) & 1u) ^ 1u, abort_flag, p)) { ok = false; break; }
-                const uint32_t d_tmem = tmem_base + a * MX_BN;
+                const int n0 = (t / p.tiles_m) * BN;
+                const uint32_t a = (C::NACC == 2) ? (jt & 1u) : 0u;
+                const uint32_t aph = (C::NACC == 2) ? ((jt >> 1) & 1u) : (jt & 1u);
+                if (jt >= static_cast<uint32_t>(C::NACC) && !mx_wait(acc_empty(a), aph ^ 1u, abort_flag, p)) { ok = false; break; }
+                const uint32_t d_tmem = tmem_base + a * BN;
                 // weight scale tiles at columns +4 .. +11 of the stage: the tile's first row is row n0 % 128 of the first
                 const uint32_t sfb_off = 4 + ((static_cast<uint32_t>(n0) & 127u) >> 5);
                 for (int j = 0; j < nch; ++j) {
                     if (!mx_wait(full(s), ph, abort_flag, p)) { ok = false; break; }
                     tc_fence_after_sync();
                     if (elect_one()) {
-                        const uint32_t st = sbase + s * MX_STAGE;
-                        const uint32_t sf_t = tmem_base + MX_COL_SF + 16 * s;
+                        const uint32_t st = sbase + s * C::STAGE;
+                        const uint32_t sf_t = tmem_base + C::COL_SF + 16 * s;
                         mx_chunk(d_tmem, (st >> 4) | (1u << 16), ((st + MX_OFF_B) >> 4) | (1u << 16), hi, idesc0, sf_t,
-                                 sf_t + sfb_off, j > 0 ? 1u : 0u, ((sbase + MX_OFF_SF + s * MX_SF_STAGE) >> 4) | (1u << 16));
+                                 sf_t + sfb_off, j > 0 ? 1u : 0u, ((sbase + C::OFF_SF + s * MX_SF_STAGE) >> 4) | (1u << 16));
                         mx_commit(empty(s));
                         if (j == nch - 1) mx_commit(acc_full(a));
                     }
                     __syncwarp();
-                    if (++s == MX_ST) { s = 0; ph ^= 1u; }
+                    if (++s == C::ST) { s = 0; ph ^= 1u; }
                 }
             }
         }
@@ -371,14 +383,14 @@ qgemm_mx_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         for (int t = pair; t < p.tiles; t += npairs, ++jt) {
             const int tm = t % p.tiles_m, tn = t / p.tiles_m;
             const int m = tm * 2 * MX_BM + static_cast<int>(rank) * MX_BM + row;
-            const int n0 = tn * MX_BN;
-            const uint32_t a = jt & 1u;
-            if (!mx_wait(acc_full(a), (jt >> 1) & 1u, abort_flag, p)) break;
+            const int n0 = tn * BN;
+            const uint32_t a = (C::NACC == 2) ? (jt & 1u) : 0u;
+            if (!mx_wait(acc_full(a), (C::NACC == 2) ? ((jt >> 1) & 1u) : (jt & 1u), abort_flag, p)) break;
             tc_fence_after_sync();
-            const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + a * MX_BN;
+            const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + a * BN;
             __nv_bfloat16* crow = p.C + static_cast<size_t>(m < p.M ? m : 0) * p.N + n0;
 #pragma unroll 1
-            for (int c = 0; c < MX_BN / 32; ++c) {
+            for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld_32x32(lane_addr + 32 * c, v);
                 tmem_ld_wait();
@@ -424,6 +436,40 @@ static int launch_quantize(qg_ctx* ctx, int rows, int K, const void* src, const 
     const int blocks = static_cast<int>(want < cap ? want : cap);
     return launch_rc(launch_kernel(ctx, mx_quantize_kernel<SRC>, dim3(blocks), dim3(256), 0, st, rows, rp, K, src,
                                    static_cast<const __half*>(src_scale), static_cast<uint8_t*>(codes), static_cast<uint8_t*>(sf)));
+}
+
+template <int BN>
+static int launch_mx_dense(qg_ctx* ctx, int M, int N, int K, const void* A_codes, const void* A_scales, const void* W_codes,
+                           const void* W_scales, void* Cout, void* stream) {
+    using C = MxCfg<BN>;
+    const CUtensorMap *tm_a, *tm_w, *tm_sa, *tm_sw;
+    const int nch = K / MX_BK;
+    int rc = get_tmap_2d(ctx, &tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, A_codes, K, M, MX_BK, MX_BM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc == QG_OK)
+        rc = get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W_codes, K, N, MX_BK, BN / 2, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc == QG_OK)
+        rc = get_tmap_2d(ctx, &tm_sa, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, A_scales, static_cast<uint64_t>(nch) * 128,
+                         static_cast<uint64_t>((M + 127) / 128), 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (rc == QG_OK)
+        rc = get_tmap_2d(ctx, &tm_sw, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, W_scales, static_cast<uint64_t>(nch) * 128,
+                         static_cast<uint64_t>((N + 127) / 128), 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (rc != QG_OK) return rc;
+    constexpr int inst = (BN == 192) ? 30 : 38;          // slots of the per-context "attribute set" flags
+    if (!ctx->attr_set[inst]) {
+        if (cudaFuncSetAttribute(qgemm_mx_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess) {
+            cudaGetLastError();
+            return QG_ERR_CUDA;
+        }
+        ctx->attr_set[inst] = true;
+    }
+    MxParams p{};
+    p.M = M; p.N = N; p.K = K;
+    p.tiles_m = (M + 2 * MX_BM - 1) / (2 * MX_BM);
+    p.tiles = p.tiles_m * ((N + BN - 1) / BN);
+    p.C = static_cast<__nv_bfloat16*>(Cout); p.status = ctx->d_status; p.wait_limit = ctx->wait_limit;
+    const int pairs = p.tiles < ctx->sm_count / 2 ? p.tiles : ctx->sm_count / 2;
+    return launch_rc(launch_kernel(ctx, qgemm_mx_kernel<BN>, dim3(2 * pairs), dim3(MX_THREADS), C::SMEM,
+                                   static_cast<cudaStream_t>(stream), *tm_a, *tm_w, *tm_sa, *tm_sw, p));
 }
 
 }  // namespace qg
@@ -490,36 +536,16 @@ int qgemm_mx_dense(qg_ctx* ctx, int M, int N, int K, const void* A_codes, const 
         !qg::aligned16(Cout))
         return QG_ERR_ALIGN;
     if (const int rc = qg::check_device(ctx)) return rc;
-    const CUtensorMap *tm_a, *tm_w, *tm_sa, *tm_sw;
     const int nch = K / qg::MX_BK;
-    int rc = qg::get_tmap_2d(ctx, &tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, A_codes, K, M, qg::MX_BK, qg::MX_BM,
-                             CU_TENSOR_MAP_SWIZZLE_128B);
-    if (rc == QG_OK)
-        rc = qg::get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W_codes, K, N, qg::MX_BK, qg::MX_BN / 2,
-                             CU_TENSOR_MAP_SWIZZLE_128B);
-    if (rc == QG_OK)
-        rc = qg::get_tmap_2d(ctx, &tm_sa, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, A_scales, static_cast<uint64_t>(nch) * 128,
-                             static_cast<uint64_t>((M + 127) / 128), 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE);
-    if (rc == QG_OK)
-        rc = qg::get_tmap_2d(ctx, &tm_sw, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, W_scales, static_cast<uint64_t>(nch) * 128,
-                             static_cast<uint64_t>((N + 127) / 128), 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE);
-    if (rc != QG_OK) return rc;
-    constexpr int inst = 30;
-    if (!ctx->attr_set[inst]) {
-        if (cudaFuncSetAttribute(qg::qgemm_mx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, qg::MX_SMEM) != cudaSuccess) {
-            cudaGetLastError();
-            return QG_ERR_CUDA;
-        }
-        ctx->attr_set[inst] = true;
-    }
-    qg::MxParams p{};
-    p.M = M; p.N = N; p.K = K;
-    p.tiles_m = (M + 2 * qg::MX_BM - 1) / (2 * qg::MX_BM);
-    p.tiles = p.tiles_m * ((N + qg::MX_BN - 1) / qg::MX_BN);
-    p.C = static_cast<__nv_bfloat16*>(Cout); p.status = ctx->d_status; p.wait_limit = ctx->wait_limit;
-    const int pairs = p.tiles < ctx->sm_count / 2 ? p.tiles : ctx->sm_count / 2;
-    return qg::launch_rc(qg::launch_kernel(ctx, qg::qgemm_mx_kernel, dim3(2 * pairs), dim3(qg::MX_THREADS), qg::MX_SMEM,
-                                           static_cast<cudaStream_t>(stream), *tm_a, *tm_w, *tm_sa, *tm_sw, p));
+    // Weight-tile width: modelled cycles of the busiest CTA pair (waves of tiles x (MMAs of a tile + the epilogue the
+    // single-accumulator shape leaves exposed)); the 256-wide tile wins when it saves a wave on a small problem.
+    const long long pairs_hw = ctx->sm_count / 2;
+    const long long tm = (M + 2 * qg::MX_BM - 1) / (2 * qg::MX_BM);
+    const long long t192 = tm * ((N + 191) / 192), t256 = tm * ((N + 255) / 256);
+    const double c192 = static_cast<double>((t192 + pairs_hw - 1) / pairs_hw) * (nch * 4.0 * 96.0);
+    const double c256 = static_cast<double>((t256 + pairs_hw - 1) / pairs_hw) * (nch * 4.0 * 128.0 + 3500.0);
+    if (c256 < c192) return qg::launch_mx_dense<256>(ctx, M, N, K, A_codes, A_scales, W_codes, W_scales, Cout, stream);
+    return qg::launch_mx_dense<192>(ctx, M, N, K, A_codes, A_scales, W_codes, W_scales, Cout, stream);
 }
 
 }  // extern "C"

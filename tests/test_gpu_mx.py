@@ -47,7 +47,8 @@ def test_pack_weights_bit_exact(qbits, N, K):
 
 # the last two give every CTA pair three or more tiles (both accumulators reused), one of them with a single chunk per tile
 SHAPES = [(128, 256, 128), (300, 392, 512), (1, 8, 128), (129, 264, 1024), (512, 2048, 2048), (2048, 2560, 2048),
-          (2048, 4224, 256), (1000, 9216, 128)]
+          (2048, 4224, 256), (1000, 9216, 128),
+          (2048, 2048, 2048), (1999, 2040, 2304)]       # one wave of 256-wide tiles: the single-accumulator shape
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES, ids=[f"{s[0]}x{s[1]}x{s[2]}" for s in SHAPES])
