@@ -35,6 +35,8 @@ CASES = [
     ("k1", 100, 8, 1, "uniform"), ("odd-E", 77, 5, 3, "ties"), ("E1024", 40, 1024, 8, "uniform"),
     ("k40", 65, 64, 40, "uniform"), ("one-token", 1, 128, 8, "uniform"), ("uniform-8192", 8192, 128, 8, "uniform"),
     ("extremes", 200, 96, 6, "extremes"),
+    # more histogram blocks than the scan kernel has warps, with a ragged last block
+    ("blocks-257", 8193, 16, 2, "skewed"), ("blocks-256-ragged", 8161, 24, 3, "ties"),
 ]
 
 
