@@ -407,7 +407,7 @@ static int launch_attn(qg_ctx* ctx, const AttnParams& p, const void* Q, long lon
                          CU_TENSOR_MAP_SWIZZLE_128B, static_cast<uint64_t>(ldv) * 2);
     if (rc != QG_OK) return rc;
     auto kern = attn_fwd_kernel<D>;
-    constexpr int inst = 20 + (D == 64 ? 0 : D == 128 ? 1 : 2);
+    constexpr int inst = ATTR_ATTN + (D == 64 ? 0 : D == 128 ? 1 : 2);
     if (!ctx->attr_set[inst]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
             cudaGetLastError();

@@ -922,8 +922,8 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_ro
     if (rc != QG_OK) return rc;
     auto kern = qgemm_kernel<QBITS, BT, EPI, SK>;
     // the shared-memory attribute belongs to the function on one device: set once per context and instantiation
-    constexpr int inst = SK ? 24 + ((QBITS == 4) ? 3 : 0) + ((BT == 128) ? 0 : (BT == 192) ? 1 : 2)
-                            : ((QBITS == 4) ? 9 : 0) + ((BT == 128) ? 0 : (BT == 192) ? 3 : 6) + EPI;
+    constexpr int inst = SK ? ATTR_GEMM_SK + ((QBITS == 4) ? 3 : 0) + ((BT == 128) ? 0 : (BT == 192) ? 1 : 2)
+                            : ATTR_GEMM + ((QBITS == 4) ? 9 : 0) + ((BT == 128) ? 0 : (BT == 192) ? 3 : 6) + EPI;
     if (!ctx->attr_set[inst]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess) {
             cudaGetLastError();

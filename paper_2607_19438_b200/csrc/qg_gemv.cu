@@ -242,7 +242,7 @@ extern "C" int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const 
     p.partial = ctx->gemv_partial; p.tickets = ctx->gemv_tickets;
     const size_t smem = static_cast<size_t>(16) * (KS + 8) * 2 + static_cast<size_t>(qg::GV_ROWS) * (KS / 32 + 2) * 2 + 16;
     auto kern = (qbits == QG_Q8) ? qg::qgemv_kernel<8> : qg::qgemv_kernel<4>;
-    const int inst = 18 + (qbits == QG_Q8 ? 0 : 1);
+    const int inst = qg::ATTR_GEMV + (qbits == QG_Q8 ? 0 : 1);
     if (!ctx->attr_set[inst]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  16 * (qg::GV_MAX_KS + 8) * 2 + qg::GV_ROWS * (qg::GV_MAX_KS / 32 + 2) * 2 + 16) != cudaSuccess) {

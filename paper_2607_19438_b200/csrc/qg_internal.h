@@ -21,6 +21,20 @@ struct TmapEntry {
 };
 constexpr int TMAP_CACHE = 64;
 constexpr uint32_t DEFAULT_WAIT_LIMIT = 1u << 18;   // polls; an unsatisfied try_wait poll lasts about 4 us: about a second
+// Slots of qg_ctx::attr_set, one per kernel instantiation that needs the dynamic shared-memory attribute.
+enum AttrSlot {
+    ATTR_GEMM = 0,          // 18 slots: format (2) x token tile (3) x epilogue (3)
+    ATTR_GEMV = 18,         // 2: Q8, Q4
+    ATTR_ATTN = 20,         // 3: head dimensions
+    ATTR_ROUTER_1 = 23,
+    ATTR_GEMM_SK = 24,      // 6: format (2) x token tile (3), stream-K
+    ATTR_MX_192 = 30,
+    ATTR_ROUTER_4 = 31,
+    ATTR_MX_MOE = 32,       // 2: down, gate/up
+    ATTR_MX_256 = 34,
+    ATTR_GEMV_RING = 35,    // 2: Q8, Q4
+    ATTR_SLOTS = 37
+};
 }  // namespace qg
 
 struct qg_ctx {
@@ -33,7 +47,7 @@ struct qg_ctx {
     int force_bt;              // QG_FORCE_BT at creation (0: heuristic)
     uint32_t wait_limit;       // polls per bounded device wait
     int skip_kb;               // test hook, consumed by the next GEMM launch (-1: none)
-    bool attr_set[32];         // per kernel instantiation: dynamic shared-memory attribute set on this device
+    bool attr_set[qg::ATTR_SLOTS];        // per kernel instantiation: dynamic shared-memory attribute set on this device
     qg::TmapEntry tmaps[qg::TMAP_CACHE];   // tensor maps of recent calls (weights and buffers recur every layer)
     int tmap_count, tmap_next;
     bool pdl;                  // launch kernels with programmatic stream serialization (QG_NO_PDL=1 turns it off)

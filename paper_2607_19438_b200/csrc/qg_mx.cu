@@ -454,7 +454,7 @@ static int launch_mx_dense(qg_ctx* ctx, int M, int N, int K, const void* A_codes
         rc = get_tmap_2d(ctx, &tm_sw, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, W_scales, static_cast<uint64_t>(nch) * 128,
                          static_cast<uint64_t>((N + 127) / 128), 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc != QG_OK) return rc;
-    constexpr int inst = (BN == 192) ? 30 : 38;          // slots of the per-context "attribute set" flags
+    constexpr int inst = (BN == 192) ? ATTR_MX_192 : ATTR_MX_256;
     if (!ctx->attr_set[inst]) {
         if (cudaFuncSetAttribute(qgemm_mx_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess) {
             cudaGetLastError();

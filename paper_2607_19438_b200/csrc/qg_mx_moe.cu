@@ -353,7 +353,7 @@ int moe_grouped_qgemm_mx(qg_ctx* ctx, int mode, int R, int E, int N, int K, cons
                              (wrows + 127) / 128, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (rc != QG_OK) return rc;
     const bool gu = (mode == QG_MODE_GATE_UP_SILU);
-    const int inst = gu ? 37 : 36;              // slots of the per-context "attribute set" flags
+    const int inst = qg::ATTR_MX_MOE + (gu ? 1 : 0);
     if (!ctx->attr_set[inst]) {
         const cudaError_t e = gu
             ? cudaFuncSetAttribute(qg::qgemm_mx_moe_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, qg::MG_SMEM)

@@ -217,7 +217,7 @@ int moe_router_logits(qg_ctx* ctx, int M, int H, int E, const void* X, const voi
     const int nkb = H / qg::RT_BK;
     // four slices of H per tile (a cluster of four CTAs) unless there are CTAs enough without, or too few blocks
     const bool split = nkb >= 8 && static_cast<long long>(tiles_m) * tiles_e < 2LL * ctx->sm_count;
-    const int inst = split ? 31 : 23;        // slots of the per-context "attribute set" flags
+    const int inst = split ? qg::ATTR_ROUTER_4 : qg::ATTR_ROUTER_1;
     if (!ctx->attr_set[inst]) {
         const cudaError_t e = split
             ? cudaFuncSetAttribute(qg::router_logits_kernel_4, cudaFuncAttributeMaxDynamicSharedMemorySize, qg::RT_SMEM)
