@@ -134,68 +134,68 @@ int check_device(const qg_ctx* ctx) {
     return dev == ctx->device ? QG_OK : QG_ERR_DEVICE;
 }
 
-int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
-                uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz,
-                uint64_t row_stride_bytes) {
-    if (row_stride_bytes == 0) row_stride_bytes = inner * static_cast<uint64_t>(elem_bytes);
-    for (int i = 0; i < ctx->tmap_count; ++i) {
-        const TmapEntry& e = ctx->tmaps[i];
-        if (e.base == base && e.inner == inner && e.rows == rows && e.box_inner == box_inner && e.box_rows == box_rows &&
-            e.row_stride == row_stride_bytes && e.planes == 0 &&
-            e.dt == static_cast<int>(dt) && e.elem_bytes == elem_bytes && e.swz == static_cast<int>(swz)) {
-            *out = &e.map;
+// The cache is a table of TMAP_CACHE entries in sets of TMAP_WAYS: a key hashes to one set, a miss replaces the set's
+// ways in turn.  A hit or a fresh encode is copied out, so nothing a caller holds changes when a later lookup replaces
+// the entry.
+static int tmap_lookup(qg_ctx* ctx, CUtensorMap* out, const TmapEntry& key, uint32_t rank) {
+    uint64_t h = reinterpret_cast<uintptr_t>(key.base) >> 4;
+    h ^= key.inner * 0x9E3779B97F4A7C15ull;
+    h ^= (static_cast<uint64_t>(key.box_inner) << 40) ^ (static_cast<uint64_t>(key.box_rows) << 24) ^ (key.rows << 3) ^
+         static_cast<uint64_t>(key.swz) ^ (key.planes << 51);
+    h *= 0xD6E8FEB86659FD93ull;
+    const int set = static_cast<int>((h >> 32) % (TMAP_CACHE / TMAP_WAYS)) * TMAP_WAYS;
+    for (int w = 0; w < TMAP_WAYS; ++w) {
+        const TmapEntry& e = ctx->tmaps[set + w];
+        if (e.base == key.base && e.inner == key.inner && e.rows == key.rows && e.box_inner == key.box_inner &&
+            e.box_rows == key.box_rows && e.row_stride == key.row_stride && e.planes == key.planes &&
+            e.plane_stride == key.plane_stride && e.box_planes == key.box_planes && e.dt == key.dt &&
+            e.elem_bytes == key.elem_bytes && e.swz == key.swz) {
+            *out = e.map;
             return QG_OK;
         }
     }
-    TmapEntry& e = ctx->tmaps[ctx->tmap_next];
-    cuuint64_t dims[2] = {inner, rows};
-    cuuint64_t strides[1] = {row_stride_bytes};
-    cuuint32_t box[2] = {box_inner, box_rows};
-    cuuint32_t estr[2] = {1, 1};
+    int way = -1;
+    for (int w = 0; w < TMAP_WAYS && way < 0; ++w)
+        if (!ctx->tmaps[set + w].base) way = w;
+    if (way < 0) way = static_cast<int>(ctx->tmap_next++ % TMAP_WAYS);
+    TmapEntry& e = ctx->tmaps[set + way];
+    cuuint64_t dims[3] = {key.inner, key.rows, key.planes};
+    cuuint64_t strides[2] = {key.row_stride, key.plane_stride};
+    cuuint32_t box[3] = {key.box_inner, key.box_rows, key.box_planes};
+    cuuint32_t estr[3] = {1, 1, 1};
     e.base = nullptr;      // not a valid entry while it is being rewritten
-    CUresult r = ctx->encode_tiled(&e.map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
-                                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    const CUresult r = ctx->encode_tiled(&e.map, static_cast<CUtensorMapDataType>(key.dt), rank, const_cast<void*>(key.base),
+                                         dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                         static_cast<CUtensorMapSwizzle>(key.swz), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return QG_ERR_CUDA;
-    e.base = base; e.inner = inner; e.rows = rows; e.row_stride = row_stride_bytes; e.box_inner = box_inner; e.box_rows = box_rows;
-    e.planes = 0; e.plane_stride = 0; e.box_planes = 0;
-    e.dt = static_cast<int>(dt); e.elem_bytes = elem_bytes; e.swz = static_cast<int>(swz);
-    *out = &e.map;
-    ctx->tmap_next = (ctx->tmap_next + 1) % TMAP_CACHE;
-    if (ctx->tmap_count < TMAP_CACHE) ++ctx->tmap_count;
+    const CUtensorMap keep = e.map;
+    e = key;
+    e.map = keep;
+    *out = e.map;
     return QG_OK;
 }
 
-int get_tmap_3d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
+int get_tmap_2d(qg_ctx* ctx, CUtensorMap* out, CUtensorMapDataType dt, int elem_bytes, const void* base,
+                uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz,
+                uint64_t row_stride_bytes) {
+    TmapEntry key{};
+    key.base = base; key.inner = inner; key.rows = rows;
+    key.row_stride = row_stride_bytes ? row_stride_bytes : inner * static_cast<uint64_t>(elem_bytes);
+    key.box_inner = box_inner; key.box_rows = box_rows;
+    key.planes = 0; key.plane_stride = 0; key.box_planes = 0;
+    key.dt = static_cast<int>(dt); key.elem_bytes = elem_bytes; key.swz = static_cast<int>(swz);
+    return tmap_lookup(ctx, out, key, 2);
+}
+
+int get_tmap_3d(qg_ctx* ctx, CUtensorMap* out, CUtensorMapDataType dt, int elem_bytes, const void* base,
                 uint64_t inner, uint64_t rows, uint64_t planes, uint64_t plane_stride_bytes, uint32_t box_inner,
                 uint32_t box_rows, uint32_t box_planes, CUtensorMapSwizzle swz) {
-    const uint64_t row_stride_bytes = inner * static_cast<uint64_t>(elem_bytes);
-    for (int i = 0; i < ctx->tmap_count; ++i) {
-        const TmapEntry& e = ctx->tmaps[i];
-        if (e.base == base && e.inner == inner && e.rows == rows && e.box_inner == box_inner && e.box_rows == box_rows &&
-            e.row_stride == row_stride_bytes && e.planes == planes && e.plane_stride == plane_stride_bytes &&
-            e.box_planes == box_planes &&
-            e.dt == static_cast<int>(dt) && e.elem_bytes == elem_bytes && e.swz == static_cast<int>(swz)) {
-            *out = &e.map;
-            return QG_OK;
-        }
-    }
-    TmapEntry& e = ctx->tmaps[ctx->tmap_next];
-    cuuint64_t dims[3] = {inner, rows, planes};
-    cuuint64_t strides[2] = {row_stride_bytes, plane_stride_bytes};
-    cuuint32_t box[3] = {box_inner, box_rows, box_planes};
-    cuuint32_t estr[3] = {1, 1, 1};
-    e.base = nullptr;      // not a valid entry while it is being rewritten
-    CUresult r = ctx->encode_tiled(&e.map, dt, 3, const_cast<void*>(base), dims, strides, box, estr,
-                                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return QG_ERR_CUDA;
-    e.base = base; e.inner = inner; e.rows = rows; e.row_stride = row_stride_bytes; e.box_inner = box_inner; e.box_rows = box_rows;
-    e.planes = planes; e.plane_stride = plane_stride_bytes; e.box_planes = box_planes;
-    e.dt = static_cast<int>(dt); e.elem_bytes = elem_bytes; e.swz = static_cast<int>(swz);
-    *out = &e.map;
-    ctx->tmap_next = (ctx->tmap_next + 1) % TMAP_CACHE;
-    if (ctx->tmap_count < TMAP_CACHE) ++ctx->tmap_count;
-    return QG_OK;
+    TmapEntry key{};
+    key.base = base; key.inner = inner; key.rows = rows; key.row_stride = inner * static_cast<uint64_t>(elem_bytes);
+    key.box_inner = box_inner; key.box_rows = box_rows;
+    key.planes = planes; key.plane_stride = plane_stride_bytes; key.box_planes = box_planes;
+    key.dt = static_cast<int>(dt); key.elem_bytes = elem_bytes; key.swz = static_cast<int>(swz);
+    return tmap_lookup(ctx, out, key, 3);
 }
 }  // namespace qg

@@ -396,7 +396,7 @@ template <int D>
 static int launch_attn(qg_ctx* ctx, const AttnParams& p, const void* Q, long long ldq, const void* K, long long ldk,
                        const void* V, long long ldv, cudaStream_t st) {
     using C = AttnCfg<D>;
-    const CUtensorMap *tm_q, *tm_k, *tm_v;
+    CUtensorMap tm_q, tm_k, tm_v;
     int rc = get_tmap_2d(ctx, &tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, static_cast<uint64_t>(p.Hq) * D, p.S, 64, 128,
                          CU_TENSOR_MAP_SWIZZLE_128B, static_cast<uint64_t>(ldq) * 2);
     if (rc == QG_OK)
@@ -416,7 +416,7 @@ static int launch_attn(qg_ctx* ctx, const AttnParams& p, const void* Q, long lon
         ctx->attr_set[inst] = true;
     }
     const int n_qb = (p.S + 2 * AT_BQ - 1) / (2 * AT_BQ);
-    if (launch_kernel(ctx, kern, dim3(p.Hq, n_qb), dim3(AT_THREADS), C::SMEM_BYTES, st, *tm_q, *tm_k, *tm_v, p) != cudaSuccess) {
+    if (launch_kernel(ctx, kern, dim3(p.Hq, n_qb), dim3(AT_THREADS), C::SMEM_BYTES, st, tm_q, tm_k, tm_v, p) != cudaSuccess) {
         cudaGetLastError();
         return QG_ERR_CUDA;
     }

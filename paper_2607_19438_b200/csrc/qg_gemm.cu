@@ -901,7 +901,7 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_ro
                        cudaStream_t st) {
     using C = Cfg<QBITS, BT>;
     static_assert(C::SMEM_BYTES <= 232448, "shared memory budget");
-    const CUtensorMap *tm_x, *tm_w, *tm_s;       // cached in the context: the same buffers recur every layer and step
+    CUtensorMap tm_x, tm_w, tm_s;       // cached in the context: the same buffers recur every layer and step
     const uint64_t wrows = static_cast<uint64_t>(p.E) * p.N;
     // activations: a box of half a token tile, or of a single row when the rows are gathered four at a time
     int rc = get_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, p.K, x_rows, BK,
@@ -937,7 +937,7 @@ static int launch_gemm(qg_ctx* ctx, const GemmParams& p, const void* X, int x_ro
     if (p.streamk) max_tiles *= p.K / (4 * BK);      // units of four k-blocks: every pair gets at least one
     const long long pairs_hw = ctx->sm_count / 2;
     const int grid = 2 * static_cast<int>(max_tiles < pairs_hw ? max_tiles : pairs_hw);
-    if (launch_kernel(ctx, kern, dim3(grid), dim3(NTHREADS), C::SMEM_BYTES, st, *tm_x, *tm_w, *tm_s, p) != cudaSuccess) {
+    if (launch_kernel(ctx, kern, dim3(grid), dim3(NTHREADS), C::SMEM_BYTES, st, tm_x, tm_w, tm_s, p) != cudaSuccess) {
         cudaGetLastError();
         return QG_ERR_CUDA;
     }

@@ -19,7 +19,7 @@ struct TmapEntry {
     int dt, elem_bytes, swz;
     CUtensorMap map;
 };
-constexpr int TMAP_CACHE = 64;
+constexpr int TMAP_CACHE = 2048, TMAP_WAYS = 8;   // entries, entries per hashed set
 constexpr uint32_t DEFAULT_WAIT_LIMIT = 1u << 18;   // polls; an unsatisfied try_wait poll lasts about 4 us: about a second
 // Slots of qg_ctx::attr_set, one per kernel instantiation that needs the dynamic shared-memory attribute.
 enum AttrSlot {
@@ -32,8 +32,8 @@ enum AttrSlot {
     ATTR_ROUTER_4 = 31,
     ATTR_MX_MOE = 32,       // 2: down, gate/up
     ATTR_MX_256 = 34,
-    ATTR_GEMV_RING = 35,    // 2: Q8, Q4
-    ATTR_SLOTS = 37
+    ATTR_GEMV_RING = 35,    // 4: format (2) x more than eight tokens (2)
+    ATTR_SLOTS = 39
 };
 }  // namespace qg
 
@@ -49,7 +49,7 @@ struct qg_ctx {
     int skip_kb;               // test hook, consumed by the next GEMM launch (-1: none)
     bool attr_set[qg::ATTR_SLOTS];        // per kernel instantiation: dynamic shared-memory attribute set on this device
     qg::TmapEntry tmaps[qg::TMAP_CACHE];   // tensor maps of recent calls (weights and buffers recur every layer)
-    int tmap_count, tmap_next;
+    unsigned tmap_next;        // replacement counter
     bool pdl;                  // launch kernels with programmatic stream serialization (QG_NO_PDL=1 turns it off)
     float* sk_partial;         // stream-K: one fp32 partial tile (256 tokens x 128 rows) per CTA
     int* sk_flags;             // stream-K: two counters per CTA, zero between launches
@@ -81,14 +81,14 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // QG_OK if the calling thread's current device is the context's, else QG_ERR_DEVICE.
 int check_device(const qg_ctx* ctx);
 // A 2-D row-major tensor map (inner = contiguous extent in elements, box in elements, row_stride_bytes = distance
-// between rows, 0 = packed): looked up in the context's cache, encoded on a miss.  The returned pointer stays valid
-// until TMAP_CACHE further misses.
-int get_tmap_2d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
+// between rows, 0 = packed): looked up in the context's cache, encoded on a miss, and copied to *out (the caller's own
+// copy: a later lookup may replace the cached entry).
+int get_tmap_2d(qg_ctx* ctx, CUtensorMap* out, CUtensorMapDataType dt, int elem_bytes, const void* base,
                 uint64_t inner, uint64_t rows, uint32_t box_inner, uint32_t box_rows, CUtensorMapSwizzle swz,
                 uint64_t row_stride_bytes = 0);
 // The same with a third dimension: `planes` planes of `rows` rows, plane_stride_bytes apart; box = box_inner x box_rows x
 // box_planes, which lands in shared memory plane after plane.
-int get_tmap_3d(qg_ctx* ctx, const CUtensorMap** out, CUtensorMapDataType dt, int elem_bytes, const void* base,
+int get_tmap_3d(qg_ctx* ctx, CUtensorMap* out, CUtensorMapDataType dt, int elem_bytes, const void* base,
                 uint64_t inner, uint64_t rows, uint64_t planes, uint64_t plane_stride_bytes, uint32_t box_inner,
                 uint32_t box_rows, uint32_t box_planes, CUtensorMapSwizzle swz);
 }  // namespace qg

@@ -442,7 +442,7 @@ template <int BN>
 static int launch_mx_dense(qg_ctx* ctx, int M, int N, int K, const void* A_codes, const void* A_scales, const void* W_codes,
                            const void* W_scales, void* Cout, void* stream) {
     using C = MxCfg<BN>;
-    const CUtensorMap *tm_a, *tm_w, *tm_sa, *tm_sw;
+    CUtensorMap tm_a, tm_w, tm_sa, tm_sw;
     const int nch = K / MX_BK;
     int rc = get_tmap_2d(ctx, &tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, A_codes, K, M, MX_BK, MX_BM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc == QG_OK)
@@ -469,7 +469,7 @@ static int launch_mx_dense(qg_ctx* ctx, int M, int N, int K, const void* A_codes
     p.C = static_cast<__nv_bfloat16*>(Cout); p.status = ctx->d_status; p.wait_limit = ctx->wait_limit;
     const int pairs = p.tiles < ctx->sm_count / 2 ? p.tiles : ctx->sm_count / 2;
     return launch_rc(launch_kernel(ctx, qgemm_mx_kernel<BN>, dim3(2 * pairs), dim3(MX_THREADS), C::SMEM,
-                                   static_cast<cudaStream_t>(stream), *tm_a, *tm_w, *tm_sa, *tm_sw, p));
+                                   static_cast<cudaStream_t>(stream), tm_a, tm_w, tm_sa, tm_sw, p));
 }
 
 }  // namespace qg

@@ -341,7 +341,7 @@ int moe_grouped_qgemm_mx(qg_ctx* ctx, int mode, int R, int E, int N, int K, cons
     if (const int rc = qg::check_device(ctx)) return rc;
     const int nch = K / qg::MG_BK;
     const uint64_t wrows = static_cast<uint64_t>(E) * N;
-    const CUtensorMap *tm_a, *tm_w, *tm_sa, *tm_sw;
+    CUtensorMap tm_a, tm_w, tm_sa, tm_sw;
     int rc = qg::get_tmap_2d(ctx, &tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, A_codes, K, R, qg::MG_BK, qg::MG_BM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc == QG_OK)
         rc = qg::get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W_codes, K, wrows, qg::MG_BK, qg::MG_BH, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -372,8 +372,8 @@ int moe_grouped_qgemm_mx(qg_ctx* ctx, int mode, int R, int E, int N, int K, cons
     const long long max_tiles = (static_cast<long long>((R + qg::MG_BM - 1) / qg::MG_BM) + E) * p.n_wt;
     const int grid = static_cast<int>(max_tiles < ctx->sm_count ? max_tiles : ctx->sm_count);
     const cudaError_t le = gu
-        ? qg::launch_kernel(ctx, qg::qgemm_mx_moe_kernel<1>, dim3(grid), dim3(qg::MG_THREADS), qg::MG_SMEM, static_cast<cudaStream_t>(stream), *tm_a, *tm_w, *tm_sa, *tm_sw, p)
-        : qg::launch_kernel(ctx, qg::qgemm_mx_moe_kernel<0>, dim3(grid), dim3(qg::MG_THREADS), qg::MG_SMEM, static_cast<cudaStream_t>(stream), *tm_a, *tm_w, *tm_sa, *tm_sw, p);
+        ? qg::launch_kernel(ctx, qg::qgemm_mx_moe_kernel<1>, dim3(grid), dim3(qg::MG_THREADS), qg::MG_SMEM, static_cast<cudaStream_t>(stream), tm_a, tm_w, tm_sa, tm_sw, p)
+        : qg::launch_kernel(ctx, qg::qgemm_mx_moe_kernel<0>, dim3(grid), dim3(qg::MG_THREADS), qg::MG_SMEM, static_cast<cudaStream_t>(stream), tm_a, tm_w, tm_sa, tm_sw, p);
     if (le != cudaSuccess) {
         cudaGetLastError();
         return QG_ERR_CUDA;

@@ -208,7 +208,7 @@ int moe_router_logits(qg_ctx* ctx, int M, int H, int E, const void* X, const voi
     if (!X || !Wr || !logits) return QG_ERR_NULL;
     if (!qg::aligned16(X) || !qg::aligned16(Wr)) return QG_ERR_ALIGN;
     if (const int rc = qg::check_device(ctx)) return rc;
-    const CUtensorMap *tm_x, *tm_w;
+    CUtensorMap tm_x, tm_w;
     int rc = qg::get_tmap_2d(ctx, &tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, H, M, qg::RT_BK, qg::RT_BM, CU_TENSOR_MAP_SWIZZLE_128B);
     if (rc == QG_OK)
         rc = qg::get_tmap_2d(ctx, &tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Wr, H, E, qg::RT_BK, 128, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -234,8 +234,8 @@ int moe_router_logits(qg_ctx* ctx, int M, int H, int E, const void* X, const voi
     p.L = logits; p.status = ctx->d_status; p.wait_limit = ctx->wait_limit;
     const dim3 grid(tiles_m, split ? 4 : 1, tiles_e);
     const cudaError_t le = split
-        ? qg::launch_kernel(ctx, qg::router_logits_kernel_4, grid, dim3(qg::RT_THREADS), qg::RT_SMEM, static_cast<cudaStream_t>(stream), *tm_x, *tm_w, p)
-        : qg::launch_kernel(ctx, qg::router_logits_kernel_1, grid, dim3(qg::RT_THREADS), qg::RT_SMEM, static_cast<cudaStream_t>(stream), *tm_x, *tm_w, p);
+        ? qg::launch_kernel(ctx, qg::router_logits_kernel_4, grid, dim3(qg::RT_THREADS), qg::RT_SMEM, static_cast<cudaStream_t>(stream), tm_x, tm_w, p)
+        : qg::launch_kernel(ctx, qg::router_logits_kernel_1, grid, dim3(qg::RT_THREADS), qg::RT_SMEM, static_cast<cudaStream_t>(stream), tm_x, tm_w, p);
     if (le != cudaSuccess) {
         cudaGetLastError();
         return QG_ERR_CUDA;

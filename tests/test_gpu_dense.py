@@ -140,3 +140,32 @@ def test_dense_gate_up_with_fused_silu(qbits, M, F, K):
     qg.poll_status()
     assert g.intact() and not bool(g.untouched_inside().any().item())
     util.assert_close(util.host_bf16_f64(g.t), orc.silu_mul(orc.qgemm_dense(qbits, A, Wq, Ws)), "dense gate/up + silu")
+
+
+def test_dense_many_distinct_weight_buffers_through_one_context():
+    """A model has hundreds of weight matrices and one set of activation buffers: the activation map is found in the
+    context's tensor-map cache on every call while weight maps keep replacing older entries.  Every call must use the
+    maps of its own arguments (a cached entry handed out by reference and then replaced made the kernel copy with
+    another buffer's map and run into its wait limit)."""
+    qbits, M, N, K = 4, 16, 256, 256
+    A, _, _ = synth.dense_problem(qbits, M, N, K, seed=11)
+    dA = util.dev_bf16(A)
+    out = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    n_weights = 2600                                             # more than the cache holds
+    Wq0 = synth.weights_q4(N, K, 11, 1)
+    Ws = util.dev_f16(synth.scales(N, K // 32, 7, 11, 2))
+    pool = torch.empty((n_weights, N, K // 2), dtype=torch.uint8, device="cuda")
+    pool[:] = util.dev(Wq0)[None]
+    marks = {0: 0x11, 1037: 0x5A, n_weights - 1: 0xC3}            # three buffers with their own codes in row 0
+    for i, byte in marks.items():
+        pool[i, 0, :] = byte
+    results = {}
+    for rep in range(2):
+        for i in range(n_weights):
+            qg.qgemm_dense(qbits, dA, pool[i], Ws, out=out)
+            if i in marks:
+                results[(rep, i)] = out.clone()
+    qg.poll_status()
+    for (rep, i), got in results.items():
+        Wq = Wq0.copy(); Wq[0, :] = marks[i]
+        util.assert_close(util.host_bf16_f64(got), orc.qgemm_dense(qbits, A, Wq, synth.scales(N, K // 32, 7, 11, 2)), f"buffer {i} pass {rep}")
