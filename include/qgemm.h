@@ -97,8 +97,13 @@ int qg_set_schedule(qg_ctx* ctx, int token_tile, int streamk_mode);
  * context leaves out the activation load of k-block `skip_kblock` of each CTA's first tile (-1: none), so
  * that a wait in that launch runs out.  The launch then returns normally and qg_poll_status() reports
  * QG_ERR_TIMEOUT; the context stays usable.  Never needed in production.
+ * For qgemm_small_m's ring kernel `skip_kblock` is the index of a 16 KB weight stage that its first CTA never loads.
+ * qg_test_gemv_mode chooses qgemm_small_m's kernel for the calls that follow: bit 0 = no thread-block clusters (K slices
+ * are then added through the scratch), bit 1 = always the ring kernel, bit 2 = never (bits 1 and 2 exclude each other;
+ * 0 = the library's own choice).
  */
 int qg_test_inject(qg_ctx* ctx, unsigned wait_limit_polls, int skip_kblock);
+int qg_test_gemv_mode(qg_ctx* ctx, int mode);
 
 /*
  * Dense quantised GEMM (Sec. 3.1: the dense projection over 4-bit / 8-bit block-quantised weights, read in
@@ -120,11 +125,16 @@ int qgemm_dense_gate_up_silu(qg_ctx* ctx, int qbits, int M, int F, int K, const 
 /*
  * The same product for 1 <= M <= 16 tokens (else QG_ERR_SHAPE): the decode-side and small verification-batch
  * regime that Sec. 2.3 describes as bound by memory bandwidth and Sec. 5.2 names as future work for the tensor
- * path.  Every weight byte is used once, so this call streams the packed weights: matrices below about 48 M weights
- * (and fewer than 16384 rows) by a kernel of its own that reduces its K slices in a fixed order (results do not depend
- * on scheduling), larger ones by qgemm_dense's kernel, which is faster there (and whose last bf16 place may differ
- * between runs, see qgemm_dense).  Same formats, constraints and numerics (weights rounded once to bf16, fp32
- * accumulate) as qgemm_dense; uses the context's scratch, so calls on one context must not overlap on the GPU.
+ * path.  Every weight byte is used once, so this call streams the packed weights.  Depending on format, size and
+ * token count it is served by a persistent kernel whose weights arrive through a TMA-fed shared-memory ring (up to
+ * eight tokens, and small 4-bit matrices at any count), by a small-block kernel, or by qgemm_dense's kernel (large
+ * matrices at more than eight tokens).  The first two add in a fixed order (K phases in order inside a CTA, K slices in
+ * slice order across CTAs), so their results do not depend on scheduling; for qgemm_dense's kernel see there.
+ * Same formats and constraints as qgemm_dense, fp32 accumulation.  Numerics: the 8-bit path and the other two kernels
+ * multiply weights rounded once to bf16 (q * scale), as qgemm_dense does; the ring kernel's 4-bit path multiplies the
+ * exact integers q and applies the block's scale to the fp32 sum of each 32-block, which is closer to the exact value
+ * (both are within the library's tolerance of it).  Uses the context's scratch, so calls on one context must not
+ * overlap on the GPU.
  */
 int qgemm_small_m(qg_ctx* ctx, int qbits, int M, int N, int K, const void* A, const void* Wq,
                   const void* Wscale, void* C, void* stream);

@@ -18,7 +18,7 @@ QG_Q8, QG_Q4 = 8, 4
 MODE_PLAIN, MODE_GATE_UP_SILU, MODE_DOWN_WEIGHTED, MODE_DOWN_ACCUM_F32 = 0, 1, 2, 3
 D_BF16, D_F32_ACC = 0, 1
 
-EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_plan_dense", "qg_set_schedule", "qg_route_workspace_bytes",
+EXPORTS = ["qg_create", "qg_destroy", "qg_strerror", "qg_poll_status", "qg_test_inject", "qg_test_gemv_mode", "qg_plan_dense", "qg_set_schedule", "qg_route_workspace_bytes",
            "qgemm_dense", "qgemm_small_m", "qgemm_dense_gate_up_silu", "prefill_attention",
            "qg_mx_scale_bytes", "qg_mx_quantize", "qg_mx_pack_weights", "qgemm_mx_dense",
            "moe_route", "moe_route_static", "moe_permute", "moe_grouped_qgemm", "moe_grouped_qgemm_gather", "moe_combine",
@@ -51,6 +51,7 @@ def load():
         lib.qg_destroy.argtypes = [C.c_void_p]
         lib.qg_poll_status.argtypes = [C.c_void_p, C.c_void_p]
         lib.qg_test_inject.argtypes = [C.c_void_p, C.c_uint, C.c_int]
+        lib.qg_test_gemv_mode.argtypes = [C.c_void_p, C.c_int]
         lib.qg_plan_dense.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         lib.qg_set_schedule.argtypes = [C.c_void_p, C.c_int, C.c_int]
         vp, ci = C.c_void_p, C.c_int
@@ -127,6 +128,11 @@ def test_inject(wait_limit_polls: int = 0, skip_kblock: int = -1):
     """Testing hook: bounded-wait limit in polls (0 = default) and the k-block whose activation load the next GEMM
     launch leaves out (-1 = none)."""
     _check(load().qg_test_inject(context(), wait_limit_polls, skip_kblock), "qg_test_inject")
+
+
+def test_gemv_mode(mode: int = 0):
+    """Testing hook: kernel choice of qgemm_small_m (bit 0 no clusters, bit 1 always the ring kernel, bit 2 never)."""
+    _check(load().qg_test_gemv_mode(context(), mode), "qg_test_gemv_mode")
 
 
 def plan_dense(qbits, M, N, K):

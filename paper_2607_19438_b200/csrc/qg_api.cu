@@ -118,6 +118,13 @@ int qg_set_schedule(qg_ctx* ctx, int token_tile, int streamk_mode) {
 void qg_debug_set_stats(qg_ctx* ctx, long long* dev_buf) { if (ctx) ctx->stats = dev_buf; }
 #endif
 
+int qg_test_gemv_mode(qg_ctx* ctx, int mode) {
+    if (!ctx) return QG_ERR_NULL;
+    if (mode < 0 || mode > 7 || (mode & 6) == 6) return QG_ERR_SHAPE;
+    ctx->gemv_mode = mode;
+    return QG_OK;
+}
+
 int qg_test_inject(qg_ctx* ctx, unsigned wait_limit_polls, int skip_kblock) {
     if (!ctx) return QG_ERR_NULL;
     ctx->wait_limit = wait_limit_polls ? wait_limit_polls : qg::DEFAULT_WAIT_LIMIT;

@@ -58,6 +58,8 @@ struct qg_ctx {
     size_t gemv_partial_bytes;
     int* gemv_tickets;         // one arrival counter per 64-row tile, zero between launches
     int gemv_ticket_count;
+    int gemv_mode;             // test hook (qg_test_gemv_mode): bit 0 no clusters, bit 1 always the ring kernel, bit 2 never
+    int gemv_max_clusters[4][9];   // ring kernel, per instantiation and cluster size: clusters that fit at once (0 unknown, -1 none)
     long long* stats;          // profiling builds only
 };
 
