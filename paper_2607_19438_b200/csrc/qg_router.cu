@@ -5,8 +5,8 @@
 //   products exact, fp32 accumulation in a fixed order.
 //
 // About one GFLOP at the model shapes (2048 x 128 x 2048) against the layer's 150, so latency decides: a first version
-// on mma.sync tiles needed 15-20 us whatever its tiling or loads (a legacy mma.sync.m16n8k16 issues only every ~19
-// cycles per scheduler on this GPU).  This one is a tcgen05 kernel: a CTA owns 128 tokens x up to 256 experts x one
+// on mma.sync tiles needed 15-20 us whatever its tiling or loads (its warps ran short chains of dependent
+// mma.sync.m16n8k16, each of which waits about 20 cycles for the one before).  This one is a tcgen05 kernel: a CTA owns 128 tokens x up to 256 experts x one
 // slice of H; both operands arrive by TMA (128-byte swizzle, four stages of 64 h) and are multiplied from shared memory
 // into a tensor-memory accumulator (one issuing thread, four MMAs per stage in one statement).  H is cut into four
 // slices, one per CTA of a cluster, so that enough CTAs exist; each leaves its fp32 partial tile in its own (by then
