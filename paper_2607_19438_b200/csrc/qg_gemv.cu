@@ -1,19 +1,20 @@
 // Small-batch (1..16 tokens) block-quantised GEMM for sm_100a: the weight-streaming, HBM-bound end of the operator.
 //
 // Operation: C[m, n] = sum_k A[m, k] * q[n, k] * scale[n, k/32], the definition of qgemm_dense, for M <= 16.  With so
-// few tokens every weight byte is used once, so the kernel is a streaming read of the packed weights at HBM speed;
-// the arithmetic (16 x 8 x 16 bf16 tensor-core tiles, mma.sync) only has to keep up.  The weights are dequantised
-// exactly as in the prefill kernel (fp32 product code x scale, one rounding to bf16), so both kernels multiply
-// the same bf16 weights.
+// few tokens every weight byte is used once, so the call is a streaming read of the packed weights; the arithmetic
+// (16 x 8 x 16 bf16 tensor-core tiles, mma.sync) only has to keep up.  Two kernels live here, and qgemm_small_m at the
+// end of the file chooses between them and the prefill kernel:
 //
-// Work split.  A block owns 64 weight rows x one K slice; its 8 warps own 8 rows each.  The token rows of the slice
-// (16 x KS bf16, rows past M zero) and the slice's scales sit in shared memory.  Lane (g, j) = (lane / 4, lane % 4)
-// streams the 16 codes k = 16 j .. 16 j + 15 of row g of every 64-wide chunk straight from global memory (16 or 8
-// bytes per load, eight loads in flight, the first ones issued before anything else in the kernel) and feeds four
-// MMAs with them; the summation index inside a chunk is permuted the same way on the activation side, so no
-// shuffles are needed.  K slices of one row tile are reduced in a fixed order by
-// whichever block finishes last (partial tiles in the context's workspace, one ticket per row tile), so the result
-// does not depend on the order in which blocks run.
+//  1. qgemv_kernel, the small-block kernel.  A block owns 64 weight rows x one K slice; its 8 warps own 8 rows each.
+//     The token rows of the slice (16 x KS bf16, rows past M zero) and the slice's scales sit in shared memory.  Lane
+//     (g, j) = (lane / 4, lane % 4) streams the 16 codes k = 16 j .. 16 j + 15 of row g of every 64-wide chunk straight
+//     from global memory (16 or 8 bytes per load, eight loads in flight, the first ones issued before anything else in
+//     the kernel), dequantises them exactly as the prefill kernel does (fp32 product code x scale, one rounding to
+//     bf16) and feeds four MMAs with them; the summation index inside a chunk is permuted the same way on the
+//     activation side, so no shuffles are needed.  K slices of one row tile are reduced in a fixed order by whichever
+//     block finishes last (partial tiles in the context's workspace, one ticket per row tile), so the result does not
+//     depend on the order in which blocks run.
+//  2. qgemv_ring_kernel, persistent CTAs fed by a TMA ring (described where it starts).
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
