@@ -129,3 +129,27 @@ def test_config4_gate_up_projection_sampled():
     out = qg.qgemm_dense(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws))
     qg.poll_status()
     _sampled_on_device(qbits, A, Wq, Ws, out, per_tile=1, seed=4)
+
+
+# the small-batch rows of the bench's sweep: every projection of the cfg-1 (Q8) and cfg-2 (Q4) layer sets at 1, 4 and 16
+# tokens, plus the largest cfg-4 matrices, through qgemm_small_m as the library dispatches it
+SMALL_M = [(8, M, N, K) for M in (1, 4, 16) for N, K in ((2560, 2048), (2048, 2048), (16384, 2048), (2048, 8192))] + \
+          [(4, M, N, K) for M in (1, 4, 16) for N, K in ((5120, 3072), (3072, 3072), (16384, 3072), (3072, 8192))] + \
+          [(8, 4, 28672, 4096), (8, 8, 4096, 14336), (4, 2, 28672, 4096)]
+
+
+@pytest.mark.parametrize("qbits,M,N,K", SMALL_M, ids=[f"q{c[0]}-{c[1]}x{c[2]}x{c[3]}" for c in SMALL_M])
+def test_small_m_full_size_sampled_rows(qbits, M, N, K):
+    """All tokens against a sample of weight rows: a few in every 128-row tile (the unit a CTA of the ring kernel owns),
+    the first and the last rows."""
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=3)
+    out = qg.qgemm_small_m(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws))
+    qg.poll_status()
+    out = util.host_bf16_f64(out)
+    rng = np.random.default_rng(N + K + M)
+    tiles = (N + 127) // 128
+    rows = np.unique(np.concatenate([np.minimum(np.arange(tiles) * 128 + rng.integers(0, 128, tiles), N - 1),
+                                     np.minimum(np.arange(tiles) * 128 + rng.integers(0, 128, tiles), N - 1),
+                                     np.arange(0, 8), np.arange(N - 8, N)]))
+    assert np.all(np.isfinite(out))
+    util.assert_close(out[:, rows], orc.qgemm_dense(qbits, A, Wq[rows], Ws[rows]), f"small-M q{qbits} {M}x{N}x{K}")
