@@ -227,7 +227,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int s = j & 1;
             // 16 keys per instruction: two 8-key groups of V; the next 64 head dimensions are one box further.  The
             // first 64 keys' products are issued as soon as their half of P is there, while the group still works on
-            // the other half (an MMA with its A operand in tensor memory takes about 125 cycles to issue).
+            // the other half (the four instructions occupy the tensor pipe for about 320 cycles).
             const uint32_t v_lo = ((sbase + C::OFF_V + s * C::TILE_BYTES) >> 4) | ((C::BOX_BYTES >> 4) << 16);
             if (!at_wait(p_full(t, 0), j & 1u, abort_flag, p) || !at_wait(v_full(s), (j >> 1) & 1u, abort_flag, p)) return false;
             tc_fence_after_sync();
