@@ -124,3 +124,24 @@ def test_fuzz_route_and_layer(i):
     assert np.array_equal(ro["topk_idx"].cpu().numpy().reshape(o["idx"].shape), o["idx"])
     assert np.array_equal(ro["row_pair"].cpu().numpy(), o["row_pair"]) and np.array_equal(ro["offsets"].cpu().numpy(), o["offsets"])
     util.assert_close(util.host_bf16_f64(y), o["y"], f"layer q{qbits} M={M} H={H} E={E} F={F} k={k}")
+
+
+@pytest.mark.parametrize("i", range(24))
+def test_fuzz_small_m(i):
+    """Random ragged shapes through qgemm_small_m with the kernel choice forced in turn (library's choice, ring kernel
+    with clusters, ring kernel with the scratch): tiles that end inside a 128-row block, K that does not divide into
+    equal slices or phases, every token count."""
+    r = _rng(500 + i)
+    qbits = int(r.choice([4, 8]))
+    M = int(r.integers(1, 17)); N = 8 * int(r.integers(1, 400)); K = 256 * int(r.integers(1, 25))
+    mode = (0, 2, 3)[i % 3]
+    A, Wq, Ws = synth.dense_problem(qbits, M, N, K, seed=i)
+    g = util.Guarded((M, N), torch.bfloat16)
+    try:
+        qg.test_gemv_mode(mode)
+        qg.qgemm_small_m(qbits, util.dev_bf16(A), util.dev(Wq), util.dev_f16(Ws), out=g.t)
+        qg.poll_status()
+    finally:
+        qg.test_gemv_mode(0)
+    assert g.intact() and not bool(g.untouched_inside().any().item())
+    util.assert_close(util.host_bf16_f64(g.t), orc.qgemm_dense(qbits, A, Wq, Ws), f"small-M q{qbits} {M}x{N}x{K} mode {mode}")
