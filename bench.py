@@ -306,7 +306,7 @@ def run_sweep(torch, qg, lib, ctx, dev, stream, peak_tf, peak_hbm, iters=20):
 
     # small batches (decode side): weight streaming, against the measured HBM copy bandwidth
     out["small_m"] = []
-    for name in ("cfg1_q8", "cfg2_q4"):
+    for name in ("cfg1_q8", "cfg2_q4", "cfg4_q8"):
         qbits, layers = LAYER_SETS[name]
         wbytes = sum(N * K * (1.0625 if qbits == 8 else 0.5625) for _, N, K in layers)
         ncopy = max(2, int(2 * L2_BYTES // wbytes) + 1)
