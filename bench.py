@@ -200,7 +200,11 @@ LAYER_SETS = {   # (label, N, K) of the four projections of one transformer laye
     "cfg2_q4": (4, [("qkv", 5120, 3072), ("o", 3072, 3072), ("gate_up", 16384, 3072), ("down", 3072, 8192)]),
     "cfg4_q8": (8, [("qkv", 6144, 4096), ("o", 4096, 4096), ("gate_up", 28672, 4096), ("down", 4096, 14336)]),
 }
-SWEEP_DENSE = [("cfg1_q8", 1024), ("cfg1_q8", 2048), ("cfg2_q4", 1024), ("cfg2_q4", 2048), ("cfg4_q8", 2048), ("cfg4_q8", 8192)]
+# the M sweep of the layer sets; below M = 1024 the weight stream (HBM) rather than the tensor pipe bounds a GEMM, the
+# rows are there for the shape of the curve
+SWEEP_DENSE = [("cfg1_q8", 128), ("cfg1_q8", 256), ("cfg1_q8", 512), ("cfg1_q8", 1024), ("cfg1_q8", 2048),
+               ("cfg2_q4", 128), ("cfg2_q4", 256), ("cfg2_q4", 512), ("cfg2_q4", 1024), ("cfg2_q4", 2048),
+               ("cfg4_q8", 2048), ("cfg4_q8", 4096), ("cfg4_q8", 8192)]
 SWEEP_MOE = [(1024, False), (2048, False), (2048, True), (8192, False), (8192, True)]
 L2_BYTES = 126e6
 
