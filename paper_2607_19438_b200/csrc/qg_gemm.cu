@@ -972,6 +972,8 @@ static DensePlan plan_dense(const qg_ctx* ctx, int qbits, int M, int n_wt, int K
             if (dp < best_cost) { best_cost = dp; best = DensePlan{cand[c], 0}; }
     }
     if (ctx->streamk_mode == 0) return best;
+    // Below K = 4096 the exchange never paid in the measurements (K = 2048 and 3072, 64 to 1024 tokens: 2 to 10 us slower).
+    if (ctx->streamk_mode != 1 && nk4 < 16) return best;
     for (int c = 0; c < 3; ++c) {
         if (M <= 128 && cand[c] > 128) break;
         const long long tiles = n_pw * ((M + cand[c] - 1) / cand[c]);
