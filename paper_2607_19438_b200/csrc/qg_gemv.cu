@@ -208,23 +208,31 @@ qgemv_kernel(const GemvParams p) {
 // ---------------------------------------------------------------------------------------------------------------------
 // The same operation with the weights arriving through a shared-memory ring fed by TMA.
 //
-// One persistent CTA per SM owns one K slice and walks over 128-row tiles of the weight matrix.  A producer warp keeps a
-// ring of 16 KB stages (128 rows x 128 bytes of codes, 128-byte swizzle) and two buffers of scale tiles full, so the
-// bytes in flight per SM (a hundred kilobytes) do not depend on registers or on how many warps are waiting.  Sixteen
-// consumer warps work in two sets of eight: set 0 takes the even stages of a tile, set 1 the odd ones, a warp 16 rows of
-// each.  The weights are the A operand of mma.sync.m16n8k16 (16 rows x 16 k) and up to eight tokens the B operand, so
-// one instruction covers 256 weights (two instructions when there are 9..16 tokens).  The token slice is copied to shared
-// memory once per CTA, in the order in which the lanes consume it.
+// Persistent CTAs, one per SM.  A CTA owns a range of K (all of it when there are row tiles enough to fill the GPU) and
+// walks over 128-row tiles of the weight matrix, once per phase of at most 2048 k (what fits in shared memory of the
+// token rows).  A producer warp keeps a ring of 16 KB stages (128 rows x 128 bytes of codes, 128-byte swizzle) and two
+// to eight buffers of scale tiles full, so the bytes in flight per SM (a hundred kilobytes and more) do not depend on
+// registers or on how many warps are waiting.  Sixteen consumer warps work in two sets of eight: set 0 takes the even
+// stages of a tile, set 1 the odd ones, a warp 16 rows of each.  The weights are the A operand of mma.sync.m16n8k16
+// (16 rows x 16 k) and up to eight tokens the B operand, so one instruction covers 256 weights (two instructions, and
+// two token fragments, when there are 9..16 tokens).  The token slice of a phase is copied to shared memory once per
+// CTA, in the order in which the lanes consume it.
 //   Q8: a lane converts 16 consecutive codes of its two rows per step exactly as the prefill kernel does (fp32 product
-//       with the block's scale, one rounding to bf16).
+//       with the block's scale, one rounding to bf16); the codes go to registers first and the slot straight back to
+//       the producer.
 //   Q4: the nibbles become the bf16 integers q = code - 8 with two logic operations and half a packed subtraction per
 //       pair (0x4300 | code is the bf16 number 128 + code); the two instructions of a 32-block accumulate into a scratch
 //       tile, which is then multiplied by the block's scale in fp32 and added to the running sum.  The result differs
 //       from the prefill kernel's in that the scaled weight is never rounded to bf16 (it is closer to the exact sum).
-// At the end of a tile set 1 hands its sums to set 0 through shared memory; set 0 writes bf16 outputs, or fp32 partial
-// sums when K is sliced, in which case the last CTA to finish a tile adds the slices in slice order (ticket per tile).
+// Output.  Both sets leave a tile's sums in shared memory and go on; three epilogue warps add them (and, from the
+// second phase on, what the phases before left in the CTA's rows of the scratch, in phase order) and write bf16
+// outputs, or fp32 partial sums when K is cut across CTAs.  The last tile is written by the consumers and the epilogue
+// warps together.  K cut across CTAs: when every CTA has one tile and the slices of a tile fit in a thread-block
+// cluster that is resident, each CTA keeps its partial tile in shared memory and the cluster adds the tiles through
+// distributed shared memory in slice order; otherwise whoever draws a tile's last ticket adds the slices from the
+// scratch in slice order.  All sums have a fixed order: results are bit-reproducible.
 // Every mbarrier wait is bounded; a warp whose wait expires records QG_ERR_TIMEOUT, stops computing and walks through
-// the remaining barriers so that nobody is left waiting for it.
+// the remaining barriers (and the cluster's) so that nobody is left waiting for it.
 
 constexpr int GR_ROWS = 128;                      // weight rows per tile
 constexpr int GR_STAGE_BYTES = GR_ROWS * 128;     // 16 KB: 128 k of Q8 codes, 256 k of Q4 codes per row
