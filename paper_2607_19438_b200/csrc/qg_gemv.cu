@@ -828,7 +828,18 @@ static int launch_gemv_ring(qg_ctx* ctx, int qbits, int M, int N, int K, const v
     cfg.attrs = at; cfg.numAttrs = n_at;
     if (cudaLaunchKernelEx(&cfg, kern, tm_w, tm_s, p) != cudaSuccess) {
         cudaGetLastError();
-        return QG_ERR_CUDA;
+        if (!best_cluster) return QG_ERR_CUDA;
+        // the cluster launch was refused although the occupancy query allowed it: remember that and add the slices
+        // through the scratch instead (if the scratch is large enough for this call)
+        ctx->gemv_max_clusters[variant][best_slices] = -1;
+        if (static_cast<size_t>(best_slices) * 16 * N * sizeof(float) > ctx->gemv_partial_bytes || tiles > ctx->gemv_ticket_count)
+            return QG_ERR_WORKSPACE;
+        p.cluster = 0;
+        cfg.numAttrs = n_at - 1;
+        if (cudaLaunchKernelEx(&cfg, kern, tm_w, tm_s, p) != cudaSuccess) {
+            cudaGetLastError();
+            return QG_ERR_CUDA;
+        }
     }
     return QG_OK;
 }
