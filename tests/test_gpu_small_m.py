@@ -146,3 +146,12 @@ def test_small_m_large_matrices_take_the_prefill_kernel(qbits, M, N, K):
     qg.poll_status()
     assert g.intact() and not bool(g.untouched_inside().any().item())
     util.assert_close(util.host_bf16_f64(g.t), orc.qgemm_dense(qbits, A, Wq, Ws), f"small-M via prefill kernel q{qbits} {M}x{N}x{K}")
+
+
+def test_gemv_mode_hook_rejects_contradictory_bits():
+    for bad in (-1, 6, 7, 8):
+        with pytest.raises(qg.QGemmError) as e:
+            qg.test_gemv_mode(bad)
+        assert e.value.code == -2
+    qg.test_gemv_mode(5)          # never the ring kernel, and no clusters: accepted
+    qg.test_gemv_mode(0)
